@@ -1,0 +1,265 @@
+"""ctypes front end of the CPU oracle (oracle/plc_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg call this;
+the CUDA library and its Python binding never do, and nothing here imports them.  The C file is
+compiled with gcc on first use (or by ``build()``) into ``oracle/libplc_oracle.so``.
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "plc_oracle.c")
+_SO = os.path.join(_HERE, "libplc_oracle.so")
+
+OK, E_INVALID, E_CAPACITY, E_CORRUPT = 0, 1, 4, 5
+Q_MIN, Q_MAX = -24, 135
+PROB_M = 1 << 15
+ESC = 63
+
+
+def build(force=False):
+    """Compile the oracle with gcc -O2 (no intrinsics, no threads)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+                               "-o", _SO, _SRC, "-lm"])
+    return _SO
+
+
+class Config(C.Structure):
+    _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("K", C.c_int32),
+                ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32), ("dense", C.c_int32)]
+
+
+class KVStrides(C.Structure):
+    _fields_ = [("layer", C.c_int64), ("kv", C.c_int64), ("session", C.c_int64), ("head", C.c_int64),
+                ("pos", C.c_int64)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("ideal_bits", C.c_double), ("token_bits", C.c_double), ("payload_bytes", C.c_uint64),
+                ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64), ("coded_positions", C.c_uint64)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.plo_half_to_double.restype = C.c_double
+        _lib.plo_half_to_double.argtypes = [C.c_uint16]
+        _lib.plo_round_bf16.restype = C.c_double
+        _lib.plo_round_bf16.argtypes = [C.c_double]
+        _lib.plo_class_from_v.argtypes = [C.c_float]
+        _lib.plo_class.argtypes = [C.c_double, C.c_float, C.c_float]
+    return _lib
+
+
+def _p(a, t=C.c_void_p):
+    return None if a is None else a.ctypes.data_as(t)
+
+
+def _h(a):
+    """fp16 array -> contiguous uint16 view."""
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float16, a.dtype
+    return a.view(np.uint16)
+
+
+def topk_softmax(logits, tokens, K):
+    """logits [N,V] float16, tokens [N] int32 or None -> idx [N,K] i32, w [N,K] f64, lse, zk, logp2 [N] f64."""
+    lg = _h(logits)
+    N, V = lg.shape
+    idx = np.zeros((N, K), np.int32)
+    w = np.zeros((N, K), np.float64)
+    lse = np.zeros(N, np.float64)
+    zk = np.zeros(N, np.float64)
+    lp = np.zeros(N, np.float64)
+    tk = None if tokens is None else np.ascontiguousarray(tokens, dtype=np.int32)
+    rc = lib().plo_topk_softmax(_p(lg), _p(tk), C.c_int64(N), V, K, _p(idx), _p(w), _p(lse), _p(zk), _p(lp))
+    if rc:
+        raise ValueError(f"plo_topk_softmax rc={rc}")
+    return idx, w, lse, zk, lp
+
+
+def mixture(table, idx, w):
+    """table [V,d] float16, idx [K], w [K] -> mu [d] f64, sigma2."""
+    tb = _h(table)
+    d = tb.shape[1]
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    mu = np.zeros(d, np.float64)
+    s2 = C.c_double()
+    lib().plo_mixture(_p(tb), d, _p(idx), _p(w), len(idx), _p(mu), C.byref(s2))
+    return mu, s2.value
+
+
+def dense_mixture(table, logits_row, lse):
+    tb = _h(table)
+    V, d = tb.shape
+    lg = _h(logits_row)
+    mu = np.zeros(d, np.float64)
+    s2 = C.c_double()
+    lib().plo_dense_mixture(_p(tb), V, d, _p(lg), C.c_double(lse), _p(mu), C.byref(s2))
+    return mu, s2.value
+
+
+def scale_class(sigma2, sigma_floor, delta):
+    return lib().plo_class(C.c_double(sigma2), C.c_float(sigma_floor), C.c_float(delta))
+
+
+def class_from_v(v):
+    return lib().plo_class_from_v(C.c_float(v))
+
+
+def class_params(q):
+    s, qp = C.c_int(), C.c_int()
+    lib().plo_class_params(int(q), C.byref(s), C.byref(qp))
+    return s.value, qp.value
+
+
+def quantise(kv, mu, delta):
+    x = _h(kv)
+    mu = np.ascontiguousarray(mu, dtype=np.float64)
+    sym = np.zeros(x.shape[0], np.int32)
+    lib().plo_quantise(_p(x), _p(mu), x.shape[0], C.c_float(delta), _p(sym))
+    return sym
+
+
+def reconstruct(mu, sym, delta):
+    mu = np.ascontiguousarray(mu, dtype=np.float64)
+    sym = np.ascontiguousarray(sym, dtype=np.int32)
+    out = np.zeros(len(sym), np.float32)
+    lib().plo_reconstruct(_p(mu), _p(sym), len(sym), C.c_float(delta), _p(out))
+    return out
+
+
+def table_constants(qp):
+    th, rh = C.c_uint32(), C.c_uint32()
+    rc = lib().plo_table_constants(int(qp), C.byref(th), C.byref(rh))
+    if rc:
+        raise ValueError("bad table id")
+    return th.value, rh.value
+
+
+def build_table(qp):
+    f = np.zeros(64, np.uint32)
+    c = np.zeros(65, np.uint32)
+    rc = lib().plo_build_table(int(qp), _p(f), _p(c))
+    if rc:
+        raise ValueError("bad table id")
+    return f, c
+
+
+def rans_encode_chunk(sym, q, cap=None):
+    """sym [P,d] int32, q [P] int32 -> (bytes ndarray u8, ideal_bits, n_escapes)."""
+    sym = np.ascontiguousarray(sym, dtype=np.int32)
+    q = np.ascontiguousarray(q, dtype=np.int32)
+    P, d = sym.shape
+    if cap is None:
+        cap = 128 + 8 * P * d + 64
+    out = np.zeros(cap, np.uint8)
+    nb, ideal, nesc = C.c_uint64(), C.c_double(), C.c_uint64()
+    rc = lib().plo_rans_encode_chunk(_p(sym), _p(q), P, d, _p(out), C.c_uint64(cap), C.byref(nb), C.byref(ideal),
+                                     C.byref(nesc))
+    if rc == E_CAPACITY:
+        raise OverflowError(nb.value)
+    if rc:
+        raise ValueError(f"plo_rans_encode_chunk rc={rc}")
+    return out[:nb.value].copy(), ideal.value, nesc.value
+
+
+def rans_decode_chunk(data, q, d):
+    """Returns (rc, sym [P,d])."""
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    q = np.ascontiguousarray(q, dtype=np.int32)
+    P = len(q)
+    sym = np.zeros((P, d), np.int32)
+    rc = lib().plo_rans_decode_chunk(_p(data), C.c_uint64(len(data)), _p(q), P, d, _p(sym))
+    return rc, sym
+
+
+def prefix_dedup(tokens, lens, logp2):
+    """tokens [S,n] i32, lens [S] i32, logp2 [S,n] f32 -> lcp [S,S] i32, dT [S,S] f64, parent, shared_len."""
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    lens = np.ascontiguousarray(lens, dtype=np.int32)
+    logp2 = np.ascontiguousarray(logp2, dtype=np.float32)
+    S, n = tokens.shape
+    lcp = np.zeros((S, S), np.int32)
+    dT = np.zeros((S, S), np.float64)
+    parent = np.zeros(S, np.int32)
+    shared = np.zeros(S, np.int32)
+    lib().plo_prefix_dedup(_p(tokens), _p(lens), _p(logp2), S, C.c_int64(n), _p(lcp), _p(dT), _p(parent), _p(shared))
+    return lcp, dT, parent, shared
+
+
+def _strides(kv):
+    """kv laid out [L,2,S,H,n,d] (any permutation of a contiguous array works): element strides."""
+    es = kv.itemsize
+    st = [s // es for s in kv.strides]
+    return KVStrides(st[0], st[1], st[2], st[3], st[4])
+
+
+def max_chunks_for(n, chunk_pos):
+    return (n + chunk_pos - 1) // chunk_pos
+
+
+def encode(cfg, T, kv, logits, tokens, pos_begin=None, pos_end=None, export=False):
+    """Whole-path encode.
+
+    T [L,2,H,V,d] f16; kv a float16 array indexed [L,2,S,H,n,d] (strides free, d contiguous);
+    logits [S,n,V] f16; tokens [S,n] i32 or None.  Returns a dict with payload, chunk_offset,
+    chunk_bytes ([S,L,2,H,max_chunks]), stats and, with export=True, sym/q/mu ([S,n,L,2,H(,d)]).
+    """
+    Tb = _h(T)
+    L, _, H, V, d = Tb.shape
+    assert kv.dtype == np.float16 and kv.strides[-1] == 2
+    kvv = kv.view(np.uint16)
+    lg = _h(logits)
+    S, n, _ = lg.shape
+    tk = None if tokens is None else np.ascontiguousarray(tokens, dtype=np.int32)
+    pb = None if pos_begin is None else np.ascontiguousarray(pos_begin, dtype=np.int32)
+    pe = None if pos_end is None else np.ascontiguousarray(pos_end, dtype=np.int32)
+    mc = max_chunks_for(n, cfg.chunk_pos)
+    nslots = S * L * 2 * H * mc
+    cap = nslots * (128 + 16) + 8 * S * n * L * 2 * H * d + 64   # worst case of the format
+    payload = np.zeros(cap, np.uint8)
+    off = np.zeros(nslots, np.uint64)
+    nby = np.zeros(nslots, np.uint32)
+    stats = Stats()
+    sym = q = mu = None
+    if export:
+        sym = np.zeros((S, n, L, 2, H, d), np.int32)
+        q = np.zeros((S, n, L, 2, H), np.int32)
+        mu = np.zeros((S, n, L, 2, H, d), np.float32)
+    st = _strides(kv)
+    rc = lib().plo_encode(C.byref(cfg), _p(Tb), C.c_void_p(kvv.ctypes.data), C.byref(st), _p(lg), _p(tk), S, n,
+                          _p(pb), _p(pe), mc, _p(payload), C.c_uint64(cap), _p(off), _p(nby), C.byref(stats),
+                          _p(sym), _p(q), _p(mu))
+    if rc:
+        raise ValueError(f"plo_encode rc={rc}")
+    shape = (S, L, 2, H, mc)
+    return dict(payload=payload, chunk_offset=off.reshape(shape), chunk_bytes=nby.reshape(shape), stats=stats,
+                sym=sym, q=q, mu=mu, max_chunks=mc)
+
+
+def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=False):
+    """Whole-path decode of the dict ``encode`` returned.  kv_shape = (L,2,S,H,n,d); returns float32 KV'."""
+    Tb = _h(T)
+    lg = _h(logits)
+    S, n, _ = lg.shape
+    pb = None if pos_begin is None else np.ascontiguousarray(pos_begin, dtype=np.int32)
+    pe = None if pos_end is None else np.ascontiguousarray(pos_end, dtype=np.int32)
+    out = np.zeros(kv_shape, np.float32)
+    st = _strides(out)
+    L, _, _, H, _, d = kv_shape
+    sym = np.zeros((S, n, L, 2, H, d), np.int32) if export else None
+    off = np.ascontiguousarray(enc["chunk_offset"]).reshape(-1)
+    nby = np.ascontiguousarray(enc["chunk_bytes"]).reshape(-1)
+    rc = lib().plo_decode(C.byref(cfg), _p(Tb), _p(lg), S, n, _p(pb), _p(pe), enc["max_chunks"], _p(enc["payload"]),
+                          _p(off), _p(nby), _p(out), C.byref(st), _p(sym))
+    return rc, out, sym
