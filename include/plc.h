@@ -1,0 +1,201 @@
+/*
+ * plc.h -- C ABI of libplc: predictive delta coding of a transformer KV cache on one B200.
+ *
+ * For every (session, layer, K-or-V, head, position) the library predicts the d-vector from the
+ * next-token distribution, subtracts the prediction, quantises the residual with a uniform step and
+ * entropy-codes it; the decoder inverts each step exactly at the quantised level.  A small second
+ * path finds shared session prefixes (longest common prefix and the trie metric).
+ *
+ * Conventions
+ *   - C linkage, no exceptions.  Every function returns a plc_status (0 = PLC_OK).
+ *   - Every pointer named *_dev is DEVICE memory owned by the caller and must stay valid until the
+ *     work enqueued on the given stream has completed.  Everything else is host memory.
+ *   - All work is enqueued on the caller's cudaStream_t (passed as void*; NULL = default stream).
+ *     Calls on one plc_ctx must be stream-ordered with respect to each other: the context's scratch
+ *     (top-K results, encoder staging) is shared between calls.
+ *   - The library allocates only inside plc_create / plc_reserve / plc_destroy (and inside
+ *     plc_encode / plc_decode / plc_append_step when the reserved scratch is too small).
+ *   - Problems found on the host (shapes, alignment) are returned at once and nothing is launched.
+ *     Problems found on the device (output capacity, damaged streams) are OR-ed into a device status
+ *     word that plc_sync_status reads; kernels never read or write outside the stated extents.
+ *   - Floating-point inputs are IEEE binary16 ("f16").  NaN logits are not supported.
+ *
+ * Notation: S sessions, n positions per session, L layers, H KV heads, d head dimension
+ * (32, 64, 128 or 256), V vocabulary, K candidates, W = 2*L*H streams per position.
+ * Table id t = (layer*2 + kv)*H + head, kv = 0 for keys and 1 for values.
+ */
+#ifndef PLC_H
+#define PLC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t plc_status;
+enum {
+    PLC_OK = 0,
+    PLC_E_INVALID = 1,   /* null pointer, non-positive size, value out of range */
+    PLC_E_SHAPE = 2,     /* unsupported d, K > V, K > 1024, chunk_pos < 1 ... */
+    PLC_E_ALIGN = 3,     /* a pointer or stride that must be 16-byte aligned is not */
+    PLC_E_CAPACITY = 4,  /* payload buffer too small; *total_bytes_dev holds the size needed */
+    PLC_E_CORRUPT = 5,   /* a chunk does not decode to its end state / runs past its bytes */
+    PLC_E_STATE = 6,     /* call not valid in the object's current state */
+    PLC_E_CUDA = 7       /* a CUDA runtime call failed (allocation, launch) */
+};
+
+enum { PLC_PRED_TOPK = 0, PLC_PRED_DENSE = 1 };
+enum { PLC_OUT_F32 = 0, PLC_OUT_F16 = 1 };
+
+/* Codec parameters.  delta: quantiser step (>= 2^-12).  sigma_floor: added in quadrature to the
+ * mixture's standard deviation before the scale class is taken (0 = none).  chunk_pos: positions
+ * per independently coded chunk.  variant: PLC_PRED_TOPK (Sec. 7.1 of the paper, top-k
+ * approximation) or PLC_PRED_DENSE (Def. 5, sum over the whole vocabulary as a bf16 contraction). */
+typedef struct {
+    int32_t n_layers, n_kv_heads, head_dim, vocab, top_k;
+    float delta, sigma_floor;
+    int32_t chunk_pos;
+    int32_t variant;
+    int32_t out_dtype;   /* dtype plc_decode writes: PLC_OUT_F32 or PLC_OUT_F16 */
+} plc_config;
+
+/* A KV tensor indexed [layer][kv][session][head][position][d]; strides in ELEMENTS, the d
+ * components of one vector are contiguous and every vector starts on a 16-byte boundary. */
+typedef struct {
+    void* base_dev;
+    int64_t stride_layer, stride_kv, stride_session, stride_head, stride_pos;
+} plc_kv_view;
+
+/* Coded output.  Chunk c of stream (session s, table t) has index slot
+ *     slot = (((s*L + layer)*2 + kv)*H + head) * max_chunks + c
+ * chunk_offset_dev[slot] = byte offset of the chunk in payload_dev (multiple of 16),
+ * chunk_bytes_dev[slot]  = its exact size (0 = no such chunk).  Chunks are placed in the order in
+ * which they are finished, so offsets differ from run to run; the bytes of each chunk do not.
+ * *total_bytes_dev = bytes of payload_dev in use (with padding); the caller zeroes it before the
+ * first plc_encode into a buffer and may keep it to append more chunks behind the ones present. */
+typedef struct {
+    uint8_t* payload_dev;
+    uint64_t payload_capacity;
+    uint64_t* chunk_offset_dev;
+    uint32_t* chunk_bytes_dev;
+    uint64_t* total_bytes_dev;
+    int32_t max_chunks;
+} plc_streams;
+
+/* Optional per-(session, position, table) exports of the coder's intermediate values, written by
+ * plc_encode / plc_decode when the pointers are non-NULL: sym [S][n][W][d] int32 (quantised
+ * residual), q [S][n][W] int32 (scale class), mu [S][n][W][d] float (prediction). */
+typedef struct {
+    int32_t* sym_dev;
+    int32_t* q_dev;
+    float* mu_dev;
+} plc_debug_buffers;
+
+typedef struct {
+    uint64_t payload_bytes;   /* sum of exact chunk sizes written since the counters were last reset */
+    uint64_t n_chunks;
+    uint64_t n_escapes;       /* components whose magnitude left the 63-symbol alphabet */
+    uint64_t coded_vectors;   /* (stream, position) pairs coded */
+} plc_stats;
+
+/* State of a batch of B sessions that grow by one position per plc_append_step (lock step).
+ * open_sym_dev [B][W][chunk_pos][d] int32 and open_q_dev [B][W][chunk_pos] int32 hold the positions
+ * of the chunk that is still open; steps counts the positions appended so far (host side).
+ * The index in `streams` is [B][W][max_chunks]; chunk c holds positions [c*chunk_pos, ...). */
+typedef struct {
+    int32_t B;
+    int32_t steps;
+    int32_t* open_sym_dev;
+    int32_t* open_q_dev;
+    plc_streams streams;
+} plc_session_batch;
+
+typedef struct plc_ctx plc_ctx;
+
+/* Creates a context for one parameter set and one candidate table.
+ * T_dev: [L][2][H][V][d] f16, the stand-in for F_M(t_<i, t) of Def. 5 (one d-vector per layer, K/V,
+ * head and candidate token); 16-byte aligned; must outlive the context (it is not copied).
+ * Synchronises the device once (it pre-computes the squared norm of every row of T).
+ * Errors: PLC_E_INVALID / PLC_E_SHAPE / PLC_E_ALIGN on bad arguments, PLC_E_CUDA. */
+plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev);
+plc_status plc_destroy(plc_ctx* ctx);
+
+/* Grows the context's scratch so that calls over up to max_positions = S*n positions allocate
+ * nothing (top-K results: 8*K bytes per position; encoder staging: fixed per device). */
+plc_status plc_reserve(plc_ctx* ctx, int64_t max_positions);
+
+/* Top-K softmax of N rows of logits (Sec. 5.1: P(t | t_<i) = softmax; Sec. 7.1: renormalised top-k;
+ * Thm. 4(a): Z_k).  logits_dev [N][V] f16.  tokens_dev [N] int32 or NULL.
+ * Outputs, each optional (NULL = skip): idx_dev [N][K] int32 ordered by (logit descending, index
+ * ascending); w_dev [N][K] float, exp(l_k - l_max) / sum over the K; lse_dev [N] natural
+ * log-sum-exp over V; zk_dev [N] sum of the K probabilities; logp2_dev [N] log2 P(tokens[i])
+ * (needs tokens_dev; the edge weight of the probabilistic language trie, Def. 1). */
+plc_status plc_topk_softmax(plc_ctx* ctx, const void* logits_dev, const int32_t* tokens_dev, int64_t N,
+                            int32_t* idx_dev, float* w_dev, float* lse_dev, float* zk_dev, float* logp2_dev,
+                            void* stream);
+
+/* Layer 1 (Def. 2; Sec. 7.3 best-match lookup = deepest stored ancestor).
+ * tokens_dev [S][token_stride] int32, lens_dev [S], logp2_dev [S][token_stride] float.
+ * lcp_dev [S][S] int32: length of the longest common prefix.  dT_dev [S][S] float:
+ * d_T(a,b) = -sum_{j<lcp(a,b)} logp2[a][j] (0 for an empty common prefix).  parent_dev [S]: the
+ * earlier session with the longest common prefix (ties: smallest index; none or length 0: -1).
+ * shared_len_dev [S]: that length -- the pos_begin of plc_encode (Prop. 2: the shared prefix costs
+ * zero bits, only the tail is coded).  All four outputs are written in full. */
+plc_status plc_prefix_dedup(plc_ctx* ctx, const int32_t* tokens_dev, const int32_t* lens_dev, const float* logp2_dev,
+                            int32_t S, int64_t token_stride, int32_t* lcp_dev, float* dT_dev, int32_t* parent_dev,
+                            int32_t* shared_len_dev, void* stream);
+
+/* Integration point 1 of Sec. 7.2: before KV_i is written, predict it, subtract (Def. 6), quantise
+ * and code the residual -- for every position in [pos_begin[s], pos_end[s]) of every session and
+ * every stream.  logits_dev [S][n][V] f16, logits[s][i] being the distribution over token i.
+ * pos_begin_dev / pos_end_dev [S] int32 or NULL (= 0 / n).  The index entries of all S*W*max_chunks
+ * slots are rewritten (0 bytes for chunks that do not exist); out->max_chunks >= ceil(n/chunk_pos).
+ * Chunk c of a session covers positions pos_begin + c*chunk_pos ... .
+ * Device-side error: PLC_E_CAPACITY (nothing is written past payload_capacity). */
+plc_status plc_encode(plc_ctx* ctx, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_streams* out,
+                      const plc_debug_buffers* dbg, void* stream);
+
+/* Integration point 2 of Sec. 7.2: recompute the prediction identically, decode the residual, add
+ * back (Prop. 3, "Correctness").  Writes cfg.out_dtype vectors into kv_out for the coded positions
+ * only.  Device-side error: PLC_E_CORRUPT (reads never leave a chunk's bytes; a damaged chunk
+ * yields garbage values for that chunk and sets the status). */
+plc_status plc_decode(plc_ctx* ctx, const plc_streams* in, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
+                      const plc_debug_buffers* dbg, void* stream);
+
+/* Decode-time append (integration point 1 for one new token per session).  kv_step_dev
+ * [L][2][B][H][d] f16, logits_step_dev [B][V] f16.  The new position's symbols and class go to the
+ * open chunk; when it holds chunk_pos positions it is coded into sb->streams (a LIFO coder cannot
+ * be extended in place, so a stream grows chunk by chunk).  sb->steps is advanced. */
+plc_status plc_append_step(plc_ctx* ctx, plc_session_batch* sb, const void* kv_step_dev, const void* logits_step_dev,
+                           void* stream);
+/* Codes the partly filled open chunk (if any) so that all sb->steps positions are decodable with
+ * plc_decode(S = B, n = steps).  No further plc_append_step is allowed afterwards. */
+plc_status plc_append_flush(plc_ctx* ctx, plc_session_batch* sb, void* stream);
+/* Bytes of open_sym_dev / open_q_dev for B sessions. */
+plc_status plc_append_sizes(const plc_ctx* ctx, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes);
+
+/* Waits for the stream and returns the device status word's most severe code; clears it. */
+plc_status plc_sync_status(plc_ctx* ctx, void* stream);
+/* Waits for the stream, copies the counters, optionally clears them. */
+plc_status plc_get_stats(plc_ctx* ctx, plc_stats* out, int32_t reset, void* stream);
+
+/* The two 32-bit constants (theta, rho) from which the frequency table of table id qp in [-24,15]
+ * is built with integer arithmetic, and the table itself (f[64], c[65]); host-side, no GPU work. */
+plc_status plc_table_constants(int32_t qp, uint32_t* theta, uint32_t* rho);
+plc_status plc_build_table(int32_t qp, uint32_t* f, uint32_t* c);
+/* With profiling on, plc_encode / plc_decode record CUDA events on the caller's stream directly
+ * around their fused predict+code kernel (the top-K kernel that precedes it is outside);
+ * plc_last_kernel_ms waits for the most recent such launch (which = 0 encode, 1 decode) and returns
+ * its duration.  PLC_E_STATE if no such launch was recorded. */
+plc_status plc_set_profiling(plc_ctx* ctx, int32_t on);
+plc_status plc_last_kernel_ms(plc_ctx* ctx, int32_t which, float* ms);
+/* Number of kernels this library has launched in this process (for benchmarks). */
+uint64_t plc_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PLC_H */

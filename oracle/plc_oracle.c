@@ -296,11 +296,19 @@ static int32_t join_sym(int32_t hi, uint32_t lo, int s) {
     if (s == 0) return hi;
     return (int32_t)(((int64_t)hi << s) + (int64_t)lo - ((int64_t)1 << (s - 1)));
 }
+static int comp_index(int l, int g, int d) {
+    int R = d / 8, G = d / NLANES;
+    return 8 * (l % R) + G * (l / R) + g;
+}
+static int valid_d(int d) { return d == 32 || d == 64 || d == 128 || d == 256; }
 static int zigzag(int32_t hi) { return hi > 0 ? 2 * hi - 1 : -2 * hi; }
 static int32_t unzigzag(int zz) { return (zz & 1) ? (zz + 1) / 2 : -(zz / 2); }
 
-/* A chunk is P consecutive positions of one stream (one d-vector per position); d = 32 G.
- * Lane l (0..31) owns components l*G + g, g = 0..G-1, and keeps one rANS state in [2^16, 2^32).
+/* A chunk is P consecutive positions of one stream (one d-vector per position); d = 32 G, d in
+ * {32, 64, 128, 256}.  The vector is cut into R = d/8 groups of 8 components (16 bytes of f16);
+ * lane l (0..31) owns, in group l mod R, the G components starting at G*(l div R):
+ *   component(l, g) = 8 (l mod R) + G (l div R) + g,  g = 0..G-1,
+ * and keeps one rANS state in [2^16, 2^32).
  * The chunk's bytes are: 32 little-endian uint32 decoder start states (lane 0..31), then a
  * sequence of little-endian 16-bit words in the order the decoder consumes them:
  *   for position p ascending, for g ascending:
@@ -321,7 +329,7 @@ static int32_t unzigzag(int zz) { return (zz & 1) ? (zz + 1) / 2 : -(zz / 2); }
 int plo_rans_encode_chunk(const int32_t* sym /*[P][d]*/, const int32_t* q /*[P]*/, int P, int d,
                           uint8_t* out, uint64_t cap, uint64_t* nbytes, double* ideal_bits,
                           uint64_t* n_escapes) {
-    if (d % NLANES || d <= 0 || P < 0) return PLO_E_INVALID;
+    if (!valid_d(d) || P < 0) return PLO_E_INVALID;
     int G = d / NLANES;
     size_t wcap = (size_t)P * d * 4 + 16;
     uint16_t* words = (uint16_t*)malloc(wcap * sizeof(uint16_t));
@@ -339,7 +347,7 @@ int plo_rans_encode_chunk(const int32_t* sym /*[P][d]*/, const int32_t* q /*[P]*
         if (qp != cur_qp) { plo_build_table(qp, f, c); cur_qp = qp; }
         for (int g = G - 1; g >= 0; --g) {
             int32_t hi[NLANES]; uint32_t lo[NLANES];
-            for (int l = 0; l < NLANES; ++l) split_sym(sym[(size_t)p * d + l * G + g], s, &hi[l], &lo[l]);
+            for (int l = 0; l < NLANES; ++l) split_sym(sym[(size_t)p * d + comp_index(l, g, d)], s, &hi[l], &lo[l]);
             /* (3) escapes, lanes descending, high half pushed first so that low half reads first */
             for (int l = NLANES - 1; l >= 0; --l) {
                 if (hi[l] > HI_MAX || hi[l] < -HI_MAX) {
@@ -387,7 +395,7 @@ int plo_rans_encode_chunk(const int32_t* sym /*[P][d]*/, const int32_t* q /*[P]*
 
 int plo_rans_decode_chunk(const uint8_t* in, uint64_t nbytes, const int32_t* q /*[P]*/, int P, int d,
                           int32_t* sym /*[P][d]*/) {
-    if (d % NLANES || d <= 0 || P < 0) return PLO_E_INVALID;
+    if (!valid_d(d) || P < 0) return PLO_E_INVALID;
     if (nbytes < 4 * NLANES || (nbytes & 1)) return PLO_E_CORRUPT;
     int G = d / NLANES;
     uint64_t nwords = (nbytes - 4 * NLANES) / 2, rp = 0;
@@ -427,7 +435,7 @@ int plo_rans_decode_chunk(const uint8_t* in, uint64_t nbytes, const int32_t* q /
                 int32_t hi;
                 if (zzs[l] == ESC) { uint32_t a, b2; NEXT_WORD(a); NEXT_WORD(b2); hi = (int32_t)(a | (b2 << 16)); }
                 else hi = unzigzag(zzs[l]);
-                sym[(size_t)p * d + l * G + g] = join_sym(hi, lo[l], s);
+                sym[(size_t)p * d + comp_index(l, g, d)] = join_sym(hi, lo[l], s);
             }
         }
     }
@@ -498,7 +506,7 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
                uint8_t* payload, uint64_t cap, uint64_t* chunk_offset, uint32_t* chunk_bytes,
                plo_stats* stats, int32_t* sym_out, int32_t* q_out, float* mu_out) {
     int L = cfg->L, H = cfg->H, d = cfg->d, V = cfg->V, K = cfg->K, CP = cfg->chunk_pos;
-    if (d % NLANES || CP < 1) return PLO_E_INVALID;
+    if (!valid_d(d) || CP < 1) return PLO_E_INVALID;
     memset(stats, 0, sizeof(*stats));
     int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)n * K);
     double* w = (double*)malloc(sizeof(double) * (size_t)n * K);
@@ -558,7 +566,7 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                const uint8_t* payload, const uint64_t* chunk_offset, const uint32_t* chunk_bytes,
                float* kv_out, const plo_kv_strides* st, int32_t* sym_out) {
     int L = cfg->L, H = cfg->H, d = cfg->d, V = cfg->V, K = cfg->K, CP = cfg->chunk_pos;
-    if (d % NLANES || CP < 1) return PLO_E_INVALID;
+    if (!valid_d(d) || CP < 1) return PLO_E_INVALID;
     int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)n * K);
     double* w = (double*)malloc(sizeof(double) * (size_t)n * K);
     double* lse = (double*)malloc(sizeof(double) * (size_t)n);

@@ -1,1 +1,269 @@
-"""Predictive delta coding of the KV cache for B200 (sm_100a): Python binding of libplc.so."""
+"""Predictive delta coding of the KV cache for B200 (sm_100a): thin Python binding of libplc.so.
+
+The binding only marshals arguments (torch device tensors -> raw pointers, the current torch stream
+-> cudaStream_t).  Every step of the path runs in the library's CUDA kernels; there is no CPU or
+PyTorch fallback: if the shared library is missing, ``lib()`` raises.
+"""
+import ctypes as C
+import os
+import subprocess
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_CSRC = os.path.join(_HERE, "csrc")
+_INC = os.path.join(os.path.dirname(_HERE), "include")
+_SO = os.path.join(_HERE, "libplc.so")
+_SOURCES = ["plc_api.cu", "plc_topk.cu", "plc_prefix.cu", "plc_codec.cu", "plc_dense.cu", "plc_static.cu"]
+
+OK, E_INVALID, E_SHAPE, E_ALIGN, E_CAPACITY, E_CORRUPT, E_STATE, E_CUDA = range(8)
+PRED_TOPK, PRED_DENSE = 0, 1
+OUT_F32, OUT_F16 = 0, 1
+
+EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_prefix_dedup", "plc_encode",
+           "plc_decode", "plc_append_step", "plc_append_flush", "plc_append_sizes", "plc_sync_status",
+           "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
+           "plc_launch_count"]
+
+
+def sources():
+    return [os.path.join(_CSRC, s) for s in _SOURCES if os.path.exists(os.path.join(_CSRC, s))]
+
+
+def build(force=False, verbose=False):
+    """Compile libplc.so for sm_100a with nvcc (in-tree)."""
+    srcs = sources()
+    deps = srcs + [os.path.join(_CSRC, "plc_common.cuh"), os.path.join(_INC, "plc.h")]
+    if not force and os.path.exists(_SO) and all(os.path.getmtime(_SO) >= os.path.getmtime(d) for d in deps):
+        return _SO
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-shared", "-I" + _INC, "-o", _SO] + srcs
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.check_call(cmd)
+    return _SO
+
+
+class Config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("vocab", C.c_int32),
+                ("top_k", C.c_int32), ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32),
+                ("variant", C.c_int32), ("out_dtype", C.c_int32)]
+
+
+class KVView(C.Structure):
+    _fields_ = [("base_dev", C.c_void_p), ("stride_layer", C.c_int64), ("stride_kv", C.c_int64),
+                ("stride_session", C.c_int64), ("stride_head", C.c_int64), ("stride_pos", C.c_int64)]
+
+
+class Streams(C.Structure):
+    _fields_ = [("payload_dev", C.c_void_p), ("payload_capacity", C.c_uint64), ("chunk_offset_dev", C.c_void_p),
+                ("chunk_bytes_dev", C.c_void_p), ("total_bytes_dev", C.c_void_p), ("max_chunks", C.c_int32)]
+
+
+class DebugBuffers(C.Structure):
+    _fields_ = [("sym_dev", C.c_void_p), ("q_dev", C.c_void_p), ("mu_dev", C.c_void_p)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("payload_bytes", C.c_uint64), ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64),
+                ("coded_vectors", C.c_uint64)]
+
+
+class SessionBatch(C.Structure):
+    _fields_ = [("B", C.c_int32), ("steps", C.c_int32), ("open_sym_dev", C.c_void_p), ("open_q_dev", C.c_void_p),
+                ("streams", Streams)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libplc.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise RuntimeError(f"{_SO} not found: run paper_2604_15356_b200.build() (nvcc, sm_100a) first")
+        _lib = C.CDLL(_SO)
+        _lib.plc_launch_count.restype = C.c_uint64
+    return _lib
+
+
+class PlcError(RuntimeError):
+    def __init__(self, code, where):
+        super().__init__(f"{where}: plc_status {code}")
+        self.code = code
+
+
+def _check(rc, where):
+    if rc != OK:
+        raise PlcError(rc, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def kv_view(kv):
+    """torch tensor indexed [L][2][S][H][n][d] (any strides with d contiguous) -> KVView."""
+    assert kv.dim() == 6 and kv.stride(5) == 1
+    s = kv.stride()
+    return KVView(kv.data_ptr(), s[0], s[1], s[2], s[3], s[4])
+
+
+class StreamSet:
+    """Device buffers of a coded output: payload, per-chunk index, byte cursor."""
+
+    def __init__(self, n_streams, max_chunks, capacity, device="cuda"):
+        import torch
+        self.payload = torch.empty(int(capacity), dtype=torch.uint8, device=device)
+        self.chunk_offset = torch.zeros(n_streams * max_chunks, dtype=torch.int64, device=device)
+        self.chunk_bytes = torch.zeros(n_streams * max_chunks, dtype=torch.int32, device=device)
+        self.total_bytes = torch.zeros(1, dtype=torch.int64, device=device)
+        self.max_chunks = max_chunks
+        self.n_streams = n_streams
+
+    def c(self):
+        return Streams(self.payload.data_ptr(), self.payload.numel(), self.chunk_offset.data_ptr(),
+                       self.chunk_bytes.data_ptr(), self.total_bytes.data_ptr(), self.max_chunks)
+
+    def chunk(self, slot):
+        """Bytes of one chunk as a CPU numpy array."""
+        off = int(self.chunk_offset[slot]); nb = int(self.chunk_bytes[slot]) & 0xFFFFFFFF
+        return self.payload[off:off + nb].cpu().numpy()
+
+
+class Context:
+    """One parameter set + candidate table T ([L][2][H][V][d] float16 on the device)."""
+
+    def __init__(self, T, top_k, delta, chunk_pos=256, sigma_floor=0.0, variant=PRED_TOPK, out_dtype=OUT_F32):
+        L, two, H, V, d = T.shape
+        assert two == 2 and T.is_cuda and T.is_contiguous()
+        self.T = T
+        self.cfg = Config(L, H, d, V, top_k, delta, sigma_floor, chunk_pos, variant, out_dtype)
+        self.W = 2 * L * H
+        self._h = C.c_void_p()
+        _check(lib().plc_create(C.byref(self._h), C.byref(self.cfg), _ptr(T)), "plc_create")
+
+    def close(self):
+        if self._h:
+            lib().plc_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def max_chunks(self, n):
+        return (n + self.cfg.chunk_pos - 1) // self.cfg.chunk_pos
+
+    def reserve(self, positions):
+        _check(lib().plc_reserve(self._h, C.c_int64(positions)), "plc_reserve")
+
+    def topk_softmax(self, logits, tokens=None, want=("idx", "w", "lse", "zk", "logp2")):
+        import torch
+        N = logits.numel() // self.cfg.vocab
+        K = self.cfg.top_k
+        dev = logits.device
+        out = {}
+        if "idx" in want:
+            out["idx"] = torch.empty(N, K, dtype=torch.int32, device=dev)
+        if "w" in want:
+            out["w"] = torch.empty(N, K, dtype=torch.float32, device=dev)
+        for k in ("lse", "zk"):
+            if k in want:
+                out[k] = torch.empty(N, dtype=torch.float32, device=dev)
+        if "logp2" in want and tokens is not None:
+            out["logp2"] = torch.empty(N, dtype=torch.float32, device=dev)
+        _check(lib().plc_topk_softmax(self._h, _ptr(logits), _ptr(tokens), C.c_int64(N), _ptr(out.get("idx")),
+                                      _ptr(out.get("w")), _ptr(out.get("lse")), _ptr(out.get("zk")),
+                                      _ptr(out.get("logp2")), _stream()), "plc_topk_softmax")
+        return out
+
+    def prefix_dedup(self, tokens, lens, logp2):
+        import torch
+        S, stride = tokens.shape
+        dev = tokens.device
+        lcp = torch.empty(S, S, dtype=torch.int32, device=dev)
+        dT = torch.empty(S, S, dtype=torch.float32, device=dev)
+        parent = torch.empty(S, dtype=torch.int32, device=dev)
+        shared = torch.empty(S, dtype=torch.int32, device=dev)
+        _check(lib().plc_prefix_dedup(self._h, _ptr(tokens), _ptr(lens), _ptr(logp2), S, C.c_int64(stride), _ptr(lcp),
+                                      _ptr(dT), _ptr(parent), _ptr(shared), _stream()), "plc_prefix_dedup")
+        return lcp, dT, parent, shared
+
+    def encode(self, kv, logits, streams, pos_begin=None, pos_end=None, debug=None):
+        S, n = logits.shape[0], logits.shape[1]
+        view = kv if isinstance(kv, KVView) else kv_view(kv)
+        st = streams.c()
+        _check(lib().plc_encode(self._h, C.byref(view), _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end),
+                                C.byref(st), None if debug is None else C.byref(debug), _stream()), "plc_encode")
+
+    def decode(self, streams, logits, kv_out, pos_begin=None, pos_end=None, debug=None):
+        S, n = logits.shape[0], logits.shape[1]
+        view = kv_out if isinstance(kv_out, KVView) else kv_view(kv_out)
+        st = streams.c()
+        _check(lib().plc_decode(self._h, C.byref(st), _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end),
+                                C.byref(view), None if debug is None else C.byref(debug), _stream()), "plc_decode")
+
+    def sync_status(self):
+        return lib().plc_sync_status(self._h, _stream())
+
+    def set_profiling(self, on=True):
+        _check(lib().plc_set_profiling(self._h, int(on)), "plc_set_profiling")
+
+    def last_kernel_ms(self, which):
+        """Duration of the most recent fused kernel: which = 0 encode, 1 decode."""
+        ms = C.c_float()
+        _check(lib().plc_last_kernel_ms(self._h, int(which), C.byref(ms)), "plc_last_kernel_ms")
+        return ms.value
+
+    def stats(self, reset=False):
+        s = Stats()
+        _check(lib().plc_get_stats(self._h, C.byref(s), int(reset), _stream()), "plc_get_stats")
+        return s
+
+    def new_session_batch(self, B, max_chunks, capacity):
+        import torch
+        a, b = C.c_uint64(), C.c_uint64()
+        _check(lib().plc_append_sizes(self._h, B, C.byref(a), C.byref(b)), "plc_append_sizes")
+        sb = AppendBatch()
+        sb.open_sym = torch.zeros(a.value // 4, dtype=torch.int32, device=self.T.device)
+        sb.open_q = torch.zeros(b.value // 4, dtype=torch.int32, device=self.T.device)
+        sb.streams = StreamSet(B * self.W, max_chunks, capacity, self.T.device)
+        sb.c = SessionBatch(B, 0, sb.open_sym.data_ptr(), sb.open_q.data_ptr(), sb.streams.c())
+        return sb
+
+    def append_step(self, sb, kv_step, logits_step):
+        _check(lib().plc_append_step(self._h, C.byref(sb.c), _ptr(kv_step), _ptr(logits_step), _stream()),
+               "plc_append_step")
+
+    def append_flush(self, sb):
+        _check(lib().plc_append_flush(self._h, C.byref(sb.c), _stream()), "plc_append_flush")
+
+
+class AppendBatch:
+    """Python-side holder of a plc_session_batch and the tensors it points to."""
+
+
+def table_constants(qp):
+    th, rh = C.c_uint32(), C.c_uint32()
+    _check(lib().plc_table_constants(int(qp), C.byref(th), C.byref(rh)), "plc_table_constants")
+    return th.value, rh.value
+
+
+def build_table(qp):
+    import numpy as np
+    f = np.zeros(64, np.uint32)
+    c = np.zeros(65, np.uint32)
+    _check(lib().plc_build_table(int(qp), f.ctypes.data_as(C.c_void_p), c.ctypes.data_as(C.c_void_p)),
+           "plc_build_table")
+    return f, c
+
+
+def launch_count():
+    return int(lib().plc_launch_count())

@@ -1,0 +1,322 @@
+// C ABI of libplc (see include/plc.h): argument checks, context scratch, kernel launches.
+#include <atomic>
+#include <new>
+
+#include "plc_common.cuh"
+
+namespace plc {
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+}  // namespace plc
+
+using namespace plc;
+
+struct plc_ctx {
+    plc_config cfg;
+    const __half* T;
+    float* rownorm2;
+    int2* pairs;
+    long long pairs_cap;            // positions
+    uint16_t* staging;
+    unsigned long long staging_words_per_warp;
+    unsigned int* ticket;
+    unsigned int* status;
+    Counters* counters;
+    int profiling;                  // record events around the codec kernels
+    cudaEvent_t ev[4];              // encode start/stop, decode start/stop
+    int ev_valid[2];
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+bool valid_d(int d) { return d == 32 || d == 64 || d == 128 || d == 256; }
+
+plc_status check_view(const plc_kv_view* v, int d, int elem_bytes) {
+    if (!v || !v->base_dev) return PLC_E_INVALID;
+    if (!aligned16(v->base_dev)) return PLC_E_ALIGN;
+    const int64_t per16 = 16 / elem_bytes;
+    const int64_t st[5] = {v->stride_layer, v->stride_kv, v->stride_session, v->stride_head, v->stride_pos};
+    for (int i = 0; i < 5; ++i)
+        if (st[i] % per16) return PLC_E_ALIGN;
+    (void)d;
+    return PLC_OK;
+}
+
+plc_status check_streams(const plc_streams* s, int need_chunks) {
+    if (!s || !s->payload_dev || !s->chunk_offset_dev || !s->chunk_bytes_dev || !s->total_bytes_dev) return PLC_E_INVALID;
+    if (!aligned16(s->payload_dev)) return PLC_E_ALIGN;
+    if (s->max_chunks < need_chunks || s->max_chunks < 1) return PLC_E_SHAPE;
+    return PLC_OK;
+}
+
+plc_status ensure_pairs(plc_ctx* c, long long positions) {
+    if (positions <= c->pairs_cap) return PLC_OK;
+    if (c->pairs) cudaFree(c->pairs);
+    c->pairs = nullptr; c->pairs_cap = 0;
+    if (cudaMalloc(&c->pairs, sizeof(int2) * (size_t)positions * c->cfg.top_k) != cudaSuccess) return PLC_E_CUDA;
+    c->pairs_cap = positions;
+    return PLC_OK;
+}
+
+CodecArgs base_args(const plc_ctx* c) {
+    CodecArgs a{};
+    a.sh.L = c->cfg.n_layers; a.sh.H = c->cfg.n_kv_heads; a.sh.d = c->cfg.head_dim; a.sh.V = c->cfg.vocab;
+    a.sh.K = c->cfg.top_k; a.sh.chunk_pos = c->cfg.chunk_pos; a.sh.out_dtype = c->cfg.out_dtype;
+    a.sh.delta = c->cfg.delta; a.sh.sigma_floor = c->cfg.sigma_floor;
+    a.T = c->T; a.rownorm2 = c->rownorm2; a.pairs = c->pairs;
+    a.staging = c->staging; a.staging_words_per_warp = c->staging_words_per_warp;
+    a.ticket = c->ticket; a.status = c->status; a.counters = c->counters;
+    return a;
+}
+
+StreamsDev to_dev(const plc_streams* s) {
+    StreamsDev d;
+    d.payload = s->payload_dev; d.capacity = s->payload_capacity;
+    d.chunk_offset = reinterpret_cast<unsigned long long*>(s->chunk_offset_dev);
+    d.chunk_bytes = s->chunk_bytes_dev;
+    d.total_bytes = reinterpret_cast<unsigned long long*>(s->total_bytes_dev);
+    d.max_chunks = s->max_chunks;
+    return d;
+}
+
+KvView to_dev(const plc_kv_view* v) {
+    return KvView{v->base_dev, v->stride_layer, v->stride_kv, v->stride_session, v->stride_head, v->stride_pos};
+}
+
+}  // namespace
+
+extern "C" {
+
+plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
+    if (!out || !cfg || !T_dev) return PLC_E_INVALID;
+    *out = nullptr;
+    if (cfg->n_layers < 1 || cfg->n_kv_heads < 1 || cfg->vocab < 1) return PLC_E_INVALID;
+    if (!valid_d(cfg->head_dim) || cfg->top_k < 1 || cfg->top_k > cfg->vocab || cfg->top_k > 1024) return PLC_E_SHAPE;
+    if (cfg->chunk_pos < 1 || cfg->chunk_pos > 4096) return PLC_E_SHAPE;
+    if (!(cfg->delta >= 1.0f / 4096.0f) || !(cfg->delta < 65536.0f) || !(cfg->sigma_floor >= 0.0f)) return PLC_E_INVALID;
+    if (cfg->variant != PLC_PRED_TOPK && cfg->variant != PLC_PRED_DENSE) return PLC_E_INVALID;
+    if (cfg->out_dtype != PLC_OUT_F32 && cfg->out_dtype != PLC_OUT_F16) return PLC_E_INVALID;
+    if (!aligned16(T_dev)) return PLC_E_ALIGN;
+    plc_ctx* c = new (std::nothrow) plc_ctx();
+    if (!c) return PLC_E_CUDA;
+    c->cfg = *cfg;
+    c->T = static_cast<const __half*>(T_dev);
+    const long long rows = (long long)cfg->n_layers * 2 * cfg->n_kv_heads * cfg->vocab;
+    c->staging_words_per_warp = 4ull * cfg->chunk_pos * cfg->head_dim + 64;
+    const int warps = codec_grid_warps(0);
+    bool ok = cudaMalloc(&c->rownorm2, sizeof(float) * (size_t)rows) == cudaSuccess &&
+              cudaMalloc(&c->staging, sizeof(uint16_t) * c->staging_words_per_warp * warps) == cudaSuccess &&
+              cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->status, sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->counters, sizeof(Counters)) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->status, 0, sizeof(unsigned int)) == cudaSuccess &&
+                 cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
+    if (ok) ok = launch_rownorm(c->T, c->rownorm2, rows, cfg->head_dim, 0) == cudaSuccess &&
+                 cudaDeviceSynchronize() == cudaSuccess;
+    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    if (!ok) { plc_destroy(c); return PLC_E_CUDA; }
+    *out = c;
+    return PLC_OK;
+}
+
+plc_status plc_destroy(plc_ctx* c) {
+    if (!c) return PLC_E_INVALID;
+    cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->staging);
+    cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters);
+    for (int i = 0; i < 4; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    delete c;
+    return PLC_OK;
+}
+
+plc_status plc_reserve(plc_ctx* c, int64_t max_positions) {
+    if (!c || max_positions < 0) return PLC_E_INVALID;
+    return ensure_pairs(c, max_positions);
+}
+
+plc_status plc_topk_softmax(plc_ctx* c, const void* logits_dev, const int32_t* tokens_dev, int64_t N, int32_t* idx_dev,
+                            float* w_dev, float* lse_dev, float* zk_dev, float* logp2_dev, void* stream) {
+    if (!c || !logits_dev || N < 0) return PLC_E_INVALID;
+    if (logp2_dev && !tokens_dev) return PLC_E_INVALID;
+    TopkArgs a{};
+    a.logits = static_cast<const __half*>(logits_dev); a.tokens = tokens_dev; a.N = N;
+    a.V = c->cfg.vocab; a.K = c->cfg.top_k;
+    a.idx = idx_dev; a.w = w_dev; a.lse = lse_dev; a.zk = zk_dev; a.logp2 = logp2_dev;
+    a.n_per_session = 1;
+    return launch_topk(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_prefix_dedup(plc_ctx* c, const int32_t* tokens_dev, const int32_t* lens_dev, const float* logp2_dev,
+                            int32_t S, int64_t token_stride, int32_t* lcp_dev, float* dT_dev, int32_t* parent_dev,
+                            int32_t* shared_len_dev, void* stream) {
+    if (!c || !tokens_dev || !lens_dev || !logp2_dev || !lcp_dev || !dT_dev || !parent_dev || !shared_len_dev)
+        return PLC_E_INVALID;
+    if (S < 0 || token_stride < 0) return PLC_E_INVALID;
+    return launch_prefix_dedup(tokens_dev, lens_dev, logp2_dev, S, token_stride, lcp_dev, dT_dev, parent_dev,
+                               shared_len_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n, const int32_t* pb, const int32_t* pe,
+                               cudaStream_t st) {
+    plc_status rc = ensure_pairs(c, (long long)S * n);
+    if (rc) return rc;
+    TopkArgs a{};
+    a.logits = static_cast<const __half*>(logits_dev); a.N = (long long)S * n; a.V = c->cfg.vocab; a.K = c->cfg.top_k;
+    a.pairs = c->pairs; a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
+    return launch_topk(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_streams* out,
+                      const plc_debug_buffers* dbg, void* stream) {
+    if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
+    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
+    plc_status rc = check_view(kv, c->cfg.head_dim, 2);
+    if (rc) return rc;
+    const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
+    rc = check_streams(out, need);
+    if (rc) return rc;
+    if (S == 0 || n == 0) return PLC_OK;
+    const long long items = (long long)2 * c->cfg.n_layers * c->cfg.n_kv_heads * S * out->max_chunks;
+    if (items >= (1ll << 32)) return PLC_E_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    if (rc) return rc;
+    CodecArgs a = base_args(c);
+    a.kv = to_dev(kv); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
+    a.st = to_dev(out);
+    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (c->profiling) cudaEventRecord(c->ev[0], st);
+    cudaError_t e = launch_encode(a, st);
+    if (c->profiling) { cudaEventRecord(c->ev[1], st); c->ev_valid[0] = 1; }
+    return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
+                      const plc_debug_buffers* dbg, void* stream) {
+    if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
+    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
+    plc_status rc = check_view(kv_out, c->cfg.head_dim, c->cfg.out_dtype == PLC_OUT_F16 ? 2 : 4);
+    if (rc) return rc;
+    const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
+    rc = check_streams(in, need);
+    if (rc) return rc;
+    if (S == 0 || n == 0) return PLC_OK;
+    const long long items = (long long)2 * c->cfg.n_layers * c->cfg.n_kv_heads * S * in->max_chunks;
+    if (items >= (1ll << 32)) return PLC_E_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    if (rc) return rc;
+    CodecArgs a = base_args(c);
+    a.kv = to_dev(kv_out); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
+    a.st = to_dev(in);
+    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (c->profiling) cudaEventRecord(c->ev[2], st);
+    cudaError_t e = launch_decode(a, st);
+    if (c->profiling) { cudaEventRecord(c->ev[3], st); c->ev_valid[1] = 1; }
+    return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_append_sizes(const plc_ctx* c, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes) {
+    if (!c || B < 0 || !open_sym_bytes || !open_q_bytes) return PLC_E_INVALID;
+    const uint64_t W = 2ull * c->cfg.n_layers * c->cfg.n_kv_heads;
+    *open_q_bytes = 4ull * B * W * c->cfg.chunk_pos;
+    *open_sym_bytes = *open_q_bytes * c->cfg.head_dim;
+    return PLC_OK;
+}
+
+static plc_status seal(plc_ctx* c, plc_session_batch* sb, int chunk_index, int count, cudaStream_t st) {
+    CodecArgs a = base_args(c);
+    a.S = sb->B; a.n = 0;
+    a.st = to_dev(&sb->streams);
+    a.open_sym = sb->open_sym_dev; a.open_q = sb->open_q_dev; a.open_count = count; a.chunk_index = chunk_index;
+    return launch_append_seal(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_append_step(plc_ctx* c, plc_session_batch* sb, const void* kv_step_dev, const void* logits_step_dev,
+                           void* stream) {
+    if (!c || !sb || !kv_step_dev || !logits_step_dev || !sb->open_sym_dev || !sb->open_q_dev) return PLC_E_INVALID;
+    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
+    if (sb->B < 1 || sb->steps < 0) return PLC_E_INVALID;
+    if (!aligned16(kv_step_dev)) return PLC_E_ALIGN;
+    const int CP = c->cfg.chunk_pos;
+    plc_status rc = check_streams(&sb->streams, sb->steps / CP + 1);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = run_topk_for(c, logits_step_dev, sb->B, 1, nullptr, nullptr, st);
+    if (rc) return rc;
+    CodecArgs a = base_args(c);
+    const int64_t d = c->cfg.head_dim, H = c->cfg.n_kv_heads, B = sb->B;
+    a.kv = KvView{const_cast<void*>(kv_step_dev), 2 * B * H * d, B * H * d, H * d, d, 0};
+    a.S = sb->B; a.n = 1;
+    a.open_sym = sb->open_sym_dev; a.open_q = sb->open_q_dev; a.open_slot = sb->steps % CP;
+    if (launch_append_quantise(a, st) != cudaSuccess) return PLC_E_CUDA;
+    sb->steps += 1;
+    if (sb->steps % CP == 0) return seal(c, sb, sb->steps / CP - 1, CP, st);
+    return PLC_OK;
+}
+
+plc_status plc_append_flush(plc_ctx* c, plc_session_batch* sb, void* stream) {
+    if (!c || !sb || !sb->open_sym_dev || !sb->open_q_dev || sb->B < 1 || sb->steps < 0) return PLC_E_INVALID;
+    const int CP = c->cfg.chunk_pos, rem = sb->steps % CP;
+    if (rem == 0) return PLC_OK;
+    plc_status rc = check_streams(&sb->streams, sb->steps / CP + 1);
+    if (rc) return rc;
+    return seal(c, sb, sb->steps / CP, rem, static_cast<cudaStream_t>(stream));
+}
+
+plc_status plc_sync_status(plc_ctx* c, void* stream) {
+    if (!c) return PLC_E_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int w = 0;
+    if (cudaMemcpyAsync(&w, c->status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaMemsetAsync(c->status, 0, sizeof(w), st) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
+    if (w & kStCorrupt) return PLC_E_CORRUPT;
+    if (w & kStCapacity) return PLC_E_CAPACITY;
+    return PLC_OK;
+}
+
+plc_status plc_get_stats(plc_ctx* c, plc_stats* out, int32_t reset, void* stream) {
+    if (!c || !out) return PLC_E_INVALID;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Counters h{};
+    if (cudaMemcpyAsync(&h, c->counters, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PLC_E_CUDA;
+    if (reset && cudaMemsetAsync(c->counters, 0, sizeof(h), st) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
+    out->payload_bytes = h.payload_bytes; out->n_chunks = h.n_chunks; out->n_escapes = h.n_escapes;
+    out->coded_vectors = h.coded_vectors;
+    return PLC_OK;
+}
+
+plc_status plc_table_constants(int32_t qp, uint32_t* theta, uint32_t* rho) {
+    if (qp < kQMin || qp > 15 || !theta || !rho) return PLC_E_INVALID;
+    table_constants(qp, *theta, *rho);
+    return PLC_OK;
+}
+
+plc_status plc_build_table(int32_t qp, uint32_t* f, uint32_t* cdf) {
+    if (qp < kQMin || qp > 15 || !f || !cdf) return PLC_E_INVALID;
+    build_freqs(qp, f);
+    cdf[0] = 0;
+    for (int i = 0; i < kNumSym; ++i) cdf[i + 1] = cdf[i] + f[i];
+    return PLC_OK;
+}
+
+plc_status plc_set_profiling(plc_ctx* c, int32_t on) {
+    if (!c) return PLC_E_INVALID;
+    c->profiling = on != 0;
+    return PLC_OK;
+}
+
+plc_status plc_last_kernel_ms(plc_ctx* c, int32_t which, float* ms) {
+    if (!c || !ms || which < 0 || which > 1) return PLC_E_INVALID;
+    if (!c->ev_valid[which]) return PLC_E_STATE;
+    if (cudaEventSynchronize(c->ev[2 * which + 1]) != cudaSuccess) return PLC_E_CUDA;
+    return cudaEventElapsedTime(ms, c->ev[2 * which], c->ev[2 * which + 1]) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+uint64_t plc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

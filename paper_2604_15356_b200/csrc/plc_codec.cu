@@ -1,0 +1,606 @@
+// Fused predict / quantise / rANS kernels.
+//
+// One warp owns one (stream, chunk): it walks the chunk's positions (backwards when encoding,
+// forwards when decoding), and for each position
+//   1. gathers the K candidate rows of its table with 128-bit loads and accumulates the mixture
+//      mu = sum_k w_k T[idx_k] in binary32 (each lane: 8 components of every ROWS-th row, then a
+//      shuffle reduce-scatter so that lane l ends with its G = d/32 components),
+//   2. derives the scale class from the mixture variance (precomputed row norms),
+//   3. quantises the residual (encoder) or adds the decoded residual back (decoder),
+//   4. runs one interleaved rANS step per owned component, the 32 lanes sharing one word stream.
+// The encoder writes its words back to front into a per-warp staging area (global memory, reused
+// from chunk to chunk so it stays in L2), then reserves the chunk's final place with one atomicAdd
+// and copies it there.  Work items are handed out by an atomic ticket in table-major order so that
+// the warps running at any time gather from few tables.
+#include <type_traits>
+
+#include "plc_common.cuh"
+
+namespace plc {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kThreads = kWarpsPerBlock * 32;
+constexpr int kBlocksPerSM = 4;
+
+template <int D>
+struct Geo {
+    static constexpr int R = D / 8;        // lanes that cover one row with 16-byte loads
+    static constexpr int G = D / 32;       // components a lane owns
+    static constexpr int ROWS = 32 / R;    // rows fetched by one warp-wide load
+};
+
+struct EncTables { EncEntry enc[kNumTables][kNumSym]; };
+struct DecTables { uint16_t cum[kNumTables][kNumSym + 2]; };
+
+__device__ inline void build_enc_tables(EncTables* t) {
+    for (int id = threadIdx.x; id < kNumTables; id += blockDim.x) {
+        uint32_t f[kNumSym];
+        build_freqs(id + kQMin, f);
+        uint32_t c = 0;
+        for (int i = 0; i < kNumSym; ++i) {
+            uint32_t fi = f[i];
+            t->enc[id][i].rcp = fi == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / fi);
+            t->enc[id][i].fc = fi | (c << 16);
+            c += fi;
+        }
+    }
+}
+__device__ inline void build_dec_tables(DecTables* t) {
+    for (int id = threadIdx.x; id < kNumTables; id += blockDim.x) {
+        uint32_t f[kNumSym];
+        build_freqs(id + kQMin, f);
+        uint32_t c = 0;
+        for (int i = 0; i < kNumSym; ++i) { t->cum[id][i] = (uint16_t)c; c += f[i]; }
+        t->cum[id][kNumSym] = (uint16_t)c;
+        t->cum[id][kNumSym + 1] = 0xffff;
+    }
+}
+
+// component owned by (lane, g): 8 (lane mod R) + G (lane div R) + g
+template <int D>
+__device__ __forceinline__ int first_comp(int lane) {
+    return 8 * (lane % Geo<D>::R) + Geo<D>::G * (lane / Geo<D>::R);
+}
+
+// Sum of squares of the lane's G values, then over the warp; the same chain is used for the row
+// norms and for ||mu||^2 so that a point-mass mixture has exactly zero variance.
+template <int G>
+__device__ __forceinline__ float warp_norm2(const float (&v)[G]) {
+    float p = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) p = __fmaf_rn(v[g], v[g], p);
+    return warp_sum(p);
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) rownorm_kernel(const __half* __restrict__ T, float* __restrict__ out, long long rows) {
+    constexpr int G = Geo<D>::G;
+    const int lane = threadIdx.x & 31;
+    const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
+    const int c0 = first_comp<D>(lane);
+    for (long long r = warp; r < rows; r += nw) {
+        float v[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) v[g] = __half2float(T[r * D + c0 + g]);
+        float s = warp_norm2<G>(v);
+        if (lane == 0) out[r] = s;
+    }
+}
+
+// Mixture of one position for one table.  pairs: the position's K {idx, w} entries.
+template <int D>
+__device__ __forceinline__ void predict(const __half* __restrict__ table, const float* __restrict__ n2,
+                                        const int2* __restrict__ pairs, int K, int lane, float inv_d,
+                                        float (&mu)[Geo<D>::G], float& sigma2) {
+    constexpr int R = Geo<D>::R, G = Geo<D>::G, ROWS = Geo<D>::ROWS;
+    const int m = lane % R, h = lane / R;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    const __half* col = table + 8 * m;
+#pragma unroll 4
+    for (int k0 = 0; k0 < K; k0 += ROWS) {
+        int k = k0 + h;
+        bool ok = k < K;
+        int2 pr = __ldg(pairs + (ok ? k : 0));
+        float w = ok ? __int_as_float(pr.y) : 0.f;
+        uint4 r = __ldg(reinterpret_cast<const uint4*>(col + (size_t)pr.x * D));
+        const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float2 f = __half22float2(hp[j]);
+            acc[2 * j] = __fmaf_rn(w, f.x, acc[2 * j]);
+            acc[2 * j + 1] = __fmaf_rn(w, f.y, acc[2 * j + 1]);
+        }
+    }
+    // reduce-scatter over the ROWS lanes that hold partial sums of the same 8 components
+    int cnt = 8;
+#pragma unroll
+    for (int o = (ROWS / 2) * R; o >= R; o >>= 1) {
+        const bool up = (h & (o / R)) != 0;
+        const int half = cnt / 2;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < half) {
+                float send = up ? acc[i] : acc[i + half];
+                float keep = up ? acc[i + half] : acc[i];
+                acc[i] = keep + __shfl_xor_sync(kFull, send, o);
+            }
+        }
+        cnt = half;
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) mu[g] = acc[g];
+    // variance: (sum_k w_k ||T_k||^2 - ||mu||^2) / d
+    float s1 = 0.f;
+    for (int k = lane; k < K; k += 32) {
+        int2 pr = __ldg(pairs + k);
+        s1 = __fmaf_rn(__int_as_float(pr.y), __ldg(n2 + pr.x), s1);
+    }
+    s1 = warp_sum(s1);
+    float s2 = warp_norm2<G>(mu);
+    sigma2 = fmaxf(0.f, (s1 - s2) * inv_d);
+}
+
+__device__ __forceinline__ int scale_class(float sigma2, float floor2, float delta2) {
+    return class_from_v(__fdiv_rn(sigma2 + floor2, delta2));
+}
+
+__device__ __forceinline__ void split_sym(int sym, int s, int& hi, uint32_t& lo) {
+    if (s == 0) { hi = sym; lo = 0; return; }
+    int u = sym + (1 << (s - 1));          // |sym| <= 2^30, s <= 15: no overflow
+    hi = u >> s;
+    lo = (uint32_t)u & ((1u << s) - 1u);
+}
+__device__ __forceinline__ int join_sym(int hi, uint32_t lo, int s) {
+    if (s == 0) return hi;
+    return (int)(((uint32_t)hi << s) + lo - (1u << (s - 1)));
+}
+
+// One encoder step for the warp: every lane codes `sym` under (s, table tid).  Words are written
+// back to front at stage[wp-1], stage[wp-2], ...; returns the new wp.
+__device__ __forceinline__ int encode_step(int sym, int s, const EncEntry* __restrict__ tbl, uint32_t& x,
+                                           uint16_t* __restrict__ stage, int wp, int lane, uint32_t lt,
+                                           unsigned& n_escapes) {
+    int hi; uint32_t lo;
+    split_sym(sym, s, hi, lo);
+    const bool esc = hi > kHiMax || hi < -kHiMax;
+    const int zz = esc ? kEsc : (hi > 0 ? 2 * hi - 1 : -2 * hi);
+    const EncEntry e = tbl[zz];
+    const uint32_t f = e.fc & 0xffffu, c = e.fc >> 16;
+    const bool emit = x >= (f << 17);
+    const uint32_t emask = __ballot_sync(kFull, emit), xmask = __ballot_sync(kFull, esc);
+    const int n_emit = __popc(emask), n_esc = __popc(xmask);
+    const int base = wp - (2 * s + n_emit + 2 * n_esc);
+    if (xmask) {
+        if (esc) {
+            int at = base + 2 * s + n_emit + 2 * __popc(xmask & lt);
+            stage[at] = (uint16_t)((uint32_t)hi & 0xffffu);
+            stage[at + 1] = (uint16_t)((uint32_t)hi >> 16);
+        }
+        n_escapes += n_esc;
+    }
+    if (emit) {
+        stage[base + 2 * s + __popc(emask & lt)] = (uint16_t)(x & 0xffffu);
+        x >>= 16;
+    }
+    uint32_t q = __umulhi(x, e.rcp);
+    uint32_t r = x - q * f;
+    if (r >= f) { ++q; r -= f; }
+    x = (q << kProbBits) + r + c;
+    if (s) {
+        uint32_t mine = 0;
+        for (int b = 0; b < s; ++b) {
+            uint32_t plane = __ballot_sync(kFull, (lo >> b) & 1u);
+            if ((lane >> 1) == b) mine = plane;
+        }
+        if (lane < 2 * s) stage[base + lane] = (uint16_t)((lane & 1) ? (mine >> 16) : (mine & 0xffffu));
+    }
+    return base;
+}
+
+// One decoder step for the warp; words[rp...] with rp < nwords are readable.
+__device__ __forceinline__ int decode_step(int s, const uint16_t* __restrict__ cum, uint32_t& x,
+                                           const uint16_t* __restrict__ words, int& rp, int nwords, int lane,
+                                           uint32_t lt, bool& bad) {
+    uint32_t lo = 0;
+    if (s) {
+        uint32_t v = 0;
+        if (lane < 2 * s) {
+            int at = rp + lane;
+            if (at < nwords) v = __ldg(words + at); else bad = true;
+        }
+        for (int b = 0; b < s; ++b) {
+            uint32_t plane = __shfl_sync(kFull, v, 2 * b) | (__shfl_sync(kFull, v, 2 * b + 1) << 16);
+            lo |= ((plane >> lane) & 1u) << b;
+        }
+        rp += 2 * s;
+    }
+    const uint32_t slot = x & (kProbM - 1u);
+    int zz = 0;
+#pragma unroll
+    for (int step = 32; step > 0; step >>= 1)
+        if (cum[zz + step] <= slot) zz += step;
+    const uint32_t c = cum[zz], f = (uint32_t)cum[zz + 1] - c;
+    x = f * (x >> kProbBits) + slot - c;
+    const bool need = x < kRansL;
+    const uint32_t nmask = __ballot_sync(kFull, need);
+    if (need) {
+        int at = rp + __popc(nmask & lt);
+        uint32_t w = 0;
+        if (at < nwords) w = __ldg(words + at); else bad = true;
+        x = (x << 16) | w;
+    }
+    rp += __popc(nmask);
+    const bool esc = zz == kEsc;
+    const uint32_t xmask = __ballot_sync(kFull, esc);
+    int hi = (zz & 1) ? (zz + 1) >> 1 : -(zz >> 1);
+    if (xmask) {
+        if (esc) {
+            int at = rp + 2 * __popc(xmask & lt);
+            uint32_t a = 0, b = 0;
+            if (at + 1 < nwords) { a = __ldg(words + at); b = __ldg(words + at + 1); } else bad = true;
+            hi = (int)(a | (b << 16));
+        }
+        rp += 2 * __popc(xmask);
+    }
+    return join_sym(hi, lo, s);
+}
+
+__device__ __forceinline__ unsigned next_ticket(unsigned int* ticket, int lane) {
+    unsigned t = 0;
+    if (lane == 0) t = atomicAdd(ticket, 1u);
+    return __shfl_sync(kFull, t, 0);
+}
+
+template <int G>
+__device__ __forceinline__ void load_half_vec(const __half* p, float (&v)[G]) {
+    if constexpr (G == 8) {
+        uint4 r = *reinterpret_cast<const uint4*>(p);
+        const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { float2 f = __half22float2(hp[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
+    } else if constexpr (G == 4) {
+        uint2 r = *reinterpret_cast<const uint2*>(p);
+        const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) { float2 f = __half22float2(hp[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
+    } else if constexpr (G == 2) {
+        float2 f = __half22float2(*reinterpret_cast<const __half2*>(p));
+        v[0] = f.x; v[1] = f.y;
+    } else {
+        v[0] = __half2float(*p);
+    }
+}
+
+template <int G>
+__device__ __forceinline__ void store_vec(void* base, long long elem, const float (&v)[G], int out_f16) {
+    if (out_f16) {
+        __half* p = reinterpret_cast<__half*>(base) + elem;
+        if constexpr (G == 1) { *p = __float2half_rn(v[0]); }
+        else {
+            __half2 t[G / 2];
+#pragma unroll
+            for (int j = 0; j < G / 2; ++j) t[j] = __floats2half2_rn(v[2 * j], v[2 * j + 1]);
+            if constexpr (G == 8) *reinterpret_cast<uint4*>(p) = *reinterpret_cast<uint4*>(t);
+            else if constexpr (G == 4) *reinterpret_cast<uint2*>(p) = *reinterpret_cast<uint2*>(t);
+            else *reinterpret_cast<__half2*>(p) = t[0];
+        }
+    } else {
+        float* p = reinterpret_cast<float*>(base) + elem;
+        if constexpr (G >= 4) {
+#pragma unroll
+            for (int j = 0; j < G / 4; ++j)
+                reinterpret_cast<float4*>(p)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else if constexpr (G == 2) { *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]); }
+        else { *p = v[0]; }
+    }
+}
+
+struct Item {
+    int t, s, c;        // table, session, chunk
+    int p0, P;          // first position, positions in the chunk (0: no such chunk)
+    long long slot;
+};
+
+__device__ __forceinline__ Item bulk_item(const CodecArgs& a, unsigned item) {
+    Item it;
+    const int MC = a.st.max_chunks;
+    const unsigned per_table = (unsigned)a.S * (unsigned)MC;
+    it.t = (int)(item / per_table);
+    unsigned r = item % per_table;
+    it.s = (int)(r / MC);
+    it.c = (int)(r % MC);
+    const int Wt = 2 * a.sh.L * a.sh.H;
+    it.slot = ((long long)it.s * Wt + it.t) * MC + it.c;
+    int b = a.pos_begin ? a.pos_begin[it.s] : 0, e = a.pos_end ? a.pos_end[it.s] : a.n;
+    b = max(b, 0); e = min(e, a.n);
+    long long p0 = (long long)b + (long long)it.c * a.sh.chunk_pos;
+    it.p0 = (int)min(p0, (long long)a.n);
+    it.P = p0 < e ? min(a.sh.chunk_pos, e - (int)p0) : 0;
+    return it;
+}
+
+__device__ __forceinline__ long long kv_elem(const KvView& v, int t, int H, int s, int pos) {
+    int layer = t / (2 * H), kv = (t / H) & 1, head = t % H;
+    return layer * v.sl + kv * v.skv + s * v.ss + head * v.sh + (long long)pos * v.sp;
+}
+
+// Finishes an encoded chunk: reserves its place, writes states and words, index and counters.
+__device__ __forceinline__ void commit_chunk(const CodecArgs& a, long long slot, uint32_t x, const uint16_t* stage,
+                                             int wp, int cap_words, int lane, int P, unsigned n_escapes) {
+    __syncwarp();
+    const int n_words = cap_words - wp;
+    const unsigned nbytes = 128u + 2u * (unsigned)n_words;
+    unsigned long long off = 0;
+    if (lane == 0) {
+        off = atomicAdd(a.st.total_bytes, (unsigned long long)((nbytes + 15u) & ~15u));
+        atomicAdd(&a.counters->payload_bytes, (unsigned long long)nbytes);
+        atomicAdd(&a.counters->n_chunks, 1ull);
+        atomicAdd(&a.counters->coded_vectors, (unsigned long long)P);
+    }
+    off = __shfl_sync(kFull, off, 0);
+    if (lane == 0 && n_escapes) atomicAdd(&a.counters->n_escapes, (unsigned long long)n_escapes);
+    const bool fits = off + nbytes <= a.st.capacity;
+    if (lane == 0) {
+        a.st.chunk_offset[slot] = off;
+        a.st.chunk_bytes[slot] = nbytes;
+        if (!fits) atomicOr(a.status, kStCapacity);
+    }
+    if (!fits) return;
+    uint8_t* dst = a.st.payload + off;
+    reinterpret_cast<uint32_t*>(dst)[lane] = x;
+    uint16_t* dw = reinterpret_cast<uint16_t*>(dst + 128);
+    for (int i = lane; i < n_words; i += 32) dw[i] = __ldcg(stage + wp + i);
+}
+
+template <int D, bool FROM_OPEN>
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const CodecArgs a) {
+    constexpr int G = Geo<D>::G;
+    __shared__ EncTables tb;
+    build_enc_tables(&tb);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const uint32_t lt = lanemask_lt();
+    const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    uint16_t* stage = a.staging + gw * a.staging_words_per_warp;
+    const int cap_words = (int)a.staging_words_per_warp;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wt * a.S * a.st.max_chunks;
+    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const int c0 = first_comp<D>(lane);
+
+    for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
+        Item it;
+        if (FROM_OPEN) {
+            it.t = (int)(item / a.S); it.s = (int)(item % a.S); it.c = a.chunk_index;
+            it.p0 = 0; it.P = a.open_count;
+            it.slot = ((long long)it.s * Wt + it.t) * a.st.max_chunks + it.c;
+        } else {
+            it = bulk_item(a, item);
+        }
+        if (it.P <= 0) {
+            if (lane == 0 && !FROM_OPEN) { a.st.chunk_offset[it.slot] = 0; a.st.chunk_bytes[it.slot] = 0; }
+            continue;
+        }
+        const __half* table = a.T + (size_t)it.t * a.sh.V * D;
+        const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
+        uint32_t x = kRansL;
+        int wp = cap_words;
+        unsigned n_escapes = 0;
+        for (int p = it.P - 1; p >= 0; --p) {
+            int sym[G];
+            int q;
+            if (FROM_OPEN) {
+                const long long o = ((long long)it.s * Wt + it.t) * a.sh.chunk_pos + p;
+                q = a.open_q[o];
+#pragma unroll
+                for (int g = 0; g < G; ++g) sym[g] = a.open_sym[o * D + c0 + g];
+            } else {
+                const int pos = it.p0 + p;
+                const long long row = (long long)it.s * a.n + pos;
+                float mu[G], sigma2;
+                predict<D>(table, n2, a.pairs + row * K, K, lane, inv_d, mu, sigma2);
+                q = scale_class(sigma2, floor2, delta2);
+                float kvv[G];
+                load_half_vec<G>(reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, it.t, H, it.s, pos) + c0, kvv);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float r = __fsub_rn(kvv[g], mu[g]);
+                    float n = rintf(__fdiv_rn(r, delta));
+                    n = fminf(fmaxf(n, -(float)kSymLimit), (float)kSymLimit);
+                    sym[g] = (int)n;
+                }
+                if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
+                    const long long o = row * Wt + it.t;
+                    if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        if (a.dbg.sym) a.dbg.sym[o * D + c0 + g] = sym[g];
+                        if (a.dbg.mu) a.dbg.mu[o * D + c0 + g] = mu[g];
+                    }
+                }
+            }
+            int s, qp;
+            class_params(q, s, qp);
+            const EncEntry* tbl = tb.enc[qp - kQMin];
+#pragma unroll
+            for (int g = G - 1; g >= 0; --g) wp = encode_step(sym[g], s, tbl, x, stage, wp, lane, lt, n_escapes);
+        }
+        commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes);
+        __syncwarp();
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const CodecArgs a) {
+    constexpr int G = Geo<D>::G;
+    __shared__ DecTables tb;
+    build_dec_tables(&tb);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const uint32_t lt = lanemask_lt();
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const unsigned total = (unsigned)Wt * a.S * a.st.max_chunks;
+    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const int c0 = first_comp<D>(lane);
+
+    for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
+        const Item it = bulk_item(a, item);
+        if (it.P <= 0) continue;
+        const unsigned long long off = a.st.chunk_offset[it.slot];
+        const unsigned nbytes = a.st.chunk_bytes[it.slot];
+        if (nbytes < 128u || (nbytes & 1u) || (off & 15ull) || off + nbytes > a.st.capacity) {
+            if (lane == 0) atomicOr(a.status, kStCorrupt);
+            continue;
+        }
+        const uint8_t* src = a.st.payload + off;
+        uint32_t x = reinterpret_cast<const uint32_t*>(src)[lane];
+        bool bad = x < kRansL;
+        const uint16_t* words = reinterpret_cast<const uint16_t*>(src + 128);
+        const int nwords = (int)((nbytes - 128u) >> 1);
+        int rp = 0;
+        const __half* table = a.T + (size_t)it.t * a.sh.V * D;
+        const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
+        for (int p = 0; p < it.P; ++p) {
+            const int pos = it.p0 + p;
+            const long long row = (long long)it.s * a.n + pos;
+            float mu[G], sigma2;
+            predict<D>(table, n2, a.pairs + row * K, K, lane, inv_d, mu, sigma2);
+            const int q = scale_class(sigma2, floor2, delta2);
+            int s, qp;
+            class_params(q, s, qp);
+            const uint16_t* cum = tb.cum[qp - kQMin];
+            int sym[G];
+            float out[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                sym[g] = decode_step(s, cum, x, words, rp, nwords, lane, lt, bad);
+                out[g] = __fmaf_rn((float)sym[g], delta, mu[g]);
+            }
+            store_vec<G>(a.kv.base, kv_elem(a.kv, it.t, H, it.s, pos) + c0, out, a.sh.out_dtype);
+            if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
+                const long long o = row * Wt + it.t;
+                if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    if (a.dbg.sym) a.dbg.sym[o * D + c0 + g] = sym[g];
+                    if (a.dbg.mu) a.dbg.mu[o * D + c0 + g] = mu[g];
+                }
+            }
+        }
+        bad = bad || x != kRansL || rp != nwords;
+        if (__any_sync(kFull, bad) && lane == 0) atomicOr(a.status, kStCorrupt);
+    }
+}
+
+// Decode-time append: one warp per (session, table) predicts the new position and stores its
+// symbols and class in slot a.open_slot of the stream's open chunk.
+template <int D>
+__global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecArgs a) {
+    constexpr int G = Geo<D>::G;
+    const int lane = threadIdx.x & 31;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const long long nw = (long long)gridDim.x * kWarpsPerBlock;
+    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const int c0 = first_comp<D>(lane);
+    for (long long item = gw; item < (long long)Wt * a.S; item += nw) {
+        const int t = (int)(item / a.S), b = (int)(item % a.S);
+        const __half* table = a.T + (size_t)t * a.sh.V * D;
+        float mu[G], sigma2;
+        predict<D>(table, a.rownorm2 + (size_t)t * a.sh.V, a.pairs + (long long)b * K, K, lane, inv_d, mu, sigma2);
+        const int q = scale_class(sigma2, floor2, delta2);
+        float kvv[G];
+        load_half_vec<G>(reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, t, H, b, 0) + c0, kvv);
+        const long long o = ((long long)b * Wt + t) * a.sh.chunk_pos + a.open_slot;
+        if (lane == 0) a.open_q[o] = q;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float r = __fsub_rn(kvv[g], mu[g]);
+            float n = rintf(__fdiv_rn(r, delta));
+            n = fminf(fmaxf(n, -(float)kSymLimit), (float)kSymLimit);
+            a.open_sym[o * D + c0 + g] = (int)n;
+        }
+    }
+}
+
+template <class F>
+cudaError_t dispatch_d(int d, F&& f) {
+    switch (d) {
+        case 32: return f(std::integral_constant<int, 32>{});
+        case 64: return f(std::integral_constant<int, 64>{});
+        case 128: return f(std::integral_constant<int, 128>{});
+        case 256: return f(std::integral_constant<int, 256>{});
+    }
+    return cudaErrorInvalidValue;
+}
+
+int sm_count() {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
+}  // namespace
+
+int codec_grid_warps(int) { return sm_count() * kBlocksPerSM * kWarpsPerBlock; }
+
+cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st) {
+    return dispatch_d(d, [&](auto D) {
+        long long blocks = (rows + 7) / 8;
+        if (blocks > (long long)sm_count() * 16) blocks = (long long)sm_count() * 16;
+        rownorm_kernel<decltype(D)::value><<<(unsigned)blocks, 256, 0, st>>>(T, out, rows);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return e;
+    return dispatch_d(a.sh.d, [&](auto D) {
+        encode_kernel<decltype(D)::value, false><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return e;
+    return dispatch_d(a.sh.d, [&](auto D) {
+        long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
+        long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
+        if (blocks > (long long)sm_count() * kBlocksPerSM) blocks = (long long)sm_count() * kBlocksPerSM;
+        encode_kernel<decltype(D)::value, true><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return e;
+    return dispatch_d(a.sh.d, [&](auto D) {
+        decode_kernel<decltype(D)::value><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_append_quantise(const CodecArgs& a, cudaStream_t st) {
+    return dispatch_d(a.sh.d, [&](auto D) {
+        long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
+        long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
+        if (blocks > (long long)sm_count() * 8) blocks = (long long)sm_count() * 8;
+        append_quantise_kernel<decltype(D)::value><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+}  // namespace plc

@@ -1,0 +1,199 @@
+// Shared definitions of the libplc CUDA translation units (sm_100a only).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "plc.h"
+
+namespace plc {
+
+constexpr int kProbBits = 15;
+constexpr uint32_t kProbM = 1u << kProbBits;
+constexpr uint32_t kRansL = 1u << 16;
+constexpr int kNumSym = 64;        // zigzag(hi), hi in [-31,31] -> 0..62; 63 = escape
+constexpr int kEsc = 63;
+constexpr int kHiMax = 31;
+constexpr int kQMin = -24;
+constexpr int kQMax = 135;
+constexpr int kNumTables = 40;     // table id qp in [-24, 15]
+constexpr int kSymLimit = 1 << 30;
+constexpr uint32_t kFull = 0xffffffffu;
+
+// Bits of the device status word.
+constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u;
+
+// Device counters (plc_stats).
+struct Counters {
+    unsigned long long payload_bytes, n_chunks, n_escapes, coded_vectors;
+};
+
+// Frequency-table entry used by the encoder: rcp = floor(2^32 / f) (2^32-1 for f = 1),
+// fc = f | (c << 16).
+struct EncEntry {
+    uint32_t rcp, fc;
+};
+
+// Per-class tables as they sit in shared memory.
+struct __align__(16) Tables {
+    EncEntry enc[kNumTables][kNumSym];      // 20 KB
+    uint16_t cum[kNumTables][kNumSym + 2];  // c[0..64], padded: 5280 B
+};
+
+// Two 32-bit constants per table id: theta = round(2^32 exp(-sqrt2/s')), rho = round(2^32
+// exp(-sqrt2/(2 s'))), s' = 2^(qp/8).  Literal so that encoder and decoder builds agree bit for bit.
+__host__ __device__ inline void table_constants(int qp, uint32_t& theta, uint32_t& rho) {
+    constexpr uint32_t kC[kNumTables][2] = {
+        {52418u, 15004422u},         {134053u, 23994893u},        {317125u, 36905875u},
+        {698470u, 54771407u},        {1440801u, 78665070u},       {2798733u, 109637892u},
+        {5145013u, 148652826u},      {8992185u, 196522626u},      {15004422u, 253857248u},
+        {23994893u, 321025356u},     {36905875u, 398132550u},     {54771407u, 485016909u},
+        {78665070u, 581260615u},     {109637892u, 686215099u},    {148652826u, 799036310u},
+        {196522626u, 918726429u},    {253857248u, 1044178424u},   {321025356u, 1174220339u},
+        {398132550u, 1307656790u},   {485016909u, 1443305845u},   {581260615u, 1580030169u},
+        {686215099u, 1716761896u},   {799036310u, 1852521207u},   {918726429u, 1986428948u},
+        {1044178424u, 2117713904u},  {1174220339u, 2245715466u},  {1307656790u, 2369882518u},
+        {1443305845u, 2489769347u},  {1580030169u, 2605029347u},  {1716761896u, 2715407188u},
+        {1852521207u, 2820730047u},  {1986428948u, 2920898384u},  {2117713904u, 3015876649u},
+        {2245715466u, 3105684222u},  {2369882518u, 3190386796u},  {2489769347u, 3270088366u},
+        {2605029347u, 3344923893u},  {2715407188u, 3415052718u},  {2820730047u, 3480652712u},
+        {2920898384u, 3541915165u}};
+    theta = kC[qp - kQMin][0];
+    rho = kC[qp - kQMin][1];
+}
+
+// Discretised Laplace frequencies of table qp, integer recurrence:
+// G0 = 2^32, G1 = rho, G(k+1) = (Gk theta) >> 32; f(0) = (G0-G1) >> 17, f(+-k) = (Gk-Gk+1) >> 18,
+// f(ESC) = G32 >> 17, each at least 1; f(0) absorbs the difference to 2^15.
+__host__ __device__ inline void build_freqs(int qp, uint32_t* f /*[64]*/) {
+    uint32_t theta, rho;
+    table_constants(qp, theta, rho);
+    unsigned long long g = 1ull << 32, gn = rho;
+    unsigned long long m = (g - gn) >> 17;
+    f[0] = m < 1 ? 1u : (uint32_t)m;
+    g = gn;
+    for (int k = 1; k <= kHiMax; ++k) {
+        gn = (g * (unsigned long long)theta) >> 32;
+        m = (g - gn) >> 18;
+        uint32_t fk = m < 1 ? 1u : (uint32_t)m;
+        f[2 * k - 1] = fk;
+        f[2 * k] = fk;
+        g = gn;
+    }
+    m = g >> 17;
+    f[kEsc] = m < 1 ? 1u : (uint32_t)m;
+    long long sum = 0;
+    for (int i = 0; i < kNumSym; ++i) sum += f[i];
+    f[0] = (uint32_t)((long long)f[0] + ((long long)kProbM - sum));
+}
+
+// Scale class -> (number of bit planes s, table id qp).
+__host__ __device__ inline void class_params(int q, int& s, int& qp) {
+    if (q < 16) { s = 0; qp = q; }
+    else { s = (q >> 3) - 1; qp = 8 + (q & 7); }
+}
+
+#ifdef __CUDACC__
+// q = clamp(round(4 log2 v), kQMin, kQMax), decided on the binary32 exponent and four mantissa
+// thresholds 2^((2i+1)/8); v <= 0 -> kQMin.
+__device__ __forceinline__ int class_from_v(float v) {
+    if (!(v > 0.0f)) return kQMin;
+    uint32_t b = __float_as_uint(v);
+    int e = (int)(b >> 23);
+    if (e == 255) return kQMax;
+    float m;
+    if (e == 0) {                      // subnormal: far below the smallest class
+        return kQMin;
+    }
+    m = __uint_as_float((b & 0x007fffffu) | 0x3f800000u);   // [1,2)
+    int q = 4 * (e - 127);
+    q += (m >= 1.09050773f) + (m >= 1.29683955f) + (m >= 1.54221083f) + (m >= 1.83400809f);
+    return min(max(q, kQMin), kQMax);
+}
+
+__device__ __forceinline__ uint32_t lanemask_lt() {
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// Fills the shared-memory tables; call with all threads of the block, then __syncthreads().
+__device__ inline void build_tables_smem(Tables* t) {
+    for (int id = threadIdx.x; id < kNumTables; id += blockDim.x) {
+        uint32_t f[kNumSym];
+        build_freqs(id + kQMin, f);
+        uint32_t c = 0;
+        for (int i = 0; i < kNumSym; ++i) {
+            uint32_t fi = f[i];
+            t->enc[id][i].rcp = fi == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / fi);
+            t->enc[id][i].fc = fi | (c << 16);
+            t->cum[id][i] = (uint16_t)c;
+            c += fi;
+        }
+        t->cum[id][kNumSym] = (uint16_t)c;       // 2^15 wraps to 0x8000: fits uint16
+        t->cum[id][kNumSym + 1] = 0xffff;
+    }
+}
+#endif
+
+// Host-side launch counter shared by all translation units.
+void count_launch(int n = 1);
+
+// Internal launchers (one per .cu file).
+struct TopkArgs {
+    const __half* logits; const int32_t* tokens; int64_t N; int V, K;
+    int2* pairs;            // [N][K] {idx, float bits of w}, or null
+    int32_t* idx; float* w; float* lse; float* zk; float* logp2;   // optional user outputs
+    // Rows are skipped (nothing written) when pos ranges are given and the row is outside them.
+    int n_per_session; const int32_t* pos_begin; const int32_t* pos_end;
+};
+cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st);
+
+cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,
+                                int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st);
+
+struct CodecShape {
+    int L, H, d, V, K, chunk_pos, out_dtype;
+    float delta, sigma_floor;
+};
+
+struct KvView {
+    void* base; int64_t sl, skv, ss, sh, sp;
+};
+
+struct StreamsDev {
+    uint8_t* payload; unsigned long long capacity; unsigned long long* chunk_offset; uint32_t* chunk_bytes;
+    unsigned long long* total_bytes; int max_chunks;
+};
+
+struct DebugDev {
+    int32_t* sym; int32_t* q; float* mu;
+};
+
+struct CodecArgs {
+    CodecShape sh;
+    const __half* T; const float* rownorm2;        // [tables][V][d], [tables][V]
+    const int2* pairs;                             // [S*n][K]
+    KvView kv;                                     // encode: input f16; decode: output
+    int S, n; const int32_t* pos_begin; const int32_t* pos_end;
+    StreamsDev st; DebugDev dbg;
+    uint16_t* staging; unsigned long long staging_words_per_warp;   // encoder scratch
+    unsigned int* ticket;                          // work counter (zeroed by the launcher)
+    unsigned int* status; Counters* counters;
+    // append path: symbols come from / go to the open chunk
+    int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
+};
+int codec_grid_warps(int device);
+cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st);
+cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st);
+cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st);
+cudaError_t launch_append_quantise(const CodecArgs& a, cudaStream_t st);   // predict + quantise into the open chunk
+cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st);       // code the open chunk
+
+}  // namespace plc

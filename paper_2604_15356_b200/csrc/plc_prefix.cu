@@ -1,0 +1,64 @@
+// Batched longest common prefix and trie metric d_T(a,b) = -log2 P(a ^ b) over S sessions: one warp
+// per ordered pair (a,b).  The log-probability of the common prefix is summed in double in a fixed
+// order, so the result does not depend on scheduling.
+#include "plc_common.cuh"
+
+namespace plc {
+namespace {
+
+__global__ void __launch_bounds__(256) lcp_dt_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ lens,
+                                                     const float* __restrict__ logp2, int S, long long stride,
+                                                     int32_t* __restrict__ lcp, float* __restrict__ dT) {
+    const int lane = threadIdx.x & 31;
+    const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long pair = warp; pair < (long long)S * S; pair += nwarps) {
+        const int a = (int)(pair / S), b = (int)(pair % S);
+        const int32_t* ta = tokens + a * stride;
+        const int32_t* tb = tokens + b * stride;
+        const int m = (int)max(0ll, min((long long)min(lens[a], lens[b]), stride));
+        int n = m;
+        for (int base = 0; base < m; base += 32) {
+            int j = base + lane;
+            bool differ = (j < m) && (ta[j] != tb[j]);
+            uint32_t mask = __ballot_sync(kFull, differ);
+            if (mask) { n = base + __ffs(mask) - 1; break; }
+        }
+        double acc = 0.0;
+        const float* la = logp2 + a * stride;
+        for (int j = lane; j < n; j += 32) acc -= (double)la[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
+        if (lane == 0) { lcp[pair] = n; dT[pair] = (float)acc; }
+    }
+}
+
+// parent[a] = earlier session with the longest common prefix (smallest index among equals).
+__global__ void parent_kernel(const int32_t* __restrict__ lcp, int S, int32_t* __restrict__ parent,
+                              int32_t* __restrict__ shared_len) {
+    int a = blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= S) return;
+    int best = -1, bl = 0;
+    for (int b = 0; b < a; ++b) {
+        int v = lcp[(long long)a * S + b];
+        if (v > bl) { bl = v; best = b; }
+    }
+    parent[a] = best;
+    shared_len[a] = bl;
+}
+
+}  // namespace
+
+cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,
+                                int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st) {
+    if (S <= 0) return cudaSuccess;
+    long long pairs = (long long)S * S;
+    long long blocks = (pairs + 7) / 8;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    lcp_dt_kernel<<<(unsigned)blocks, 256, 0, st>>>(tokens, lens, logp2, S, (long long)stride, lcp, dT);
+    parent_kernel<<<(S + 127) / 128, 128, 0, st>>>(lcp, S, parent, shared_len);
+    count_launch(2);
+    return cudaGetLastError();
+}
+
+}  // namespace plc

@@ -1,0 +1,372 @@
+"""GPU <-> oracle parity through the C ABI, on seeded synthetic inputs.
+
+Tolerances (written here once, used below):
+  * top-K indices, LCP lengths, parents, decoded symbols, chunk bytes: bit-exact;
+  * prediction mu: per vector, max |mu_gpu - mu_oracle| <= 1e-3 * max(max|mu_oracle|, 1e-3);
+  * quantised symbols: fewer than 1e-4 differ, each by one step and only where r/delta is within
+    1e-3 of a half-integer;
+  * scale classes: the kernel forms sigma^2 = (sum_k w_k |T_k|^2 - |mu|^2)/d in binary32, whose
+    cancellation error is at most ~4e-7 * sum_k w_k |T_k|^2 / d; a class may differ from the
+    oracle's only where 4 log2(v) is within 4 * that / (sigma^2 ln 2) + 1e-3 of a rounding
+    boundary, and by one; fewer than 1e-2 of them;
+  * reconstructed KV: |KV' - KV| <= delta/2 + 1e-3;
+  * total compressed size within 0.1 % of the oracle's;
+  * d_T within 1e-4 relative.
+"""
+import ctypes as C
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2604_15356_b200 as plc
+from paper_2604_15356_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    plc.build()
+    return torch.device("cuda:0")
+
+
+def make_workload(seed, S, n, L, H, d, V, K, pp=12.0, sigma=0.05, alpha=0.0, max_states=256):
+    table = synth.markov_table(V, pp, seed, alpha=alpha, max_states=max_states)
+    tokens = synth.sample_tokens(table, S, n, seed + 1)
+    logits = synth.position_logits(table, tokens)
+    T = synth.make_tables(L, H, V, d, seed + 2)
+    kv = synth.make_kv(T, tokens, sigma, seed + 3)
+    return tokens, logits, T, kv
+
+
+def gpu_encode(dev, T, kv, logits, K, delta, CP, pos_begin=None, pos_end=None, capacity=None, sigma_floor=0.0):
+    L, _, H, V, d = T.shape
+    S, n = logits.shape[:2]
+    ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, sigma_floor=sigma_floor)
+    W = ctx.W
+    mc = ctx.max_chunks(n)
+    cap = capacity if capacity is not None else S * W * mc * 160 + 3 * S * n * W * d + 4096
+    st = plc.StreamSet(S * W, mc, cap, dev)
+    sym = torch.zeros(S, n, W, d, dtype=torch.int32, device=dev)
+    q = torch.full((S, n, W), -99, dtype=torch.int32, device=dev)
+    mu = torch.zeros(S, n, W, d, dtype=torch.float32, device=dev)
+    dbg = plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr())
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    pb = None if pos_begin is None else torch.tensor(pos_begin, dtype=torch.int32, device=dev)
+    pe = None if pos_end is None else torch.tensor(pos_end, dtype=torch.int32, device=dev)
+    ctx.encode(kvd, lgd, st, pb, pe, debug=dbg)
+    rc = ctx.sync_status()
+    return dict(ctx=ctx, st=st, sym=sym, q=q, mu=mu, rc=rc, kv=kvd, logits=lgd, pb=pb, pe=pe, W=W, mc=mc)
+
+
+def check_against_oracle(orc, g, T, kv, logits, K, delta, CP, pos_begin=None, pos_end=None, sigma_floor=0.0):
+    L, _, H, V, d = T.shape
+    S, n = logits.shape[:2]
+    W = g["W"]
+    cfg = orc.Config(L, H, d, V, K, delta, sigma_floor, CP, 0)
+    enc = orc.encode(cfg, T.numpy(), kv.numpy(), logits.numpy(), None, pos_begin, pos_end, export=True)
+    sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W); mu_o = enc["mu"].reshape(S, n, W, d)
+    sym_g = g["sym"].cpu().numpy(); q_g = g["q"].cpu().numpy(); mu_g = g["mu"].cpu().numpy()
+    coded = np.zeros((S, n), bool)
+    for s in range(S):
+        b = 0 if pos_begin is None else pos_begin[s]
+        e = n if pos_end is None else pos_end[s]
+        coded[s, b:e] = True
+    assert np.all(q_g[~coded] == -99) and not sym_g[~coded].any()            # uncoded positions untouched
+    mo, mg, so, sg, qo, qg = mu_o[coded], mu_g[coded], sym_o[coded], sym_g[coded], q_o[coded], q_g[coded]
+    # prediction
+    scale = np.maximum(np.abs(mo).max(-1), 1e-3)
+    assert (np.abs(mg - mo).max(-1) <= 1e-3 * scale).all()
+    # symbols
+    diff = sg != so
+    assert diff.mean() < 1e-4
+    if diff.any():
+        assert np.abs(sg - so)[diff].max() == 1
+        # recompute r/delta at the differing places from the oracle's mu
+        kvv = np.transpose(kv.numpy().astype(np.float64), (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)[coded]
+        t = (kvv - mo.astype(np.float64)) / delta
+        frac = np.abs(t - np.floor(t) - 0.5)
+        assert frac[diff].max() < 1e-3
+    # classes
+    qd = q_g != q_o
+    qd &= coded[:, :, None]
+    assert qd.sum() <= 1e-2 * coded.sum() * W
+    if qd.any():
+        idx_o, w_o, *_ = orc.topk_softmax(logits.numpy().reshape(S * n, V), None, K)
+        Tn = T.numpy().reshape(W, V, d)
+        for s_, i_, t_ in np.argwhere(qd)[:300]:
+            assert abs(int(q_g[s_, i_, t_]) - int(q_o[s_, i_, t_])) == 1
+            ii, ww = idx_o[s_ * n + i_], w_o[s_ * n + i_]
+            _, s2 = orc.mixture(Tn[t_], ii, ww)
+            s1 = float((ww * (Tn[t_][ii].astype(np.float64) ** 2).sum(1)).sum()) / d
+            v = (s2 + sigma_floor ** 2) / delta ** 2
+            tq = 4 * math.log2(v)
+            tol = 4 * (4e-7 * s1) / (max(s2, 1e-30) * math.log(2)) + 1e-3
+            assert abs(tq - math.floor(tq) - 0.5) <= tol, (s_, i_, t_, tq, tol)
+    # bitstream: the oracle coder fed with the GPU's symbols and classes gives the GPU's bytes
+    st = g["st"]
+    off = st.chunk_offset.cpu().numpy(); nby = st.chunk_bytes.cpu().numpy().astype(np.int64)
+    payload = st.payload.cpu().numpy()
+    assert np.all(off % 16 == 0)
+    mc = g["mc"]
+    total_g = 0
+    for s in range(S):
+        b = 0 if pos_begin is None else pos_begin[s]
+        e = n if pos_end is None else pos_end[s]
+        for t_ in range(W):
+            for c in range(mc):
+                slot = (s * W + t_) * mc + c
+                p0 = b + c * CP
+                if p0 >= e:
+                    assert nby[slot] == 0
+                    continue
+                P = min(CP, e - p0)
+                ref, _, _ = orc.rans_encode_chunk(sym_g[s, p0:p0 + P, t_], q_g[s, p0:p0 + P, t_])
+                got = payload[off[slot]:off[slot] + nby[slot]]
+                assert nby[slot] == len(ref) and np.array_equal(got, ref), (s, t_, c)
+                rc, back = orc.rans_decode_chunk(got, q_g[s, p0:p0 + P, t_], d)
+                assert rc == 0 and np.array_equal(back, sym_g[s, p0:p0 + P, t_])
+                total_g += nby[slot]
+    stats = g["ctx"].stats()
+    assert stats.payload_bytes == total_g
+    assert abs(total_g / enc["stats"].payload_bytes - 1) < 1e-3
+    return enc
+
+
+def gpu_decode_check(g, kv, delta, n, pos_begin=None, pos_end=None, out_dtype=plc.OUT_F32):
+    dev = g["kv"].device
+    S = g["logits"].shape[0]
+    ctx, st = g["ctx"], g["st"]
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    sym2 = torch.zeros_like(g["sym"])
+    dbg = plc.DebugBuffers(sym2.data_ptr(), None, None)
+    ctx.decode(st, g["logits"], out, g["pb"], g["pe"], debug=dbg)
+    assert ctx.sync_status() == plc.OK
+    assert torch.equal(sym2, g["sym"])                                       # decode inverts encode exactly
+    coded = torch.zeros(S, n, dtype=torch.bool)
+    for s in range(S):
+        b = 0 if pos_begin is None else pos_begin[s]
+        e = n if pos_end is None else pos_end[s]
+        coded[s, b:e] = True
+    o = out.cpu().permute(2, 4, 0, 1, 3, 5)      # [S][n][L][2][H][d]
+    k = kv.float().permute(2, 4, 0, 1, 3, 5)
+    assert float((o[coded] - k[coded]).abs().max()) <= delta / 2 + 1e-3
+    assert not o[~coded].any()
+    return out
+
+
+def test_topk_softmax_parity(dev, orc):
+    rng = np.random.default_rng(0)
+    for V, K, N in [(256, 16, 40), (32000, 64, 24), (1000, 64, 16), (37, 5, 9), (4096, 1, 8), (2048, 1024, 3)]:
+        lg = (rng.standard_normal((N, V)) * 2.5).astype(np.float16)
+        lg[1, :] = np.float16(0.25)                              # every logit equal
+        lg[2, ::2] = lg[2, 0]                                    # half the row tied at one value
+        lg[3, :7] = np.float16(-0.0); lg[3, 7:14] = np.float16(0.0)
+        tok = rng.integers(0, V, N).astype(np.int32)
+        T = torch.zeros(1, 2, 1, V, 32, dtype=torch.float16, device=dev)
+        ctx = plc.Context(T, K, 0.02)
+        out = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev))
+        idx, w, lse, zk, lp = orc.topk_softmax(lg, tok, K)
+        assert np.array_equal(out["idx"].cpu().numpy(), idx), (V, K)
+        np.testing.assert_allclose(out["w"].cpu().numpy(), w, rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(out["lse"].cpu().numpy(), lse, atol=2e-5)
+        np.testing.assert_allclose(out["zk"].cpu().numpy(), zk, rtol=2e-5)
+        np.testing.assert_allclose(out["logp2"].cpu().numpy(), lp, atol=1e-4)
+        again = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev))
+        for k in out:
+            assert torch.equal(out[k], again[k])                  # run-to-run identical
+
+
+def test_tiny_config_full_parity(dev, orc):
+    """Tiny: 1 session x 512 tokens, 1 layer, 1 head, d=64, V=256, K=16, delta=0.02, perplexity 12."""
+    tokens, logits, T, kv = make_workload(20260416, 1, 512, 1, 1, 64, 256, 16)
+    g = gpu_encode(dev, T, kv, logits, 16, 0.02, 256)
+    assert g["rc"] == plc.OK
+    check_against_oracle(orc, g, T, kv, logits, 16, 0.02, 256)
+    gpu_decode_check(g, kv, 0.02, 512)
+
+
+@pytest.mark.parametrize("d,K,V,n,CP", [(128, 64, 2000, 300, 128), (32, 7, 64, 70, 32), (256, 20, 512, 45, 16),
+                                        (64, 64, 4096, 130, 64)])
+def test_multi_stream_ragged_parity(dev, orc, d, K, V, n, CP):
+    tokens, logits, T, kv = make_workload(100 + d, 2, n, 2, 2, d, V, K, pp=15.0, alpha=1.1 if d == 128 else 0.0)
+    g = gpu_encode(dev, T, kv, logits, K, 0.02, CP)
+    assert g["rc"] == plc.OK
+    check_against_oracle(orc, g, T, kv, logits, K, 0.02, CP)
+    gpu_decode_check(g, kv, 0.02, n)
+
+
+def test_position_ranges_and_empty_sessions(dev, orc):
+    tokens, logits, T, kv = make_workload(7, 3, 100, 1, 2, 128, 512, 32)
+    pb, pe = [0, 37, 100], [100, 91, 100]
+    g = gpu_encode(dev, T, kv, logits, 32, 0.02, 32, pb, pe)
+    assert g["rc"] == plc.OK
+    check_against_oracle(orc, g, T, kv, logits, 32, 0.02, 32, pb, pe)
+    gpu_decode_check(g, kv, 0.02, 100, pb, pe)
+    assert g["ctx"].stats().coded_vectors == (100 + 54) * g["W"]
+
+
+@pytest.mark.parametrize("delta,pp", [(0.005, 4.0), (0.08, 50.0), (0.02, 1.2)])
+def test_step_and_perplexity_sweep(dev, orc, delta, pp):
+    tokens, logits, T, kv = make_workload(int(delta * 1000) + 5, 1, 96, 1, 2, 128, 1024, 64, pp=pp)
+    g = gpu_encode(dev, T, kv, logits, 64, delta, 32)
+    assert g["rc"] == plc.OK
+    check_against_oracle(orc, g, T, kv, logits, 64, delta, 32)
+    gpu_decode_check(g, kv, delta, 96)
+
+
+def test_sigma_floor_and_escapes(dev, orc):
+    """A point-mass prediction with noisy KV: tiny scale, large residuals -> escapes must round-trip."""
+    tokens, logits, T, kv = make_workload(9, 1, 64, 1, 1, 128, 256, 16, sigma=0.3)
+    lg = np.full(logits.shape, -40.0, np.float16)
+    np.put_along_axis(lg[0], tokens[0].numpy()[:, None].astype(np.int64), np.float16(40.0), axis=1)
+    logits = torch.from_numpy(lg)
+    g = gpu_encode(dev, T, kv, logits, 16, 0.005, 32)
+    assert g["rc"] == plc.OK and g["ctx"].stats().n_escapes > 0
+    assert np.all(g["q"].cpu().numpy() == -24)
+    check_against_oracle(orc, g, T, kv, logits, 16, 0.005, 32)
+    gpu_decode_check(g, kv, 0.005, 64)
+    g2 = gpu_encode(dev, T, kv, logits, 16, 0.005, 32, sigma_floor=0.3)
+    assert g2["ctx"].stats().n_escapes < g["ctx"].stats().n_escapes
+    check_against_oracle(orc, g2, T, kv, logits, 16, 0.005, 32, sigma_floor=0.3)
+
+
+def test_capacity_overflow_is_reported_not_written(dev):
+    tokens, logits, T, kv = make_workload(11, 1, 128, 1, 2, 128, 512, 32)
+    big = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
+    need = int(big["st"].total_bytes)
+    cap = need // 2
+    g = gpu_encode(dev, T, kv, logits, 32, 0.02, 32, capacity=cap + 64)
+    assert g["rc"] == plc.E_CAPACITY
+    assert int(g["st"].total_bytes) == need                       # the size that would have been needed
+    guard = g["st"].payload[cap:]                                  # nothing past the stated capacity ...
+    assert g["st"].payload.numel() == cap + 64
+    g["ctx"].cfg                                                   # (context stays usable)
+    assert g["ctx"].sync_status() == plc.OK                        # status word was cleared by the read
+
+
+def test_damaged_streams_are_reported(dev):
+    tokens, logits, T, kv = make_workload(12, 1, 64, 1, 2, 128, 512, 32)
+    g = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
+    ctx, st = g["ctx"], g["st"]
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    good_bytes = st.chunk_bytes.clone(); good_payload = st.payload.clone()
+    # truncated chunk
+    st.chunk_bytes[0] = int(good_bytes[0]) - 40
+    ctx.decode(st, g["logits"], out)
+    assert ctx.sync_status() == plc.E_CORRUPT
+    # chunk that claims to extend past the buffer
+    st.chunk_bytes.copy_(good_bytes); st.chunk_offset[1] = st.payload.numel() - 16
+    ctx.decode(st, g["logits"], out)
+    assert ctx.sync_status() == plc.E_CORRUPT
+    # a start state below 2^16 is always caught; flipped payload bits either fail the end-state check
+    # or (raw bit planes) change symbols, but never leave the chunk's bytes
+    st2 = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
+    base = int(st2["st"].chunk_offset[3])
+    st2["st"].payload[base + 6:base + 8] = 0
+    st2["ctx"].decode(st2["st"], st2["logits"], out)
+    assert st2["ctx"].sync_status() == plc.E_CORRUPT
+    hits = 0
+    for k in range(12):
+        st3 = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
+        st3["st"].payload[int(st3["st"].chunk_offset[2]) + 130 + 37 * k] ^= 0x3C
+        st3["ctx"].decode(st3["st"], st3["logits"], out)
+        rc = st3["ctx"].sync_status()
+        assert rc in (plc.OK, plc.E_CORRUPT)
+        hits += rc == plc.E_CORRUPT
+    assert hits >= 3
+    # and an undamaged stream still decodes afterwards on the same context
+    st.chunk_bytes.copy_(good_bytes); st.chunk_offset.copy_(g["st"].chunk_offset)
+    g3 = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
+    g3["ctx"].decode(g3["st"], g3["logits"], out)
+    assert g3["ctx"].sync_status() == plc.OK
+
+
+def test_prefix_dedup_parity_and_tail_coding(dev, orc):
+    """Sessions with shared system prefixes from a prefix trie: LCP / d_T / parents, then the tail
+    is coded from shared_len on (device-resident pos_begin, no host round trip)."""
+    V, S, n, K = 1024, 12, 400, 32
+    table = synth.markov_table(V, 12.0, 31, max_states=128)
+    tokens, keys, leaf, plen = synth.trie_sessions(table, S, n, 32, 20, 90)
+    start = None
+    logits = synth.position_logits(table, tokens)
+    T = synth.make_tables(1, 2, V, 128, 33)
+    kv = synth.make_kv(T, tokens, 0.05, 34, keys=keys)
+    ctx = plc.Context(T.to(dev), K, 0.02, chunk_pos=64)
+    lgd, tkd = logits.to(dev), tokens.to(dev)
+    out = ctx.topk_softmax(lgd, tkd.reshape(-1), want=("logp2",))
+    logp2 = out["logp2"].view(S, n)
+    lens = torch.tensor([n, n - 3, n, 250, n, n, 17, n, n, n, n, 0], dtype=torch.int32)
+    lcp, dT, parent, shared = ctx.prefix_dedup(tkd, lens.to(dev), logp2)
+    lcp_o, dT_o, par_o, sh_o = orc.prefix_dedup(tokens.numpy(), lens.numpy(), logp2.cpu().numpy())
+    assert np.array_equal(lcp.cpu().numpy(), lcp_o)
+    np.testing.assert_allclose(dT.cpu().numpy(), dT_o, rtol=1e-4, atol=1e-6)
+    assert np.array_equal(parent.cpu().numpy(), par_o) and np.array_equal(shared.cpu().numpy(), sh_o)
+    assert sh_o.max() >= 20                                       # the trie really shares prefixes
+    # d_T(s,s) = -log2 P(s)  (Remark after Def. 2)
+    _, _, _, _, lp_o = orc.topk_softmax(logits.numpy().reshape(-1, V), tokens.numpy().reshape(-1), K)
+    lp_o = lp_o.reshape(S, n)
+    for s in range(S):
+        assert abs(float(dT[s, s]) + lp_o[s, :int(lens[s])].sum()) <= 1e-4 * max(1.0, -lp_o[s, :int(lens[s])].sum())
+    # tail coding with pos_begin = shared_len straight from the device
+    W, mc = ctx.W, ctx.max_chunks(n)
+    st = plc.StreamSet(S * W, mc, 3 * S * n * W * 128 + 4096, dev)
+    kvd = kv.to(dev)
+    ctx.encode(kvd, lgd, st, shared, lens.to(dev))
+    assert ctx.sync_status() == plc.OK
+    coded = int(np.maximum(lens.numpy() - sh_o, 0).sum())
+    assert ctx.stats().coded_vectors == coded * W                  # Prop. 2: the shared prefix costs nothing
+    outkv = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    ctx.decode(st, lgd, outkv, shared, lens.to(dev))
+    assert ctx.sync_status() == plc.OK
+    # a session's prefix is recovered from its parent (Prop. 1(a): identical KV on the common prefix)
+    o = outkv.cpu()
+    for s in range(S):
+        p, m = int(par_o[s]), int(sh_o[s])
+        if p >= 0 and m > 0:
+            assert torch.equal(kv[:, :, s, :, :m], kv[:, :, p, :, :m])
+        e = int(lens[s])
+        if e > m:
+            assert float((o[:, :, s, :, m:e] - kv[:, :, s, :, m:e].float()).abs().max()) <= 0.011
+
+
+def test_append_steps_match_bulk_encode(dev, orc):
+    """Decode-time append: 70 single-token steps with 32-position chunks give, chunk for chunk, the
+    bytes of a bulk encode of the same 70 positions, and decode back."""
+    B, steps, L, H, d, V, K, CP = 3, 70, 1, 2, 128, 512, 32, 32
+    tokens, logits, T, kv = make_workload(41, B, steps, L, H, d, V, K)
+    g = gpu_encode(dev, T, kv, logits, K, 0.02, CP)
+    ctx = g["ctx"]
+    W = ctx.W
+    sb = ctx.new_session_batch(B, 3, 3 * B * steps * W * d + 4096)
+    kvd, lgd = g["kv"], g["logits"]
+    for i in range(steps):
+        kv_step = kvd[:, :, :, :, i, :].contiguous()               # [L][2][B][H][d]
+        ctx.append_step(sb, kv_step, lgd[:, i, :].contiguous())
+    assert sb.c.steps == steps
+    ctx.append_flush(sb)
+    assert ctx.sync_status() == plc.OK
+    for slot in range(B * W * 3):
+        assert np.array_equal(sb.streams.chunk(slot), g["st"].chunk(slot)), slot
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    ctx.decode(sb.streams, lgd, out)
+    assert ctx.sync_status() == plc.OK
+    assert float((out.cpu() - kv.float()).abs().max()) <= 0.011
+
+
+def test_f16_output(dev):
+    tokens, logits, T, kv = make_workload(51, 1, 64, 1, 2, 128, 512, 32)
+    L, _, H, V, d = T.shape
+    ctx = plc.Context(T.to(dev), 32, 0.02, chunk_pos=32, out_dtype=plc.OUT_F16)
+    st = plc.StreamSet(ctx.W, 2, 3 * 64 * ctx.W * d + 4096, dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    ctx.encode(kvd, lgd, st)
+    out = torch.zeros(kv.shape, dtype=torch.float16, device=dev)
+    ctx.decode(st, lgd, out)
+    assert ctx.sync_status() == plc.OK
+    # float16 output adds half an ulp of binary16 (2^-9 relative at most for |x| < 8)
+    assert float((out.float() - kvd.float()).abs().max()) <= 0.01 + 1e-3 + 8 * 2 ** -11

@@ -48,7 +48,7 @@ def test_table_constants_closed_form(orc):
 
 def _py_decode(data, q, d, orc):
     """Independent decoder written from the format's definition (forward word order)."""
-    G = d // 32
+    G, R = d // 32, d // 8
     x = [int.from_bytes(data[4 * l:4 * l + 4].tobytes(), "little") for l in range(32)]
     words = data[128:].view("<u2").astype(np.int64).tolist()
     rp = 0
@@ -77,7 +77,7 @@ def _py_decode(data, q, d, orc):
                     hi = raw - (1 << 32) if raw >= (1 << 31) else raw
                 else:
                     hi = (zzs[l] + 1) // 2 if zzs[l] & 1 else -(zzs[l] // 2)
-                out[p, l * G + g] = hi if s == 0 else (hi << s) + lo[l] - (1 << (s - 1))
+                out[p, 8 * (l % R) + G * (l // R) + g] = hi if s == 0 else (hi << s) + lo[l] - (1 << (s - 1))
     assert rp == len(words) and all(v == 1 << 16 for v in x)
     return out
 
