@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the predictive-delta-coding hot path (encode then decode of one synthetic batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama2-7b] [--impl own|reference]
+
+A step = one pass of the whole path over one batch: top-K softmax, fused predict + quantise + rANS
+encode of every (stream, position), then the decode of the same batch.  The metric is KV tokens per
+second (a KV token = one token position of one session across all 2*L*H streams) that were both
+encoded and decoded.  With N > 1 (torchrun) every rank runs its own batch (streams shard with no
+exchange): weak scaling, value = tokens of all ranks / slowest rank's time.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KV tokens/s encoded+decoded per B200"
+UNIT = "KV tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        cmd = ["nvidia-smi", "-i", uuid, "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "200"]
+        try:
+            self.p = subprocess.Popen(cmd, stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(",") for r in open(self.f.name) if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for nme, v in zip(names, r[3:7]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_rate(w, positions, layers):
+    """Times the CPU oracle (encode + decode) on a slice of the workload: `positions` positions of
+    session 0, `layers` layers, all heads.  Returns KV tokens/s (vectors / W / seconds)."""
+    import oracle
+    cfg = w["cfg"]
+    H, d, V, K = cfg["H"], cfg["d"], cfg["V"], cfg["K"]
+    Tn = w["T"][:layers].cpu().numpy()
+    kvn = w["kv"][:layers, :, :1, :, :positions].cpu().numpy()
+    lgn = w["logits"][:1, :positions].cpu().numpy()
+    ocfg = oracle.Config(layers, H, d, V, K, cfg["delta"], 0.0, cfg["chunk_pos"], 0)
+    t0 = time.perf_counter()
+    enc = oracle.encode(ocfg, Tn, kvn, lgn, None)
+    t1 = time.perf_counter()
+    rc, out, _ = oracle.decode(ocfg, Tn, lgn, enc, kvn.shape)
+    t2 = time.perf_counter()
+    assert rc == 0
+    W_full = 2 * cfg["L"] * H
+    vecs = positions * 2 * layers * H
+    return dict(value=vecs / W_full / (t2 - t0), encode=vecs / W_full / (t1 - t0), decode=vecs / W_full / (t2 - t1),
+                seconds=t2 - t0, bytes=int(enc["stats"].payload_bytes), vectors=vecs)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--chunk-pos", type=int, default=None)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--set", action="append", default=[], help="override a workload field, e.g. --set L=4")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    import torch
+    from paper_2604_15356_b200 import workloads
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args, workloads)
+
+    import paper_2604_15356_b200 as plc
+    plc.build()
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    over = {}
+    for kvs in args.set:
+        k, v = kvs.split("=")
+        over[k] = float(v) if "." in v else int(v)
+    if args.chunk_pos:
+        over["chunk_pos"] = args.chunk_pos
+    w = workloads.build(args.workload, dev, seed=20260415 + 1000 * rank, **over)
+    cfg = w["cfg"]
+    S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
+    W = 2 * L * H
+    ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16)
+    ctx.reserve(S * n)
+    ctx.set_profiling(True)
+    mc = ctx.max_chunks(n)
+    kv_bytes = w["kv"].numel() * 2
+    st = plc.StreamSet(S * W, mc, int(0.70 * kv_bytes) + (1 << 20), dev)
+    out = torch.empty_like(w["kv"])
+    tokens_per_step = S * n
+
+    def step():
+        st.total_bytes.zero_()
+        ctx.encode(w["kv"], w["logits"], st)
+        ctx.decode(st, w["logits"], out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    barrier()
+    assert ctx.sync_status() == plc.OK, "device status after warm-up"
+    ctx.stats(reset=True)
+
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+    launches0 = plc.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * args.steps)]
+    enc_k, dec_k = [], []
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        st.total_bytes.zero_()
+        ev[3 * i].record()
+        ctx.encode(w["kv"], w["logits"], st)
+        ev[3 * i + 1].record()
+        ctx.decode(st, w["logits"], out)
+        ev[3 * i + 2].record()
+        enc_k.append(ctx.last_kernel_ms(0)); dec_k.append(ctx.last_kernel_ms(1))
+    t_end.record()
+    barrier()
+    launches = plc.launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    enc_ms = [ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(args.steps)]
+    dec_ms = [ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(args.steps)]
+    assert ctx.sync_status() == plc.OK, "device status after the timed region"
+    stats = ctx.stats()
+    payload_per_step = stats.payload_bytes / args.steps
+    chunks_per_step = stats.n_chunks / args.steps
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t[0]) / args.steps
+    value = world * tokens_per_step / (ms_per_step / 1e3)
+
+    # spot check of the decoded batch (outside the timed region)
+    sel = torch.randint(0, n, (64,), device=dev)
+    err = float((out[:, :, :, :, sel].float() - w["kv"][:, :, :, :, sel].float()).abs().max())
+    assert err <= cfg["delta"] / 2 + 1e-3 + 8 * 2 ** -11, err
+
+    peak, peak_kind = measured_peaks()
+    vecs = S * n * W
+    ek, dk = statistics.mean(enc_k), statistics.mean(dec_k)
+    gathered = vecs * K * d * 2
+    bytes_ns = vecs * d * 2 + gathered + payload_per_step    # KV + T rows read + bitstream (either direction)
+    bytes_c = vecs * d * 2 + w["T"].numel() * 2 + payload_per_step
+    dom_enc = ek >= dk
+    dom_ms = ek if dom_enc else dk
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
+    fma_ach = vecs * K * d / (dom_ms / 1e3)
+    roofline = {"kernel": "encode_kernel" if dom_enc else "decode_kernel", "bound": "hbm",
+                "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
+                "frac": bytes_ns / (dom_ms / 1e3) / 1e9 / peak, "traffic": None, "peak_kind": peak_kind,
+                "accounting": "KV + gathered T rows (K*d*2 B per vector, mostly served by L2) + bitstream, per launch",
+                "bytes_per_launch": bytes_ns, "ms_per_launch": dom_ms,
+                "compulsory": {"bytes_per_launch": bytes_c, "achieved": bytes_c / (dom_ms / 1e3) / 1e9,
+                               "frac": bytes_c / (dom_ms / 1e3) / 1e9 / peak},
+                "fp32_fma": {"achieved_gfma_s": fma_ach / 1e9, "peak_gfma_s": fma_peak / 1e9, "frac": fma_ach / fma_peak},
+                "encode_kernel_ms": ek, "decode_kernel_ms": dk}
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        layers, pos = min(L, 2), min(n, 256)
+        r = oracle_sample_rate(w, pos, layers)
+        cpu = {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"session 0, first {pos} positions, {layers} of {L} layers, all heads ({r['vectors']} vectors, "
+                         f"{r['seconds']:.1f} s encode+decode); rate scaled by W={W} vectors per KV token",
+               "encode": r["encode"], "decode": r["decode"]}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
+                       "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
+                       "kv_dtype": "f16", "decode_out": "f16",
+                       "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
+            "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
+            "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),
+            "encode_ms": statistics.mean(enc_ms), "decode_ms": statistics.mean(dec_ms),
+            "bits_per_token": 8 * (payload_per_step + 12 * chunks_per_step) / tokens_per_step,
+            "bits_per_component": 8 * payload_per_step / (vecs * d),
+            "paper_bound_bits_per_token": "3.3-4.3 at perplexity 10-20 (Cor. 1: theory for the token stream, not this synthetic KV)",
+            "escapes_per_step": stats.n_escapes / args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step):
+    """Same step with HOST buffers: pinned inputs are copied in, the coded bytes and index are
+    copied out and back in, the decoded KV is copied out -- all inside the timed region."""
+    kv_h = w["kv"].cpu().pin_memory()
+    lg_h = w["logits"].cpu().pin_memory()
+    pay_h = torch.empty(st.payload.numel(), dtype=torch.uint8).pin_memory()
+    off_h = torch.empty_like(st.chunk_offset, device="cpu").pin_memory()
+    nby_h = torch.empty_like(st.chunk_bytes, device="cpu").pin_memory()
+    tot_h = torch.zeros(1, dtype=torch.int64).pin_memory()
+    kvo_h = torch.empty_like(kv_h).pin_memory()
+    kv_d, lg_d = torch.empty_like(w["kv"]), torch.empty_like(w["logits"])
+
+    def step():
+        kv_d.copy_(kv_h, non_blocking=True); lg_d.copy_(lg_h, non_blocking=True)
+        st.total_bytes.zero_()
+        ctx.encode(kv_d, lg_d, st)
+        tot_h.copy_(st.total_bytes, non_blocking=True)
+        torch.cuda.current_stream().synchronize()           # the byte count decides how much to copy out
+        used = int(tot_h[0])
+        pay_h[:used].copy_(st.payload[:used], non_blocking=True)
+        off_h.copy_(st.chunk_offset, non_blocking=True); nby_h.copy_(st.chunk_bytes, non_blocking=True)
+        st.payload[:used].copy_(pay_h[:used], non_blocking=True)
+        st.chunk_offset.copy_(off_h, non_blocking=True); st.chunk_bytes.copy_(nby_h, non_blocking=True)
+        ctx.decode(st, lg_d, out)
+        kvo_h.copy_(out, non_blocking=True)
+        return used
+
+    used = step()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.e2e_steps):
+        used = step()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / args.e2e_steps
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    idx_bytes = off_h.numel() * 8 + nby_h.numel() * 4
+    return {"value": world * tokens_per_step / (float(t[0]) / 1e3), "unit": UNIT, "ms_per_step": float(t[0]),
+            "h2d_bytes_per_step": kv_h.numel() * 2 + lg_h.numel() * 2 + used + idx_bytes,
+            "d2h_bytes_per_step": used + idx_bytes + 8 + kvo_h.numel() * 2, "steps": args.e2e_steps}
+
+
+def reference_arm(args, workloads):
+    """The reference arm is the CPU oracle as it stands, on a bounded sample of the same workload."""
+    cfg = dict(workloads.CONFIGS[args.workload])
+    layers, pos = 1, min(cfg["n"], 64)
+    # the sample is built on the CPU at the sample's own size (same recipe)
+    w = workloads.build(args.workload, "cpu", seed=20260415, S=1, n=pos, L=layers, max_states=64)
+    w["cfg"]["L"] = cfg["L"]                                  # the rate is scaled to the full number of streams
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_rate(w, pos, layers)
+    rates = []
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        rates.append(oracle_sample_rate(w, pos, layers))
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = statistics.mean(r["value"] for r in rates)
+    W = 2 * cfg["L"] * cfg["H"]
+    sample = (f"1 session, {pos} positions, {layers} of {cfg['L']} layers, all heads "
+              f"({rates[0]['vectors']} vectors per step); rate scaled by W={W} vectors per KV token")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

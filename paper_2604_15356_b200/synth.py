@@ -120,6 +120,19 @@ def hashed_normal(keys, stream, d, seed):
     return (torch.sqrt(-2.0 * torch.log(u1)) * torch.cos(2.0 * math.pi * u2)).to(torch.float32)
 
 
+def prefix_keys(tokens):
+    """int64 [S][n] rolling hash of the token prefix x_0..x_i: equal prefixes give equal keys, so KV
+    built from these keys is a function of the token prefix alone."""
+    S, n = tokens.shape
+    keys = torch.empty(S, n, dtype=torch.int64, device=tokens.device)
+    k = torch.zeros(S, dtype=torch.int64, device=tokens.device)
+    tok = tokens.to(torch.int64)
+    for i in range(n):
+        k = _mix64(k * _wrap(0x9E3779B97F4A7C15) + tok[:, i] + 1)
+        keys[:, i] = k
+    return keys
+
+
 def make_kv(T, tokens, sigma, seed, keys=None, out=None):
     """KV [L][2][S][H][n][d] float16 = T[l][kv][h][x_i] + sigma * noise(key[s][i])."""
     L, _, H, V, d = T.shape
@@ -146,7 +159,8 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
     The trie has depth+1 levels (1+2+...+2^depth segments); each segment is Markov-sampled,
     length U[seg_lo, seg_hi]; a session picks one of the 2^depth leaves uniformly, takes that
     root-to-leaf path as its prefix and continues sampling.  Returns tokens int32 [S][n], keys
-    int64 [S][n] (equal on shared prefix positions), leaf [S], prefix_len [S].
+    int64 [S][n] (a hash of the token prefix, so equal exactly where prefixes are equal), leaf [S],
+    prefix_len [S].
     """
     dev = table.device
     g = _gen(seed, "cpu")
@@ -159,7 +173,6 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
         segs[node] = sample_tokens(table, 1, int(seg_len[node]), seed * 1000 + 17 + node, start=start)
     leaf = torch.randint(0, 1 << depth, (S,), generator=g)
     tokens = torch.zeros(S, n, dtype=torch.int32, device=dev)
-    keys = torch.zeros(S, n, dtype=torch.int64, device=dev)
     plen = torch.zeros(S, dtype=torch.int32)
     for s in range(S):
         node = (1 << depth) - 1 + int(leaf[s])
@@ -172,11 +185,9 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
         for nd in path:
             m = min(int(seg_len[nd]), n - pos)
             tokens[s, pos:pos + m] = segs[nd][0, :m]
-            keys[s, pos:pos + m] = (nd + 1) * (1 << 32) + torch.arange(m, device=dev)
             pos += m
         plen[s] = pos
         if pos < n:
             start = tokens[s, pos - 1:pos].to(torch.int64)
             tokens[s, pos:] = sample_tokens(table, 1, n - pos, seed * 1000 + 500 + s, start=start)[0]
-            keys[s, pos:] = (1000 + s) * (1 << 32) + torch.arange(pos, n, device=dev)
-    return tokens, keys, leaf, plen
+    return tokens, prefix_keys(tokens), leaf, plen

@@ -225,12 +225,13 @@ def test_sigma_floor_and_escapes(dev, orc):
     lg = np.full(logits.shape, -40.0, np.float16)
     np.put_along_axis(lg[0], tokens[0].numpy()[:, None].astype(np.int64), np.float16(40.0), axis=1)
     logits = torch.from_numpy(lg)
-    g = gpu_encode(dev, T, kv, logits, 16, 0.005, 32)
+    cap = 9 * 64 * 2 * 128 + 4096                                 # escapes cost up to 8 bytes per component
+    g = gpu_encode(dev, T, kv, logits, 16, 0.005, 32, capacity=cap)
     assert g["rc"] == plc.OK and g["ctx"].stats().n_escapes > 0
     assert np.all(g["q"].cpu().numpy() == -24)
     check_against_oracle(orc, g, T, kv, logits, 16, 0.005, 32)
     gpu_decode_check(g, kv, 0.005, 64)
-    g2 = gpu_encode(dev, T, kv, logits, 16, 0.005, 32, sigma_floor=0.3)
+    g2 = gpu_encode(dev, T, kv, logits, 16, 0.005, 32, sigma_floor=0.3, capacity=cap)
     assert g2["ctx"].stats().n_escapes < g["ctx"].stats().n_escapes
     check_against_oracle(orc, g2, T, kv, logits, 16, 0.005, 32, sigma_floor=0.3)
 
