@@ -177,6 +177,29 @@ plc_status plc_append_flush(plc_ctx* ctx, plc_session_batch* sb, void* stream);
 /* Bytes of open_sym_dev / open_q_dev for B sessions. */
 plc_status plc_append_sizes(const plc_ctx* ctx, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes);
 
+/* Entropy-codes one chunk per stream from symbols and classes that are already on the device,
+ * without allocating anything.  (The paper has no counterpart for this call: it exists for callers
+ * that are not allowed to allocate device memory at the point where they seal a chunk -- code that
+ * runs inside a serving loop with a frozen memory pool, inside a memory-budgeted plugin, or after
+ * start-up in a process whose allocator is locked down -- and that therefore cannot own a plc_ctx,
+ * whose creation allocates.)  The bitstream is exactly the one plc_append_step / plc_append_flush
+ * write for the same symbols and classes.
+ *   sym_dev [n_streams][chunk_capacity][head_dim] int32, q_dev [n_streams][chunk_capacity] int32:
+ *   the first n_pos positions of every stream are coded (the layout of plc_session_batch's open
+ *   chunk, with n_streams = B*W); classes outside [-24, 135] are clamped and reported.
+ *   Chunk `chunk_index` of stream i goes to index slot i*out->max_chunks + chunk_index.
+ *   status_dev: one device word, an OUTPUT: 0, or a bit-or of 1 (payload capacity exceeded; nothing
+ *   is written past it and *total_bytes_dev holds the size needed) and 4 (a class was out of range).
+ * Limits: n_pos * head_dim <= 4096 components per chunk (PLC_E_SHAPE beyond that); head_dim in
+ * {32, 64, 128, 256}.  All working memory is one static device array of about 8 MiB that every GPU
+ * using the library holds until the process exits.  Every call on a device shares that array, so
+ * two calls whose kernels could overlap on the GPU (different streams, no ordering) race with each
+ * other: order them.  The first call on each device looks up the array's device address (with that
+ * device current); make that first call before starting any stream capture. */
+plc_status plc_rans_encode_static(const int32_t* sym_dev, const int32_t* q_dev, int32_t n_streams, int32_t n_pos,
+                                  int32_t head_dim, int32_t chunk_capacity, int32_t chunk_index,
+                                  const plc_streams* out, uint32_t* status_dev, void* stream);
+
 /* Waits for the stream and returns the device status word's most severe code; clears it. */
 plc_status plc_sync_status(plc_ctx* ctx, void* stream);
 /* Waits for the stream, copies the counters, optionally clears them. */

@@ -21,7 +21,7 @@ OUT_F32, OUT_F16 = 0, 1
 EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_prefix_dedup", "plc_encode",
            "plc_decode", "plc_append_step", "plc_append_flush", "plc_append_sizes", "plc_sync_status",
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
-           "plc_launch_count"]
+           "plc_launch_count", "plc_rans_encode_static"]
 
 
 def sources():
@@ -248,6 +248,18 @@ class Context:
 
 class AppendBatch:
     """Python-side holder of a plc_session_batch and the tensors it points to."""
+
+
+def rans_encode_static(sym, q, n_pos, chunk_index, streams, status):
+    """Codes chunk ``chunk_index`` of every stream from symbols / classes on the device, using only
+    the library's static working memory (no allocation inside the call).
+
+    sym [n_streams][chunk_capacity][d] int32, q [n_streams][chunk_capacity] int32, status: one int32
+    device word that receives 0 or the error bits.  Returns the plc_status of the host-side checks."""
+    n_streams, cap, d = sym.shape
+    st = streams.c()
+    return lib().plc_rans_encode_static(_ptr(sym), _ptr(q), n_streams, int(n_pos), d, cap, int(chunk_index),
+                                        C.byref(st), _ptr(status), _stream())
 
 
 def table_constants(qp):
