@@ -216,13 +216,17 @@ void plo_class_params(int q, int* s, int* qp) {
 /* ---------------------------------------------------------------- quantiser */
 
 /* Def. 6 then a uniform mid-tread quantiser of step delta, no clamping below 2^30.
- * The rounding decision is taken in binary32: mu is rounded to float, r = kv - mu, t = r / delta,
- * sym = nearest integer (ties to even). */
+ * The rounding decision is taken in binary32: mu is rounded to float, r = kv - mu,
+ * t = r * (1/delta) with the reciprocal itself rounded to binary32 once, sym = nearest integer
+ * (ties to even).  (The paper fixes no quantiser arithmetic, Prop. 3: "any per-vector quantizer";
+ * a scaled multiply is the usual form of a uniform quantiser and keeps |KV' - KV| <= delta/2 up
+ * to one part in 2^23 of the residual.) */
 void plo_quantise(const uint16_t* kv, const double* mu, int d, float delta, int32_t* sym) {
     for (int j = 0; j < d; ++j) {
         float muf = (float)mu[j];
         float r = (float)half_to_double(kv[j]) - muf;
-        float t = r / delta;
+        float inv = 1.0f / delta;
+        float t = r * inv;
         float n = nearbyintf(t);
         if (n > (float)SYM_LIMIT) n = (float)SYM_LIMIT;
         if (n < -(float)SYM_LIMIT) n = -(float)SYM_LIMIT;

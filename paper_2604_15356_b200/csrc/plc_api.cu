@@ -50,11 +50,16 @@ plc_status check_streams(const plc_streams* s, int need_chunks) {
     return PLC_OK;
 }
 
+int padded_k(const plc_config& cfg) {
+    const int rows = 256 / cfg.head_dim;      // rows of T that one warp-wide 16-byte-per-lane load fetches
+    return (cfg.top_k + rows - 1) / rows * rows;
+}
+
 plc_status ensure_pairs(plc_ctx* c, long long positions) {
     if (positions <= c->pairs_cap) return PLC_OK;
     if (c->pairs) cudaFree(c->pairs);
     c->pairs = nullptr; c->pairs_cap = 0;
-    if (cudaMalloc(&c->pairs, sizeof(int2) * (size_t)positions * c->cfg.top_k) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaMalloc(&c->pairs, sizeof(int2) * (size_t)positions * padded_k(c->cfg)) != cudaSuccess) return PLC_E_CUDA;
     c->pairs_cap = positions;
     return PLC_OK;
 }
@@ -62,7 +67,7 @@ plc_status ensure_pairs(plc_ctx* c, long long positions) {
 CodecArgs base_args(const plc_ctx* c) {
     CodecArgs a{};
     a.sh.L = c->cfg.n_layers; a.sh.H = c->cfg.n_kv_heads; a.sh.d = c->cfg.head_dim; a.sh.V = c->cfg.vocab;
-    a.sh.K = c->cfg.top_k; a.sh.chunk_pos = c->cfg.chunk_pos; a.sh.out_dtype = c->cfg.out_dtype;
+    a.sh.K = c->cfg.top_k; a.sh.Kp = padded_k(c->cfg); a.sh.chunk_pos = c->cfg.chunk_pos; a.sh.out_dtype = c->cfg.out_dtype;
     a.sh.delta = c->cfg.delta; a.sh.sigma_floor = c->cfg.sigma_floor;
     a.T = c->T; a.rownorm2 = c->rownorm2; a.pairs = c->pairs;
     a.staging = c->staging; a.staging_words_per_warp = c->staging_words_per_warp;
@@ -162,7 +167,7 @@ static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n,
     if (rc) return rc;
     TopkArgs a{};
     a.logits = static_cast<const __half*>(logits_dev); a.N = (long long)S * n; a.V = c->cfg.vocab; a.K = c->cfg.top_k;
-    a.pairs = c->pairs; a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
+    a.pairs = c->pairs; a.Kp = padded_k(c->cfg); a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
     return launch_topk(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 

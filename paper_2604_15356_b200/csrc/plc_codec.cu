@@ -89,30 +89,38 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const __half* __restrict__
     }
 }
 
-// Mixture of one position for one table.  pairs: the position's K {idx, w} entries.
+// Two binary32 fused multiply-adds in one instruction (sm_100 packed f32x2); each half is an
+// IEEE fma, so the result equals two scalar __fmaf_rn.
+__device__ __forceinline__ void ffma2(float& a0, float& a1, float w, float x0, float x1) {
+    asm("{ .reg .b64 ra, rb, rc;\n mov.b64 ra, {%2,%2};\n mov.b64 rb, {%3,%4};\n mov.b64 rc, {%0,%1};\n"
+        " fma.rn.f32x2 rc, ra, rb, rc;\n mov.b64 {%0,%1}, rc; }"
+        : "+f"(a0), "+f"(a1) : "f"(w), "f"(x0), "f"(x1));
+}
+
+// Mixture of one position for one table.  pairs: the position's Kp {idx, w} entries, Kp = K rounded
+// up to a multiple of ROWS (the padding has weight 0 and a valid index).
 template <int D>
 __device__ __forceinline__ void predict(const __half* __restrict__ table, const float* __restrict__ n2,
-                                        const int2* __restrict__ pairs, int K, int lane, float inv_d,
+                                        const int2* __restrict__ pairs, int Kp, int lane, float inv_d,
                                         float (&mu)[Geo<D>::G], float& sigma2) {
     constexpr int R = Geo<D>::R, G = Geo<D>::G, ROWS = Geo<D>::ROWS;
     const int m = lane % R, h = lane / R;
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    const __half* col = table + 8 * m;
-#pragma unroll 4
-    for (int k0 = 0; k0 < K; k0 += ROWS) {
-        int k = k0 + h;
-        bool ok = k < K;
-        int2 pr = __ldg(pairs + (ok ? k : 0));
-        float w = ok ? __int_as_float(pr.y) : 0.f;
-        uint4 r = __ldg(reinterpret_cast<const uint4*>(col + (size_t)pr.x * D));
+    const char* col = reinterpret_cast<const char*>(table + 8 * m);
+    const int2* pl = pairs + h;
+    const int iters = Kp / ROWS;
+#pragma unroll 8
+    for (int it = 0; it < iters; ++it) {
+        const int2 pr = __ldg(pl + it * ROWS);
+        const float w = __int_as_float(pr.y);
+        const uint4 r = __ldg(reinterpret_cast<const uint4*>(col + (long long)pr.x * (D * 2)));
         const __half2* hp = reinterpret_cast<const __half2*>(&r);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            float2 f = __half22float2(hp[j]);
-            acc[2 * j] = __fmaf_rn(w, f.x, acc[2 * j]);
-            acc[2 * j + 1] = __fmaf_rn(w, f.y, acc[2 * j + 1]);
+            const float2 f = __half22float2(hp[j]);
+            ffma2(acc[2 * j], acc[2 * j + 1], w, f.x, f.y);
         }
     }
     // reduce-scatter over the ROWS lanes that hold partial sums of the same 8 components
@@ -135,7 +143,7 @@ __device__ __forceinline__ void predict(const __half* __restrict__ table, const 
     for (int g = 0; g < G; ++g) mu[g] = acc[g];
     // variance: (sum_k w_k ||T_k||^2 - ||mu||^2) / d
     float s1 = 0.f;
-    for (int k = lane; k < K; k += 32) {
+    for (int k = lane; k < Kp; k += 32) {
         int2 pr = __ldg(pairs + k);
         s1 = __fmaf_rn(__int_as_float(pr.y), __ldg(n2 + pr.x), s1);
     }
@@ -367,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     uint16_t* stage = a.staging + gw * a.staging_words_per_warp;
     const int cap_words = (int)a.staging_words_per_warp;
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
     const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wt * a.S * a.st.max_chunks;
     const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
@@ -442,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const uint32_t lt = lanemask_lt();
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
     const unsigned total = (unsigned)Wt * a.S * a.st.max_chunks;
     const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
@@ -502,7 +510,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     const int lane = threadIdx.x & 31;
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.K;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
     const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const long long nw = (long long)gridDim.x * kWarpsPerBlock;
     const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;

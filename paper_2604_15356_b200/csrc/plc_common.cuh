@@ -148,7 +148,8 @@ void count_launch(int n = 1);
 // Internal launchers (one per .cu file).
 struct TopkArgs {
     const __half* logits; const int32_t* tokens; int64_t N; int V, K;
-    int2* pairs;            // [N][K] {idx, float bits of w}, or null
+    int2* pairs;            // [N][Kp] {idx, float bits of w}, or null; entries K..Kp-1 get {idx_0, 0}
+    int Kp;
     int32_t* idx; float* w; float* lse; float* zk; float* logp2;   // optional user outputs
     // Rows are skipped (nothing written) when pos ranges are given and the row is outside them.
     int n_per_session; const int32_t* pos_begin; const int32_t* pos_end;
@@ -159,7 +160,7 @@ cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, cons
                                 int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st);
 
 struct CodecShape {
-    int L, H, d, V, K, chunk_pos, out_dtype;
+    int L, H, d, V, K, Kp, chunk_pos, out_dtype;   // Kp: K rounded up to the rows one warp-wide load fetches
     float delta, sigma_floor;
 };
 

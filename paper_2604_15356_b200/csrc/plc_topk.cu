@@ -259,10 +259,12 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
         for (int k = tid; k < K; k += kThreads) {
             float w = sm.ek[k] / sum_k;
             int idx = sm.cand_idx[k];
-            if (a.pairs) a.pairs[rowi * K + k] = make_int2(idx, __float_as_int(w));
+            if (a.pairs) a.pairs[rowi * a.Kp + k] = make_int2(idx, __float_as_int(w));
             if (a.idx) a.idx[rowi * K + k] = idx;
             if (a.w) a.w[rowi * K + k] = w;
         }
+        if (a.pairs)
+            for (int k = K + tid; k < a.Kp; k += kThreads) a.pairs[rowi * a.Kp + k] = make_int2(sm.cand_idx[0], 0);
         if (tid == 0) {
             float lse = lmax + logf(sum_all);
             if (a.lse) a.lse[rowi] = lse;
