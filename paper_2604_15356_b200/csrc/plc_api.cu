@@ -69,6 +69,8 @@ CodecArgs base_args(const plc_ctx* c) {
     a.sh.L = c->cfg.n_layers; a.sh.H = c->cfg.n_kv_heads; a.sh.d = c->cfg.head_dim; a.sh.V = c->cfg.vocab;
     a.sh.K = c->cfg.top_k; a.sh.Kp = padded_k(c->cfg); a.sh.chunk_pos = c->cfg.chunk_pos; a.sh.out_dtype = c->cfg.out_dtype;
     a.sh.delta = c->cfg.delta; a.sh.sigma_floor = c->cfg.sigma_floor;
+    a.sh.inv_delta = 1.0f / c->cfg.delta;
+    a.sh.inv_delta2 = (float)(1.0 / ((double)c->cfg.delta * (double)c->cfg.delta));
     a.T = c->T; a.rownorm2 = c->rownorm2; a.pairs = c->pairs;
     a.staging = c->staging; a.staging_words_per_warp = c->staging_words_per_warp;
     a.ticket = c->ticket; a.status = c->status; a.counters = c->counters;

@@ -19,9 +19,16 @@
 namespace plc {
 namespace {
 
+#ifndef PLC_BLOCKS_PER_SM
+#define PLC_BLOCKS_PER_SM 5
+#endif
+#ifndef PLC_GATHER_UNROLL
+#define PLC_GATHER_UNROLL 8
+#endif
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
-constexpr int kBlocksPerSM = 4;
+constexpr int kBlocksPerSM = PLC_BLOCKS_PER_SM;
+constexpr int kGatherUnroll = PLC_GATHER_UNROLL;
 
 template <int D>
 struct Geo {
@@ -31,7 +38,8 @@ struct Geo {
 };
 
 struct EncTables { EncEntry enc[kNumTables][kNumSym]; };
-struct DecTables { uint16_t cum[kNumTables][kNumSym + 2]; };
+// Decoder tables: cum[] for the search, fc[] = f | (c << 16) for the state update.
+struct DecTables { uint16_t cum[kNumTables][kNumSym + 2]; uint32_t fc[kNumTables][kNumSym]; };
 
 __device__ inline void build_enc_tables(EncTables* t) {
     for (int id = threadIdx.x; id < kNumTables; id += blockDim.x) {
@@ -51,7 +59,11 @@ __device__ inline void build_dec_tables(DecTables* t) {
         uint32_t f[kNumSym];
         build_freqs(id + kQMin, f);
         uint32_t c = 0;
-        for (int i = 0; i < kNumSym; ++i) { t->cum[id][i] = (uint16_t)c; c += f[i]; }
+        for (int i = 0; i < kNumSym; ++i) {
+            t->cum[id][i] = (uint16_t)c;
+            t->fc[id][i] = f[i] | (c << 16);
+            c += f[i];
+        }
         t->cum[id][kNumSym] = (uint16_t)c;
         t->cum[id][kNumSym + 1] = 0xffff;
     }
@@ -97,23 +109,28 @@ __device__ __forceinline__ void ffma2(float& a0, float& a1, float w, float x0, f
         : "+f"(a0), "+f"(a1) : "f"(w), "f"(x0), "f"(x1));
 }
 
-// Mixture of one position for one table.  pairs: the position's Kp {idx, w} entries, Kp = K rounded
-// up to a multiple of ROWS (the padding has weight 0 and a valid index).
+// Mixture of one position for one table.  sp: the position's Kp {idx, w} entries in shared memory,
+// Kp = K rounded up to a multiple of ROWS (the padding has weight 0 and a valid index).
 template <int D>
-__device__ __forceinline__ void predict(const __half* __restrict__ table, const float* __restrict__ n2,
-                                        const int2* __restrict__ pairs, int Kp, int lane, float inv_d,
+__device__ __forceinline__ void predict(const char* __restrict__ col, const float* __restrict__ n2,
+                                        const int2* sp, int Kp, int lane, float inv_d,
                                         float (&mu)[Geo<D>::G], float& sigma2) {
     constexpr int R = Geo<D>::R, G = Geo<D>::G, ROWS = Geo<D>::ROWS;
-    const int m = lane % R, h = lane / R;
+    const int h = lane / R;
+    // variance term first: its row-norm loads are in flight while the rows are gathered
+    float s1 = 0.f;
+    for (int k = lane; k < Kp; k += 32) {
+        const int2 pr = sp[k];
+        s1 = __fmaf_rn(__int_as_float(pr.y), __ldg(n2 + pr.x), s1);
+    }
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    const char* col = reinterpret_cast<const char*>(table + 8 * m);
-    const int2* pl = pairs + h;
+    const int2* pl = sp + h;
     const int iters = Kp / ROWS;
-#pragma unroll 8
+#pragma unroll kGatherUnroll
     for (int it = 0; it < iters; ++it) {
-        const int2 pr = __ldg(pl + it * ROWS);
+        const int2 pr = pl[it * ROWS];
         const float w = __int_as_float(pr.y);
         const uint4 r = __ldg(reinterpret_cast<const uint4*>(col + (long long)pr.x * (D * 2)));
         const __half2* hp = reinterpret_cast<const __half2*>(&r);
@@ -142,119 +159,148 @@ __device__ __forceinline__ void predict(const __half* __restrict__ table, const 
 #pragma unroll
     for (int g = 0; g < G; ++g) mu[g] = acc[g];
     // variance: (sum_k w_k ||T_k||^2 - ||mu||^2) / d
-    float s1 = 0.f;
-    for (int k = lane; k < Kp; k += 32) {
-        int2 pr = __ldg(pairs + k);
-        s1 = __fmaf_rn(__int_as_float(pr.y), __ldg(n2 + pr.x), s1);
-    }
     s1 = warp_sum(s1);
     float s2 = warp_norm2<G>(mu);
     sigma2 = fmaxf(0.f, (s1 - s2) * inv_d);
 }
 
-__device__ __forceinline__ int scale_class(float sigma2, float floor2, float delta2) {
-    return class_from_v(__fdiv_rn(sigma2 + floor2, delta2));
+// The pairs of a position are brought into the warp's shared-memory slot with cp.async, one
+// position ahead of their use and without passing through registers (two slots per warp).
+__device__ __forceinline__ void prefetch_pairs(int2* sp, const int2* __restrict__ gp, int Kp, int lane) {
+    for (int k = lane; k < Kp; k += 32) {
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(sp + k);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(gp + k) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+// Waits for this lane's copies (all but the newest `pending` groups), then makes the whole warp's
+// copies visible to every lane.
+template <int PENDING>
+__device__ __forceinline__ void pairs_ready() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+    __syncwarp();
 }
 
-__device__ __forceinline__ void split_sym(int sym, int s, int& hi, uint32_t& lo) {
-    if (s == 0) { hi = sym; lo = 0; return; }
-    int u = sym + (1 << (s - 1));          // |sym| <= 2^30, s <= 15: no overflow
-    hi = u >> s;
-    lo = (uint32_t)u & ((1u << s) - 1u);
+__device__ __forceinline__ int scale_class(float sigma2, float floor2, float inv_delta2) {
+    return class_from_v((sigma2 + floor2) * inv_delta2);
 }
+
 __device__ __forceinline__ int join_sym(int hi, uint32_t lo, int s) {
     if (s == 0) return hi;
     return (int)(((uint32_t)hi << s) + lo - (1u << (s - 1)));
 }
 
-// One encoder step for the warp: every lane codes `sym` under (s, table tid).  Words are written
-// back to front at stage[wp-1], stage[wp-2], ...; returns the new wp.
-__device__ __forceinline__ int encode_step(int sym, int s, const EncEntry* __restrict__ tbl, uint32_t& x,
+// Values that are the same for all components of one position.
+struct PosCode {
+    int s;               // bit planes
+    uint32_t half;       // 2^(s-1), 0 when s = 0
+    uint32_t lomask;     // 2^s - 1
+};
+__device__ __forceinline__ PosCode pos_code(int s) {
+    PosCode pc;
+    pc.s = s;
+    pc.half = s ? (1u << (s - 1)) : 0u;
+    pc.lomask = (1u << s) - 1u;
+    return pc;
+}
+
+// One encoder step for the warp: every lane codes `sym`.  Words are written back to front at
+// stage[wp-1], stage[wp-2], ...; returns the new wp.
+__device__ __forceinline__ int encode_step(int sym, const PosCode pc, const EncEntry* tbl, uint32_t& x,
                                            uint16_t* __restrict__ stage, int wp, int lane, uint32_t lt,
                                            unsigned& n_escapes) {
-    int hi; uint32_t lo;
-    split_sym(sym, s, hi, lo);
-    const bool esc = hi > kHiMax || hi < -kHiMax;
-    const int zz = esc ? kEsc : (hi > 0 ? 2 * hi - 1 : -2 * hi);
+    const int u = sym + (int)pc.half;              // |sym| <= 2^30, s <= 15: no overflow
+    const int hi = u >> pc.s;
+    const uint32_t lo = (uint32_t)u & pc.lomask;
+    const bool esc = (uint32_t)(hi + kHiMax) > 2u * kHiMax;
+    const int nh = -hi;
+    const int zz = esc ? kEsc : ((nh << 1) ^ (nh >> 31));     // 0, +1 -> 1, -1 -> 2, +2 -> 3, ...
     const EncEntry e = tbl[zz];
     const uint32_t f = e.fc & 0xffffu, c = e.fc >> 16;
     const bool emit = x >= (f << 17);
-    const uint32_t emask = __ballot_sync(kFull, emit), xmask = __ballot_sync(kFull, esc);
-    const int n_emit = __popc(emask), n_esc = __popc(xmask);
-    const int base = wp - (2 * s + n_emit + 2 * n_esc);
-    if (xmask) {
+    const uint32_t emask = __ballot_sync(kFull, emit);
+    const int s2 = 2 * pc.s;
+    int base = wp - s2 - __popc(emask);
+    if (__any_sync(kFull, esc)) {                  // rare: raw 32-bit hi of the escaped lanes
+        const uint32_t xmask = __ballot_sync(kFull, esc);
+        const int n_esc = __popc(xmask);
+        base -= 2 * n_esc;
         if (esc) {
-            int at = base + 2 * s + n_emit + 2 * __popc(xmask & lt);
+            const int at = base + s2 + __popc(emask) + 2 * __popc(xmask & lt);
             stage[at] = (uint16_t)((uint32_t)hi & 0xffffu);
             stage[at + 1] = (uint16_t)((uint32_t)hi >> 16);
         }
         n_escapes += n_esc;
     }
     if (emit) {
-        stage[base + 2 * s + __popc(emask & lt)] = (uint16_t)(x & 0xffffu);
+        stage[base + s2 + __popc(emask & lt)] = (uint16_t)(x & 0xffffu);
         x >>= 16;
     }
     uint32_t q = __umulhi(x, e.rcp);
     uint32_t r = x - q * f;
     if (r >= f) { ++q; r -= f; }
     x = (q << kProbBits) + r + c;
-    if (s) {
+    if (pc.s) {
         uint32_t mine = 0;
-        for (int b = 0; b < s; ++b) {
-            uint32_t plane = __ballot_sync(kFull, (lo >> b) & 1u);
-            if ((lane >> 1) == b) mine = plane;
+        const int myb = lane >> 1;
+        for (int b = 0; b < pc.s; ++b) {
+            const uint32_t plane = __ballot_sync(kFull, (lo >> b) & 1u);
+            if (myb == b) mine = plane;
         }
-        if (lane < 2 * s) stage[base + lane] = (uint16_t)((lane & 1) ? (mine >> 16) : (mine & 0xffffu));
+        if (lane < s2) stage[base + lane] = (uint16_t)((lane & 1) ? (mine >> 16) : mine);
     }
     return base;
 }
 
-// One decoder step for the warp; words[rp...] with rp < nwords are readable.
-__device__ __forceinline__ int decode_step(int s, const uint16_t* __restrict__ cum, uint32_t& x,
+// One decoder step for the warp; words[0 .. nwords) are readable.
+__device__ __forceinline__ int decode_step(const PosCode pc, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
                                            const uint16_t* __restrict__ words, int& rp, int nwords, int lane,
                                            uint32_t lt, bool& bad) {
     uint32_t lo = 0;
-    if (s) {
+    if (pc.s) {
+        const int s2 = 2 * pc.s;
         uint32_t v = 0;
-        if (lane < 2 * s) {
-            int at = rp + lane;
+        if (lane < s2) {
+            const int at = rp + lane;
             if (at < nwords) v = __ldg(words + at); else bad = true;
         }
-        for (int b = 0; b < s; ++b) {
-            uint32_t plane = __shfl_sync(kFull, v, 2 * b) | (__shfl_sync(kFull, v, 2 * b + 1) << 16);
-            lo |= ((plane >> lane) & 1u) << b;
+        const int hs = lane >> 4, sh = lane & 15;    // which half of the plane word, which bit of it
+        for (int b = 0; b < pc.s; ++b) {
+            const uint32_t hw = __shfl_sync(kFull, v, 2 * b + hs);
+            lo |= ((hw >> sh) & 1u) << b;
         }
-        rp += 2 * s;
+        rp += s2;
     }
     const uint32_t slot = x & (kProbM - 1u);
     int zz = 0;
 #pragma unroll
     for (int step = 32; step > 0; step >>= 1)
         if (cum[zz + step] <= slot) zz += step;
-    const uint32_t c = cum[zz], f = (uint32_t)cum[zz + 1] - c;
+    const uint32_t fc = fcs[zz];
+    const uint32_t f = fc & 0xffffu, c = fc >> 16;
     x = f * (x >> kProbBits) + slot - c;
     const bool need = x < kRansL;
     const uint32_t nmask = __ballot_sync(kFull, need);
     if (need) {
-        int at = rp + __popc(nmask & lt);
+        const int at = rp + __popc(nmask & lt);
         uint32_t w = 0;
         if (at < nwords) w = __ldg(words + at); else bad = true;
         x = (x << 16) | w;
     }
     rp += __popc(nmask);
     const bool esc = zz == kEsc;
-    const uint32_t xmask = __ballot_sync(kFull, esc);
     int hi = (zz & 1) ? (zz + 1) >> 1 : -(zz >> 1);
-    if (xmask) {
+    if (__any_sync(kFull, esc)) {
+        const uint32_t xmask = __ballot_sync(kFull, esc);
         if (esc) {
-            int at = rp + 2 * __popc(xmask & lt);
+            const int at = rp + 2 * __popc(xmask & lt);
             uint32_t a = 0, b = 0;
             if (at + 1 < nwords) { a = __ldg(words + at); b = __ldg(words + at + 1); } else bad = true;
             hi = (int)(a | (b << 16));
         }
         rp += 2 * __popc(xmask);
     }
-    return join_sym(hi, lo, s);
+    return join_sym(hi, lo, pc.s);
 }
 
 __device__ __forceinline__ unsigned next_ticket(unsigned int* ticket, int lane) {
@@ -364,6 +410,15 @@ __device__ __forceinline__ void commit_chunk(const CodecArgs& a, long long slot,
     for (int i = lane; i < n_words; i += 32) dw[i] = __ldcg(stage + wp + i);
 }
 
+// Quantiser decision in binary32: sym = rint((kv - mu) * fl(1/delta)), clamped to +-2^30.
+__device__ __forceinline__ int quantise(float kv, float mu, float inv_delta) {
+    float n = rintf(__fmul_rn(__fsub_rn(kv, mu), inv_delta));
+    n = fminf(fmaxf(n, -(float)kSymLimit), (float)kSymLimit);
+    return (int)n;
+}
+
+extern __shared__ int2 g_pair_smem[];   // per warp: two slots of Kp entries
+
 template <int D, bool FROM_OPEN>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
@@ -375,9 +430,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     uint16_t* stage = a.staging + gw * a.staging_words_per_warp;
     const int cap_words = (int)a.staging_words_per_warp;
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
+    int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
     const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wt * a.S * a.st.max_chunks;
-    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const float inv_d = 1.0f / D, inv_delta = a.sh.inv_delta, inv_delta2 = a.sh.inv_delta2,
+                floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
 
     for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
@@ -393,11 +450,20 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             if (lane == 0 && !FROM_OPEN) { a.st.chunk_offset[it.slot] = 0; a.st.chunk_bytes[it.slot] = 0; }
             continue;
         }
-        const __half* table = a.T + (size_t)it.t * a.sh.V * D;
+        const char* col = reinterpret_cast<const char*>(a.T + (size_t)it.t * a.sh.V * D + 8 * (lane % Geo<D>::R));
         const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
         uint32_t x = kRansL;
         int wp = cap_words;
         unsigned n_escapes = 0;
+        const int2* gp = nullptr;
+        const __half* kvp = nullptr;
+        int buf = 0;
+        if (!FROM_OPEN) {
+            gp = a.pairs + ((long long)it.s * a.n + it.p0 + it.P - 1) * Kp;      // last position first
+            __syncwarp();                                                        // slot 0 is free again
+            prefetch_pairs(sp0, gp, Kp, lane);
+            kvp = reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, it.t, H, it.s, it.p0 + it.P - 1) + c0;
+        }
         for (int p = it.P - 1; p >= 0; --p) {
             int sym[G];
             int q;
@@ -407,22 +473,26 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
 #pragma unroll
                 for (int g = 0; g < G; ++g) sym[g] = a.open_sym[o * D + c0 + g];
             } else {
-                const int pos = it.p0 + p;
-                const long long row = (long long)it.s * a.n + pos;
-                float mu[G], sigma2;
-                predict<D>(table, n2, a.pairs + row * K, K, lane, inv_d, mu, sigma2);
-                q = scale_class(sigma2, floor2, delta2);
-                float kvv[G];
-                load_half_vec<G>(reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, it.t, H, it.s, pos) + c0, kvv);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float r = __fsub_rn(kvv[g], mu[g]);
-                    float n = rintf(__fdiv_rn(r, delta));
-                    n = fminf(fmaxf(n, -(float)kSymLimit), (float)kSymLimit);
-                    sym[g] = (int)n;
+                const int2* sp = sp0 + buf * Kp;
+                if (p > 0) {                                                      // one position ahead
+                    gp -= Kp;
+                    prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
+                    pairs_ready<1>();
+                } else {
+                    pairs_ready<0>();
                 }
+                buf ^= 1;
+                float mu[G], sigma2;
+                predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+                q = scale_class(sigma2, floor2, inv_delta2);
+                float kvv[G];
+                load_half_vec<G>(kvp, kvv);
+                kvp -= a.kv.sp;
+#pragma unroll
+                for (int g = 0; g < G; ++g) sym[g] = quantise(kvv[g], mu[g], inv_delta);
+                __syncwarp();                                                     // readers of this slot are done
                 if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
-                    const long long o = row * Wt + it.t;
+                    const long long o = ((long long)it.s * a.n + it.p0 + p) * Wt + it.t;
                     if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
@@ -433,9 +503,10 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             }
             int s, qp;
             class_params(q, s, qp);
+            const PosCode pc = pos_code(s);
             const EncEntry* tbl = tb.enc[qp - kQMin];
 #pragma unroll
-            for (int g = G - 1; g >= 0; --g) wp = encode_step(sym[g], s, tbl, x, stage, wp, lane, lt, n_escapes);
+            for (int g = G - 1; g >= 0; --g) wp = encode_step(sym[g], pc, tbl, x, stage, wp, lane, lt, n_escapes);
         }
         commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes);
         __syncwarp();
@@ -450,9 +521,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const uint32_t lt = lanemask_lt();
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
+    int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
     const unsigned total = (unsigned)Wt * a.S * a.st.max_chunks;
-    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const float inv_d = 1.0f / D, delta = a.sh.delta, inv_delta2 = a.sh.inv_delta2,
+                floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
 
     for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
@@ -470,27 +543,43 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
         const uint16_t* words = reinterpret_cast<const uint16_t*>(src + 128);
         const int nwords = (int)((nbytes - 128u) >> 1);
         int rp = 0;
-        const __half* table = a.T + (size_t)it.t * a.sh.V * D;
+        const char* col = reinterpret_cast<const char*>(a.T + (size_t)it.t * a.sh.V * D + 8 * (lane % Geo<D>::R));
         const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
+        const int2* gp = a.pairs + ((long long)it.s * a.n + it.p0) * Kp;
+        __syncwarp();
+        prefetch_pairs(sp0, gp, Kp, lane);
+        int buf = 0;
+        long long kvo = kv_elem(a.kv, it.t, H, it.s, it.p0) + c0;
         for (int p = 0; p < it.P; ++p) {
-            const int pos = it.p0 + p;
-            const long long row = (long long)it.s * a.n + pos;
+            const int2* sp = sp0 + buf * Kp;
+            if (p + 1 < it.P) {
+                gp += Kp;
+                prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
+                pairs_ready<1>();
+            } else {
+                pairs_ready<0>();
+            }
+            buf ^= 1;
             float mu[G], sigma2;
-            predict<D>(table, n2, a.pairs + row * K, K, lane, inv_d, mu, sigma2);
-            const int q = scale_class(sigma2, floor2, delta2);
+            predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+            const int q = scale_class(sigma2, floor2, inv_delta2);
+            __syncwarp();                                                         // readers of this slot are done
             int s, qp;
             class_params(q, s, qp);
+            const PosCode pc = pos_code(s);
             const uint16_t* cum = tb.cum[qp - kQMin];
+            const uint32_t* fcs = tb.fc[qp - kQMin];
             int sym[G];
             float out[G];
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                sym[g] = decode_step(s, cum, x, words, rp, nwords, lane, lt, bad);
+                sym[g] = decode_step(pc, cum, fcs, x, words, rp, nwords, lane, lt, bad);
                 out[g] = __fmaf_rn((float)sym[g], delta, mu[g]);
             }
-            store_vec<G>(a.kv.base, kv_elem(a.kv, it.t, H, it.s, pos) + c0, out, a.sh.out_dtype);
+            store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
+            kvo += a.kv.sp;
             if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
-                const long long o = row * Wt + it.t;
+                const long long o = ((long long)it.s * a.n + it.p0 + p) * Wt + it.t;
                 if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
@@ -510,28 +599,29 @@ template <int D>
 __global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     const int lane = threadIdx.x & 31;
-    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, K = a.sh.Kp;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
+    int2* sp = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
     const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const long long nw = (long long)gridDim.x * kWarpsPerBlock;
-    const float inv_d = 1.0f / D, delta = a.sh.delta, delta2 = delta * delta, floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
+    const float inv_d = 1.0f / D, inv_delta = a.sh.inv_delta, inv_delta2 = a.sh.inv_delta2,
+                floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
     for (long long item = gw; item < (long long)Wt * a.S; item += nw) {
         const int t = (int)(item / a.S), b = (int)(item % a.S);
-        const __half* table = a.T + (size_t)t * a.sh.V * D;
-        float mu[G], sigma2;
-        predict<D>(table, a.rownorm2 + (size_t)t * a.sh.V, a.pairs + (long long)b * K, K, lane, inv_d, mu, sigma2);
-        const int q = scale_class(sigma2, floor2, delta2);
+        const char* col = reinterpret_cast<const char*>(a.T + (size_t)t * a.sh.V * D + 8 * (lane % Geo<D>::R));
+        const int2* gp = a.pairs + (long long)b * Kp;
+        __syncwarp();
+        prefetch_pairs(sp, gp, Kp, lane);
+        pairs_ready<0>();
         float kvv[G];
         load_half_vec<G>(reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, t, H, b, 0) + c0, kvv);
+        float mu[G], sigma2;
+        predict<D>(col, a.rownorm2 + (size_t)t * a.sh.V, sp, Kp, lane, inv_d, mu, sigma2);
+        const int q = scale_class(sigma2, floor2, inv_delta2);
         const long long o = ((long long)b * Wt + t) * a.sh.chunk_pos + a.open_slot;
         if (lane == 0) a.open_q[o] = q;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float r = __fsub_rn(kvv[g], mu[g]);
-            float n = rintf(__fdiv_rn(r, delta));
-            n = fminf(fmaxf(n, -(float)kSymLimit), (float)kSymLimit);
-            a.open_sym[o * D + c0 + g] = (int)n;
-        }
+        for (int g = 0; g < G; ++g) a.open_sym[o * D + c0 + g] = quantise(kvv[g], mu[g], inv_delta);
     }
 }
 
@@ -544,6 +634,14 @@ cudaError_t dispatch_d(int d, F&& f) {
         case 256: return f(std::integral_constant<int, 256>{});
     }
     return cudaErrorInvalidValue;
+}
+
+// Dynamic shared memory of the kernels that stage pairs: one slot of Kp entries per warp.
+template <class Kern>
+cudaError_t pair_smem_bytes(Kern kern, int Kp, size_t& bytes) {
+    bytes = (size_t)kWarpsPerBlock * 2 * Kp * sizeof(int2);
+    if (bytes > 24 * 1024) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    return cudaSuccess;
 }
 
 int sm_count() {
@@ -571,7 +669,11 @@ cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     return dispatch_d(a.sh.d, [&](auto D) {
-        encode_kernel<decltype(D)::value, false><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+        auto kern = encode_kernel<decltype(D)::value, false>;
+        size_t sm = 0;
+        cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
+        if (e2 != cudaSuccess) return e2;
+        kern<<<sm_count() * kBlocksPerSM, kThreads, sm, st>>>(a);
         count_launch();
         return cudaGetLastError();
     });
@@ -594,7 +696,11 @@ cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     return dispatch_d(a.sh.d, [&](auto D) {
-        decode_kernel<decltype(D)::value><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+        auto kern = decode_kernel<decltype(D)::value>;
+        size_t sm = 0;
+        cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
+        if (e2 != cudaSuccess) return e2;
+        kern<<<sm_count() * kBlocksPerSM, kThreads, sm, st>>>(a);
         count_launch();
         return cudaGetLastError();
     });
@@ -605,7 +711,11 @@ cudaError_t launch_append_quantise(const CodecArgs& a, cudaStream_t st) {
         long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (long long)sm_count() * 8) blocks = (long long)sm_count() * 8;
-        append_quantise_kernel<decltype(D)::value><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        auto kern = append_quantise_kernel<decltype(D)::value>;
+        size_t sm = 0;
+        cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
+        if (e2 != cudaSuccess) return e2;
+        kern<<<(unsigned)blocks, kThreads, sm, st>>>(a);
         count_launch();
         return cudaGetLastError();
     });

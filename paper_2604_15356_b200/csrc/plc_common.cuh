@@ -162,6 +162,7 @@ cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, cons
 struct CodecShape {
     int L, H, d, V, K, Kp, chunk_pos, out_dtype;   // Kp: K rounded up to the rows one warp-wide load fetches
     float delta, sigma_floor;
+    float inv_delta, inv_delta2;   // fl(1/delta), fl(1/(delta*delta)), rounded once on the host
 };
 
 struct KvView {
