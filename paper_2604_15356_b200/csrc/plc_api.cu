@@ -22,6 +22,8 @@ struct plc_ctx {
     unsigned int* ticket;
     unsigned int* status;
     Counters* counters;
+    uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1
+    size_t dense_bytes;
     int profiling;                  // record events around the codec kernels
     cudaEvent_t ev[4];              // encode start/stop, decode start/stop
     int ev_valid[2];
@@ -77,6 +79,24 @@ CodecArgs base_args(const plc_ctx* c) {
     return a;
 }
 
+DenseShape dense_shape(const plc_ctx* c, long long rows) {
+    DenseShape sh;
+    sh.rows = rows; sh.V = c->cfg.vocab; sh.d = c->cfg.head_dim; sh.tables = 2 * c->cfg.n_kv_heads;
+    sh.ldv = (sh.V + 63) / 64 * 64;
+    sh.ncols = sh.tables * sh.d; sh.ncols_pad = (sh.ncols + 255) / 256 * 256;
+    return sh;
+}
+
+plc_status ensure_dense(plc_ctx* c, const DenseShape& sh, size_t* off) {
+    const size_t need = dense_scratch_bytes(sh, off);
+    if (need <= c->dense_bytes) return PLC_OK;
+    if (c->dense_scratch) cudaFree(c->dense_scratch);
+    c->dense_scratch = nullptr; c->dense_bytes = 0;
+    if (cudaMalloc(&c->dense_scratch, need) != cudaSuccess) return PLC_E_CUDA;
+    c->dense_bytes = need;
+    return PLC_OK;
+}
+
 StreamsDev to_dev(const plc_streams* s) {
     StreamsDev d;
     d.payload = s->payload_dev; d.capacity = s->payload_capacity;
@@ -130,7 +150,7 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
 plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
     cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->staging);
-    cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters);
+    cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch);
     for (int i = 0; i < 4; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
     return PLC_OK;
@@ -173,11 +193,29 @@ static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n,
     return launch_topk(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
+// Dense variant: softmax once, then per layer the bf16 contraction and the coding of its 2H tables.
+static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, bool encode, cudaStream_t st) {
+    const DenseShape sh = dense_shape(c, (long long)a.S * a.n);
+    size_t off[5];
+    plc_status rc = ensure_dense(c, sh, off);
+    if (rc) return rc;
+    if (dense_softmax(static_cast<const __half*>(logits_dev), sh, c->dense_scratch, off, st) != cudaSuccess) return PLC_E_CUDA;
+    a.mu_dense = reinterpret_cast<const float*>(c->dense_scratch + off[3]);
+    a.s1_dense = reinterpret_cast<const float*>(c->dense_scratch + off[4]);
+    a.mu_ld = sh.ncols; a.s1_ld = sh.tables;
+    const size_t layer_elems = (size_t)sh.tables * sh.V * sh.d;
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st) != cudaSuccess) return PLC_E_CUDA;
+        a.dense_layer = l;
+        if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;
+    }
+    return PLC_OK;
+}
+
 plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
                       const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_streams* out,
                       const plc_debug_buffers* dbg, void* stream) {
     if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
-    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
     plc_status rc = check_view(kv, c->cfg.head_dim, 2);
     if (rc) return rc;
     const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
@@ -187,12 +225,14 @@ plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev,
     const long long items = (long long)2 * c->cfg.n_layers * c->cfg.n_kv_heads * S * out->max_chunks;
     if (items >= (1ll << 32)) return PLC_E_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
-    if (rc) return rc;
     CodecArgs a = base_args(c);
     a.kv = to_dev(kv); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
     a.st = to_dev(out);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, true, st);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    if (rc) return rc;
+    a.pairs = c->pairs;
     if (c->profiling) cudaEventRecord(c->ev[0], st);
     cudaError_t e = launch_encode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[1], st); c->ev_valid[0] = 1; }
@@ -203,7 +243,6 @@ plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev,
                       const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
                       const plc_debug_buffers* dbg, void* stream) {
     if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
-    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
     plc_status rc = check_view(kv_out, c->cfg.head_dim, c->cfg.out_dtype == PLC_OUT_F16 ? 2 : 4);
     if (rc) return rc;
     const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
@@ -213,12 +252,14 @@ plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev,
     const long long items = (long long)2 * c->cfg.n_layers * c->cfg.n_kv_heads * S * in->max_chunks;
     if (items >= (1ll << 32)) return PLC_E_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
-    if (rc) return rc;
     CodecArgs a = base_args(c);
     a.kv = to_dev(kv_out); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
     a.st = to_dev(in);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, false, st);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    if (rc) return rc;
+    a.pairs = c->pairs;
     if (c->profiling) cudaEventRecord(c->ev[2], st);
     cudaError_t e = launch_decode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[3], st); c->ev_valid[1] = 1; }
@@ -280,6 +321,7 @@ plc_status plc_sync_status(plc_ctx* c, void* stream) {
     if (cudaMemcpyAsync(&w, c->status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PLC_E_CUDA;
     if (cudaMemsetAsync(c->status, 0, sizeof(w), st) != cudaSuccess) return PLC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
+    if (w & kStTimeout) return PLC_E_CUDA;
     if (w & kStCorrupt) return PLC_E_CORRUPT;
     if (w & kStCapacity) return PLC_E_CAPACITY;
     return PLC_OK;

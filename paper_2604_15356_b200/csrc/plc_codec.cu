@@ -359,11 +359,11 @@ struct Item {
     long long slot;
 };
 
-__device__ __forceinline__ Item bulk_item(const CodecArgs& a, unsigned item) {
+__device__ __forceinline__ Item bulk_item(const CodecArgs& a, unsigned item, int t_first = 0) {
     Item it;
     const int MC = a.st.max_chunks;
     const unsigned per_table = (unsigned)a.S * (unsigned)MC;
-    it.t = (int)(item / per_table);
+    it.t = t_first + (int)(item / per_table);
     unsigned r = item % per_table;
     it.s = (int)(r / MC);
     it.c = (int)(r % MC);
@@ -419,9 +419,27 @@ __device__ __forceinline__ int quantise(float kv, float mu, float inv_delta) {
 
 extern __shared__ int2 g_pair_smem[];   // per warp: two slots of Kp entries
 
-template <int D, bool FROM_OPEN>
+// Prediction read from the dense variant's buffers: mu [row][tables_in_layer*D] and the variance
+// term s1 [row][tables_in_layer] (sum_v p_v ||T_v||^2 / d); sigma2 = max(0, s1 - ||mu||^2 / d).
+template <int D>
+__device__ __forceinline__ void predict_dense(const CodecArgs& a, long long row, int t_local, int c0, float inv_d,
+                                              float (&mu)[Geo<D>::G], float& sigma2) {
+    constexpr int G = Geo<D>::G;
+    const float* mp = a.mu_dense + row * a.mu_ld + (long long)t_local * D + c0;
+#pragma unroll
+    for (int g = 0; g < G; ++g) mu[g] = __ldg(mp + g);
+    const float s1 = __ldg(a.s1_dense + row * a.s1_ld + t_local);
+    const float s2 = warp_norm2<G>(mu);
+    sigma2 = fmaxf(0.f, s1 - s2 * inv_d);
+}
+
+enum { kSrcGather = 0, kSrcOpen = 1, kSrcDense = 2 };
+
+template <int D, int SRC>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
+    constexpr bool FROM_OPEN = SRC == kSrcOpen;
+    constexpr bool DENSE = SRC == kSrcDense;
     __shared__ EncTables tb;
     build_enc_tables(&tb);
     __syncthreads();
@@ -432,7 +450,8 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     const int cap_words = (int)a.staging_words_per_warp;
     const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
     int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
-    const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wt * a.S * a.st.max_chunks;
+    const int Wl = DENSE ? 2 * H : Wt;                       // tables this launch covers
+    const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wl * a.S * a.st.max_chunks;
     const float inv_d = 1.0f / D, inv_delta = a.sh.inv_delta, inv_delta2 = a.sh.inv_delta2,
                 floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
@@ -444,7 +463,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             it.p0 = 0; it.P = a.open_count;
             it.slot = ((long long)it.s * Wt + it.t) * a.st.max_chunks + it.c;
         } else {
-            it = bulk_item(a, item);
+            it = bulk_item(a, item, DENSE ? a.dense_layer * Wl : 0);
         }
         if (it.P <= 0) {
             if (lane == 0 && !FROM_OPEN) { a.st.chunk_offset[it.slot] = 0; a.st.chunk_bytes[it.slot] = 0; }
@@ -459,9 +478,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
         const __half* kvp = nullptr;
         int buf = 0;
         if (!FROM_OPEN) {
-            gp = a.pairs + ((long long)it.s * a.n + it.p0 + it.P - 1) * Kp;      // last position first
-            __syncwarp();                                                        // slot 0 is free again
-            prefetch_pairs(sp0, gp, Kp, lane);
+            if (!DENSE) {
+                gp = a.pairs + ((long long)it.s * a.n + it.p0 + it.P - 1) * Kp;  // last position first
+                __syncwarp();                                                    // slot 0 is free again
+                prefetch_pairs(sp0, gp, Kp, lane);
+            }
             kvp = reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, it.t, H, it.s, it.p0 + it.P - 1) + c0;
         }
         for (int p = it.P - 1; p >= 0; --p) {
@@ -473,17 +494,21 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
 #pragma unroll
                 for (int g = 0; g < G; ++g) sym[g] = a.open_sym[o * D + c0 + g];
             } else {
-                const int2* sp = sp0 + buf * Kp;
-                if (p > 0) {                                                      // one position ahead
-                    gp -= Kp;
-                    prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
-                    pairs_ready<1>();
-                } else {
-                    pairs_ready<0>();
-                }
-                buf ^= 1;
                 float mu[G], sigma2;
-                predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+                if (DENSE) {
+                    predict_dense<D>(a, (long long)it.s * a.n + it.p0 + p, it.t - a.dense_layer * Wl, c0, inv_d, mu, sigma2);
+                } else {
+                    const int2* sp = sp0 + buf * Kp;
+                    if (p > 0) {                                                  // one position ahead
+                        gp -= Kp;
+                        prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
+                        pairs_ready<1>();
+                    } else {
+                        pairs_ready<0>();
+                    }
+                    buf ^= 1;
+                    predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+                }
                 q = scale_class(sigma2, floor2, inv_delta2);
                 float kvv[G];
                 load_half_vec<G>(kvp, kvv);
@@ -513,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     }
 }
 
-template <int D>
+template <int D, bool DENSE>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     __shared__ DecTables tb;
@@ -523,13 +548,14 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
     const uint32_t lt = lanemask_lt();
     const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
     int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
-    const unsigned total = (unsigned)Wt * a.S * a.st.max_chunks;
+    const int Wl = DENSE ? 2 * H : Wt;
+    const unsigned total = (unsigned)Wl * a.S * a.st.max_chunks;
     const float inv_d = 1.0f / D, delta = a.sh.delta, inv_delta2 = a.sh.inv_delta2,
                 floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
 
     for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
-        const Item it = bulk_item(a, item);
+        const Item it = bulk_item(a, item, DENSE ? a.dense_layer * Wl : 0);
         if (it.P <= 0) continue;
         const unsigned long long off = a.st.chunk_offset[it.slot];
         const unsigned nbytes = a.st.chunk_bytes[it.slot];
@@ -547,21 +573,25 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
         const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
         const int2* gp = a.pairs + ((long long)it.s * a.n + it.p0) * Kp;
         __syncwarp();
-        prefetch_pairs(sp0, gp, Kp, lane);
+        if (!DENSE) prefetch_pairs(sp0, gp, Kp, lane);
         int buf = 0;
         long long kvo = kv_elem(a.kv, it.t, H, it.s, it.p0) + c0;
         for (int p = 0; p < it.P; ++p) {
-            const int2* sp = sp0 + buf * Kp;
-            if (p + 1 < it.P) {
-                gp += Kp;
-                prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
-                pairs_ready<1>();
-            } else {
-                pairs_ready<0>();
-            }
-            buf ^= 1;
             float mu[G], sigma2;
-            predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+            if (DENSE) {
+                predict_dense<D>(a, (long long)it.s * a.n + it.p0 + p, it.t - a.dense_layer * Wl, c0, inv_d, mu, sigma2);
+            } else {
+                const int2* sp = sp0 + buf * Kp;
+                if (p + 1 < it.P) {
+                    gp += Kp;
+                    prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
+                    pairs_ready<1>();
+                } else {
+                    pairs_ready<0>();
+                }
+                buf ^= 1;
+                predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+            }
             const int q = scale_class(sigma2, floor2, inv_delta2);
             __syncwarp();                                                         // readers of this slot are done
             int s, qp;
@@ -669,7 +699,12 @@ cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     return dispatch_d(a.sh.d, [&](auto D) {
-        auto kern = encode_kernel<decltype(D)::value, false>;
+        if (a.mu_dense) {
+            encode_kernel<decltype(D)::value, kSrcDense><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+            count_launch();
+            return cudaGetLastError();
+        }
+        auto kern = encode_kernel<decltype(D)::value, kSrcGather>;
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
@@ -686,7 +721,7 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
         long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (long long)sm_count() * kBlocksPerSM) blocks = (long long)sm_count() * kBlocksPerSM;
-        encode_kernel<decltype(D)::value, true><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        encode_kernel<decltype(D)::value, kSrcOpen><<<(unsigned)blocks, kThreads, 0, st>>>(a);
         count_launch();
         return cudaGetLastError();
     });
@@ -696,7 +731,12 @@ cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     return dispatch_d(a.sh.d, [&](auto D) {
-        auto kern = decode_kernel<decltype(D)::value>;
+        if (a.mu_dense) {
+            decode_kernel<decltype(D)::value, true><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+            count_launch();
+            return cudaGetLastError();
+        }
+        auto kern = decode_kernel<decltype(D)::value, false>;
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;

@@ -21,7 +21,7 @@ constexpr int kSymLimit = 1 << 30;
 constexpr uint32_t kFull = 0xffffffffu;
 
 // Bits of the device status word.
-constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u;
+constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u, kStTimeout = 8u;
 
 // Device counters (plc_stats).
 struct Counters {
@@ -188,10 +188,24 @@ struct CodecArgs {
     uint16_t* staging; unsigned long long staging_words_per_warp;   // encoder scratch
     unsigned int* ticket;                          // work counter (zeroed by the launcher)
     unsigned int* status; Counters* counters;
+    // dense variant: prediction read from buffers; one launch covers the 2*H tables of dense_layer
+    const float* mu_dense; const float* s1_dense; long long mu_ld, s1_ld; int dense_layer;
     // append path: symbols come from / go to the open chunk
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
 };
 int codec_grid_warps(int device);
+
+// Dense (full-vocabulary) prediction, one layer at a time.
+struct DenseShape {
+    long long rows;        // S * n positions
+    int V, d, tables;      // tables = 2 * H of one layer
+    int ldv;               // V rounded up to 64 (row pitch of P and Tb, in elements)
+    int ncols, ncols_pad;  // tables * d, rounded up to 256
+};
+size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]: P, Tb, n2b, mu, s1*/);
+cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st);
+cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
+                        unsigned int* status, cudaStream_t st);
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st);
 cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st);
 cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st);

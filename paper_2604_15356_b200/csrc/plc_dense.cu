@@ -1,0 +1,361 @@
+// Full-vocabulary prediction (Def. 5 of the paper: KV^ = sum over the whole vocabulary of
+// P(t | t_<i) F(t_<i, t)) as a dense bf16 contraction on the 5th-generation tensor cores:
+//   MU[rows x (2H*d)] = P[rows x V] * Tb[(2H*d) x V]^T     per layer, fp32 accumulation in TMEM.
+// P = bf16(softmax(logits)); Tb = bf16(T) of the layer, transposed so that both operands are
+// K-major (V contiguous).  One CTA computes a 128 x 256 tile: a TMA producer thread fills a
+// 4-stage shared-memory ring (128B-swizzled boxes of 64 K-elements), one thread issues
+// tcgen05.mma (128x256x16) into 256 TMEM columns and releases ring slots with tcgen05.commit,
+// four warps read the accumulators back with tcgen05.ld and store the tile.  No cluster, no
+// multicast.  Every mbarrier wait is bounded; a wait that runs out sets an error bit, the CTA
+// drains its own copies, frees its TMEM and returns.
+// The variance term s1[row][table] = sum_v P[row][v] * bf16(||Tb_v||^2 / d) is a small CUDA-core
+// kernel (1/128 of the contraction's work).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "plc_common.cuh"
+
+namespace plc {
+namespace {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4, kUmmaK = 16;
+constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 + 256;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and the error bit set) if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int* status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    atomicOr(status, kStTimeout);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    // K-major, 128-byte swizzle: start >> 4, LBO = 1 (unused), SBO = 1024 B between 8-row groups,
+    // descriptor version 1, layout type 2 (SWIZZLE_128B)
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  float* __restrict__ out, long long ldo, int rows, int ncols, int num_kb, unsigned int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);   // full[4], empty[4], tmem_full
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), tfull = smem_u32(bars + 2 * kStages);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(tfull, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0 && lane == 0) {
+        // TMA producer
+        int issued = 0;
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % kStages;
+            const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+            ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, status);
+            if (!ok) break;
+            mbar_expect_tx(full0 + 8 * s, kStageBytes);
+            const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+            tma_load_2d(sa, &map_a, kb * kBK, m0, full0 + 8 * s);
+            tma_load_2d(sa + kABytes, &map_b, kb * kBK, n0, full0 + 8 * s);
+            ++issued;
+        }
+        if (!ok) {
+            // drain: the copies already issued still land in this CTA's shared memory
+            for (int kb = issued > kStages ? issued - kStages : 0; kb < issued; ++kb)
+                mbar_wait(full0 + 8 * (kb % kStages), (uint32_t)(kb / kStages) & 1u, status);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // MMA issuer
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % kStages;
+            const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+            ok = mbar_wait(full0 + 8 * s, ph, status);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+            const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kABytes);
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k)
+                umma_bf16(tmem_base, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+            umma_commit(empty0 + 8 * s);              // frees the ring slot when these MMAs have read it
+        }
+        umma_commit(tfull);                           // accumulators complete (or nothing pending)
+    } else if (warp >= 2) {
+        // epilogue: warp w reads TMEM lanes 32*(w%4) ... +31
+        const bool ok = mbar_wait(tfull, 0, status);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int q = warp & 3;
+        const int row = m0 + q * 32 + lane;
+        if (ok) {
+            for (int c = 0; c < kBN / 32; ++c) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                      "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                      "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                      "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                    : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int col = n0 + c * 32;
+                if (row < rows && col < ncols) {
+                    float4* dst = reinterpret_cast<float4*>(out + (long long)row * ldo + col);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                             __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    }
+}
+
+// P[row][v] = bf16(exp(l_v - lse)), columns V..ldp-1 = 0.  One block per row.
+__global__ void __launch_bounds__(256) softmax_bf16_kernel(const __half* __restrict__ logits, long long rows, int V, int ldp,
+                                                           __nv_bfloat16* __restrict__ P) {
+    __shared__ float red_m[8], red_s[8];
+    __shared__ float sh_lse;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const __half* lr = logits + row * V;
+        float m = -INFINITY, s = 0.f;
+        for (int v = tid; v < V; v += 256) {
+            const float x = __half2float(lr[v]);
+            if (x > m) { s = s * expf(m - x) + 1.f; m = x; } else if (x > -INFINITY) s += expf(x - m);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(kFull, m, o), s2 = __shfl_xor_sync(kFull, s, o);
+            const float mm = fmaxf(m, m2);
+            s = ((m > -INFINITY) ? s * expf(m - mm) : 0.f) + ((m2 > -INFINITY) ? s2 * expf(m2 - mm) : 0.f);
+            m = mm;
+        }
+        __syncthreads();
+        if (lane == 0) { red_m[wid] = m; red_s[wid] = s; }
+        __syncthreads();
+        if (tid == 0) {
+            float mm = red_m[0], ss = red_s[0];
+            for (int w = 1; w < 8; ++w) {
+                const float m2 = red_m[w], s2 = red_s[w], nm = fmaxf(mm, m2);
+                ss = ((mm > -INFINITY) ? ss * expf(mm - nm) : 0.f) + ((m2 > -INFINITY) ? s2 * expf(m2 - nm) : 0.f);
+                mm = nm;
+            }
+            sh_lse = mm + logf(ss);
+        }
+        __syncthreads();
+        const float lse = sh_lse;
+        __nv_bfloat16* pr = P + row * ldp;
+        for (int v = tid; v < ldp; v += 256)
+            pr[v] = v < V ? __float2bfloat16_rn(expf(__half2float(lr[v]) - lse)) : __float2bfloat16_rn(0.f);
+    }
+}
+
+// Tb[t*d + j][v] = bf16(T_layer[t][v][j]): 32 x 32 tiles through shared memory.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __half* __restrict__ Tl, int tables, int V, int d, int ldv,
+                                                             __nv_bfloat16* __restrict__ Tb) {
+    __shared__ __nv_bfloat16 tile[32][33];
+    const int t = blockIdx.z, v0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;      // 32 x 8
+    const __half* src = Tl + (size_t)t * V * d;
+    for (int r = ty; r < 32; r += 8) {
+        const int v = v0 + r;
+        tile[r][tx] = (v < V) ? __float2bfloat16_rn(__half2float(src[(size_t)v * d + j0 + tx])) : __float2bfloat16_rn(0.f);
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int v = v0 + tx;
+        if (v < ldv) Tb[((size_t)t * d + j0 + r) * ldv + v] = tile[tx][r];
+    }
+}
+
+// n2b[t][v] = bf16(sum_j bf16(T[t][v][j])^2 / d), kept as float.  One warp per row.
+__global__ void __launch_bounds__(256) rownorm_bf16_kernel(const __half* __restrict__ Tl, long long nrows, int d, float* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const long long warp = (long long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long long)gridDim.x * 8;
+    for (long long r = warp; r < nrows; r += nw) {
+        float s = 0.f;
+        for (int j = lane; j < d; j += 32) {
+            const float x = __bfloat162float(__float2bfloat16_rn(__half2float(Tl[r * d + j])));
+            s = __fmaf_rn(x, x, s);
+        }
+        s = warp_sum(s);
+        if (lane == 0) out[r] = __bfloat162float(__float2bfloat16_rn(s / (float)d));
+    }
+}
+
+// s1[row][t] = sum_v P[row][v] * n2b[t][v].  One block per row, 8 tables at a time.
+__global__ void __launch_bounds__(256) s1_kernel(const __nv_bfloat16* __restrict__ P, int ldp, const float* __restrict__ n2b,
+                                                 long long rows, int V, int tables, float* __restrict__ s1) {
+    __shared__ float red[8][8];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const __nv_bfloat16* pr = P + row * ldp;
+        for (int t0 = 0; t0 < tables; t0 += 8) {
+            float acc[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) acc[g] = 0.f;
+            for (int v = tid; v < V; v += 256) {
+                const float p = __bfloat162float(pr[v]);
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    if (t0 + g < tables) acc[g] = __fmaf_rn(p, __ldg(n2b + (size_t)(t0 + g) * V + v), acc[g]);
+            }
+#pragma unroll
+            for (int g = 0; g < 8; ++g) acc[g] = warp_sum(acc[g]);
+            __syncthreads();
+            if (lane == 0)
+#pragma unroll
+                for (int g = 0; g < 8; ++g) red[wid][g] = acc[g];
+            __syncthreads();
+            if (tid < 8 && t0 + tid < tables) {
+                float s = 0.f;
+                for (int w = 0; w < 8; ++w) s += red[w][tid];
+                s1[row * tables + t0 + tid] = s;
+            }
+        }
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [outer][inner] (inner contiguous, row pitch ld elements), boxes of 64 x box_outer.
+bool make_map(CUtensorMap* map, void* base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
+    auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    size_t o = 0;
+    off[0] = o; o += up((size_t)sh.rows * sh.ldv * 2);                 // P
+    off[1] = o; o += up((size_t)sh.ncols_pad * sh.ldv * 2);            // Tb
+    off[2] = o; o += up((size_t)sh.tables * sh.V * 4);                 // n2b
+    off[3] = o; o += up((size_t)sh.rows * sh.ncols * 4);               // mu
+    off[4] = o; o += up((size_t)sh.rows * sh.tables * 4);              // s1
+    return o;
+}
+
+cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st) {
+    long long blocks = sh.rows < 148 * 8 ? sh.rows : 148 * 8;
+    softmax_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>(logits, sh.rows, sh.V, sh.ldv,
+                                                          reinterpret_cast<__nv_bfloat16*>(scratch + off[0]));
+    count_launch();
+    return cudaGetLastError();
+}
+
+// Prediction of one layer: fills mu [rows][ncols] and s1 [rows][tables] in the scratch.
+cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
+                        unsigned int* status, cudaStream_t st) {
+    __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(scratch + off[0]);
+    __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(scratch + off[1]);
+    float* n2b = reinterpret_cast<float*>(scratch + off[2]);
+    float* mu = reinterpret_cast<float*>(scratch + off[3]);
+    float* s1 = reinterpret_cast<float*>(scratch + off[4]);
+    cudaError_t e;
+    if (sh.ncols_pad > sh.ncols) {       // rows of Tb beyond the real columns must read as zero
+        e = cudaMemsetAsync(Tb + (size_t)sh.ncols * sh.ldv, 0, (size_t)(sh.ncols_pad - sh.ncols) * sh.ldv * 2, st);
+        if (e != cudaSuccess) return e;
+    }
+    dim3 tg((sh.ldv + 31) / 32, sh.d / 32, sh.tables);
+    transpose_bf16_kernel<<<tg, 256, 0, st>>>(T_layer, sh.tables, sh.V, sh.d, sh.ldv, Tb);
+    const long long nrows = (long long)sh.tables * sh.V;
+    rownorm_bf16_kernel<<<(unsigned)((nrows + 7) / 8 < 148 * 16 ? (nrows + 7) / 8 : 148 * 16), 256, 0, st>>>(T_layer, nrows, sh.d, n2b);
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, P, (uint64_t)sh.ldv, (uint64_t)sh.rows, (uint64_t)sh.ldv, kBM)) return cudaErrorUnknown;
+    if (!make_map(&mb, Tb, (uint64_t)sh.ldv, (uint64_t)sh.ncols_pad, (uint64_t)sh.ldv, kBN)) return cudaErrorUnknown;
+    e = cudaFuncSetAttribute(dense_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+    if (e != cudaSuccess) return e;
+    dim3 gg((unsigned)((sh.rows + kBM - 1) / kBM), (unsigned)(sh.ncols_pad / kBN));
+    dense_gemm_kernel<<<gg, kGemmThreads, kGemmSmem, st>>>(ma, mb, mu, (long long)sh.ncols, (int)sh.rows, sh.ncols,
+                                                           sh.ldv / kBK, status);
+    long long blocks = sh.rows < 148 * 8 ? sh.rows : 148 * 8;
+    s1_kernel<<<(unsigned)blocks, 256, 0, st>>>(P, sh.ldv, n2b, sh.rows, sh.V, sh.tables, s1);
+    count_launch(4);
+    return cudaGetLastError();
+}
+
+}  // namespace plc

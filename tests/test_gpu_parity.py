@@ -371,3 +371,52 @@ def test_f16_output(dev):
     assert ctx.sync_status() == plc.OK
     # float16 output adds half an ulp of binary16 (2^-9 relative at most for |x| < 8)
     assert float((out.float() - kvd.float()).abs().max()) <= 0.01 + 1e-3 + 8 * 2 ** -11
+
+
+@pytest.mark.parametrize("S,n,L,H,d,V", [(1, 200, 1, 1, 128, 1000), (2, 70, 2, 2, 64, 520), (1, 130, 1, 1, 64, 4096)])
+def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
+    """Def. 5 over the whole vocabulary as a bf16 tensor-core contraction (fp32 accumulation).
+    Tolerances: mu as for the top-K path; symbols may differ from the oracle (exact sum of the same
+    bf16 products) where (kv - mu)/delta is within 5e-3 of a rounding boundary -- the accumulation
+    error of a V-term fp32 tensor-core sum plus the binary32 exp of the softmax -- fewer than 2e-3
+    of them; the coder stays bit-exact on the GPU's own symbols and decode inverts encode."""
+    K, CP, delta = 8, 32, 0.02
+    tokens, logits, T, kv = make_workload(300 + V, S, n, L, H, d, V, K, pp=12.0)
+    ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, variant=plc.PRED_DENSE)
+    W, mc = ctx.W, ctx.max_chunks(n)
+    st = plc.StreamSet(S * W, mc, S * W * mc * 160 + 3 * S * n * W * d + 4096, dev)
+    sym = torch.zeros(S, n, W, d, dtype=torch.int32, device=dev)
+    q = torch.zeros(S, n, W, dtype=torch.int32, device=dev)
+    mu = torch.zeros(S, n, W, d, dtype=torch.float32, device=dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    ctx.encode(kvd, lgd, st, debug=plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr()))
+    assert ctx.sync_status() == plc.OK
+    cfg = orc.Config(L, H, d, V, K, delta, 0.0, CP, 1)
+    enc = orc.encode(cfg, T.numpy(), kv.numpy(), logits.numpy(), None, export=True)
+    mu_o = enc["mu"].reshape(S, n, W, d); sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W)
+    mu_g, sym_g, q_g = mu.cpu().numpy(), sym.cpu().numpy(), q.cpu().numpy()
+    scale = np.maximum(np.abs(mu_o).max(-1), 1e-3)
+    assert (np.abs(mu_g - mu_o).max(-1) <= 1e-3 * scale).all(), float((np.abs(mu_g - mu_o).max(-1) / scale).max())
+    diff = sym_g != sym_o
+    assert diff.mean() < 2e-3, diff.mean()
+    if diff.any():
+        assert np.abs(sym_g - sym_o)[diff].max() == 1
+        kvv = np.transpose(kv.numpy().astype(np.float64), (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)
+        t = (kvv - mu_o.astype(np.float64)) / delta
+        assert np.abs(t - np.floor(t) - 0.5)[diff].max() < 5e-3
+    assert (q_g != q_o).mean() < 2e-2 and np.abs(q_g - q_o).max() <= 1
+    total = 0
+    for s_ in range(S):
+        for t_ in range(W):
+            for c in range(mc):
+                P = min(CP, n - c * CP)
+                ref, _, _ = orc.rans_encode_chunk(sym_g[s_, c * CP:c * CP + P, t_], q_g[s_, c * CP:c * CP + P, t_])
+                assert np.array_equal(st.chunk((s_ * W + t_) * mc + c), ref), (s_, t_, c)
+                total += len(ref)
+    assert abs(total / enc["stats"].payload_bytes - 1) < 2e-3
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    sym2 = torch.zeros_like(sym)
+    ctx.decode(st, lgd, out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None))
+    assert ctx.sync_status() == plc.OK
+    assert torch.equal(sym2, sym)
+    assert float((out.cpu() - kv.float()).abs().max()) <= delta / 2 + 1e-3
