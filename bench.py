@@ -127,6 +127,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--set", action="append", default=[], help="override a workload field, e.g. --set L=4")
+    ap.add_argument("--variant", default="topk", choices=["topk", "dense"],
+                    help="prediction: top-K gather (default) or full-vocabulary bf16 tensor-core contraction")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -160,7 +162,9 @@ def main():
     cfg = w["cfg"]
     S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
     W = 2 * L * H
-    ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16)
+    dense = args.variant == "dense"
+    ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                      variant=plc.PRED_DENSE if dense else plc.PRED_TOPK)
     ctx.reserve(S * n)
     ctx.set_profiling(True)
     mc = ctx.max_chunks(n)
@@ -189,7 +193,7 @@ def main():
     sampler = ClockSampler(uuid)
     launches0 = plc.launch_count()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * args.steps)]
-    enc_k, dec_k = [], []
+    enc_k, dec_k, gemm_k = [], [], []
     barrier()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_start.record()
@@ -201,6 +205,8 @@ def main():
         ctx.decode(st, w["logits"], out)
         ev[3 * i + 2].record()
         enc_k.append(ctx.last_kernel_ms(0)); dec_k.append(ctx.last_kernel_ms(1))
+        if dense:
+            gemm_k.append(ctx.last_kernel_ms(2))
     t_end.record()
     barrier()
     launches = plc.launch_count() - launches0
@@ -234,7 +240,7 @@ def main():
     fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
     fma_ach = vecs * K * d / (dom_ms / 1e3)
     dom_name = "encode_kernel" if dom_enc else "decode_kernel"
-    default_cfg = args.workload == "llama2-7b" and not over
+    default_cfg = args.workload == "llama2-7b" and not over and not dense
     traffic = NCU_DRAM_BYTES_PER_VECTOR[dom_name] * vecs if default_cfg else None
     roofline = {"kernel": dom_name, "bound": "hbm",
                 "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
@@ -248,6 +254,17 @@ def main():
                 "fp32_fma": {"achieved_gfma_s": fma_ach / 1e9, "peak_gfma_s": fma_peak / 1e9, "frac": fma_ach / fma_peak},
                 "encode_kernel_ms": ek, "decode_kernel_ms": dk}
 
+    if dense:
+        # the contraction dominates: 2 * rows * V * (2H*d) flop per layer and direction
+        gm = statistics.mean(gemm_k)
+        flop = 2.0 * S * n * V * (2 * H * d)
+        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+        tpeak = float(pk.get("bf16_tflops_sustained", 1400.0))
+        roofline = {"kernel": "dense_gemm_kernel", "bound": "tensor", "achieved": flop / (gm / 1e3) / 1e12, "peak": tpeak,
+                    "unit": "TFLOP/s", "frac": flop / (gm / 1e3) / 1e12 / tpeak, "traffic": None,
+                    "peak_kind": "measured sustained bf16" if pk else "fallback", "ms_per_launch": gm,
+                    "flop_per_launch": flop, "launches_per_step": 2 * L,
+                    "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step)
@@ -268,7 +285,7 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
                        "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
-                       "kv_dtype": "f16", "decode_out": "f16",
+                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant,
                        "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
             "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
             "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),

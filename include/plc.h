@@ -211,8 +211,9 @@ plc_status plc_table_constants(int32_t qp, uint32_t* theta, uint32_t* rho);
 plc_status plc_build_table(int32_t qp, uint32_t* f, uint32_t* c);
 /* With profiling on, plc_encode / plc_decode record CUDA events on the caller's stream directly
  * around their fused predict+code kernel (the top-K kernel that precedes it is outside);
- * plc_last_kernel_ms waits for the most recent such launch (which = 0 encode, 1 decode) and returns
- * its duration.  PLC_E_STATE if no such launch was recorded. */
+ * plc_last_kernel_ms waits for the most recent such launch (which = 0 encode, 1 decode, 2 the dense
+ * variant's tensor-core contraction of the last layer) and returns its duration.  PLC_E_STATE if
+ * no such launch was recorded. */
 plc_status plc_set_profiling(plc_ctx* ctx, int32_t on);
 plc_status plc_last_kernel_ms(plc_ctx* ctx, int32_t which, float* ms);
 /* Number of kernels this library has launched in this process (for benchmarks). */

@@ -25,8 +25,8 @@ struct plc_ctx {
     uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1
     size_t dense_bytes;
     int profiling;                  // record events around the codec kernels
-    cudaEvent_t ev[4];              // encode start/stop, decode start/stop
-    int ev_valid[2];
+    cudaEvent_t ev[6];              // encode start/stop, decode start/stop, dense contraction start/stop
+    int ev_valid[3];
 };
 
 namespace {
@@ -141,7 +141,7 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
                  cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
     if (ok) ok = launch_rownorm(c->T, c->rownorm2, rows, cfg->head_dim, 0) == cudaSuccess &&
                  cudaDeviceSynchronize() == cudaSuccess;
-    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    for (int i = 0; i < 6 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
     if (!ok) { plc_destroy(c); return PLC_E_CUDA; }
     *out = c;
     return PLC_OK;
@@ -151,7 +151,7 @@ plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
     cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->staging);
     cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch);
-    for (int i = 0; i < 4; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (int i = 0; i < 6; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
     return PLC_OK;
 }
@@ -196,6 +196,7 @@ static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n,
 // Dense variant: softmax once, then per layer the bf16 contraction and the coding of its 2H tables.
 static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, bool encode, cudaStream_t st) {
     const DenseShape sh = dense_shape(c, (long long)a.S * a.n);
+    if (sh.tables > 256) return PLC_E_SHAPE;              // one norm column per table, at most 256 per launch
     size_t off[5];
     plc_status rc = ensure_dense(c, sh, off);
     if (rc) return rc;
@@ -205,9 +206,15 @@ static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, boo
     a.mu_ld = sh.ncols; a.s1_ld = sh.tables;
     const size_t layer_elems = (size_t)sh.tables * sh.V * sh.d;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-        if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st) != cudaSuccess) return PLC_E_CUDA;
+        const bool prof = c->profiling != 0;
+        if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st, prof ? c->ev[4] : nullptr,
+                        prof ? c->ev[5] : nullptr) != cudaSuccess) return PLC_E_CUDA;
+        if (prof) c->ev_valid[2] = 1;
         a.dense_layer = l;
+        const int w = encode ? 0 : 1;
+        if (prof) cudaEventRecord(c->ev[2 * w], st);
         if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;
+        if (prof) { cudaEventRecord(c->ev[2 * w + 1], st); c->ev_valid[w] = 1; }
     }
     return PLC_OK;
 }
@@ -360,7 +367,7 @@ plc_status plc_set_profiling(plc_ctx* c, int32_t on) {
 }
 
 plc_status plc_last_kernel_ms(plc_ctx* c, int32_t which, float* ms) {
-    if (!c || !ms || which < 0 || which > 1) return PLC_E_INVALID;
+    if (!c || !ms || which < 0 || which > 2) return PLC_E_INVALID;
     if (!c->ev_valid[which]) return PLC_E_STATE;
     if (cudaEventSynchronize(c->ev[2 * which + 1]) != cudaSuccess) return PLC_E_CUDA;
     return cudaEventElapsedTime(ms, c->ev[2 * which], c->ev[2 * which + 1]) == cudaSuccess ? PLC_OK : PLC_E_CUDA;

@@ -205,7 +205,7 @@ struct DenseShape {
 size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]: P, Tb, n2b, mu, s1*/);
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st);
 cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
-                        unsigned int* status, cudaStream_t st);
+                        unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1);   // events bracket the contraction
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st);
 cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st);
 cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st);

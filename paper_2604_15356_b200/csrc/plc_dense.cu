@@ -8,8 +8,8 @@
 // four warps read the accumulators back with tcgen05.ld and store the tile.  No cluster, no
 // multicast.  Every mbarrier wait is bounded; a wait that runs out sets an error bit, the CTA
 // drains its own copies, frees its TMEM and returns.
-// The variance term s1[row][table] = sum_v P[row][v] * bf16(||Tb_v||^2 / d) is a small CUDA-core
-// kernel (1/128 of the contraction's work).
+// The variance term s1[row][table] = sum_v P[row][v] * bf16(||Tb_v||^2 / d) is a second launch of
+// the same kernel with a narrow N tile (one column per table).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -68,18 +68,21 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = bn (multiple of 16, <= 256)
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  float* __restrict__ out, long long ldo, int rows, int ncols, int num_kb, unsigned int* status) {
+                  float* __restrict__ out, long long ldo, int rows, int ncols, int num_kb, int bn, unsigned int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);   // full[4], empty[4], tmem_full
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * bn;
+    const uint32_t stage_tx = (uint32_t)(kABytes + bn * kBK * 2), idesc = make_idesc(bn);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), tfull = smem_u32(bars + 2 * kStages);
 
     if (threadIdx.x == 0) {
@@ -105,7 +108,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
             ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, status);
             if (!ok) break;
-            mbar_expect_tx(full0 + 8 * s, kStageBytes);
+            mbar_expect_tx(full0 + 8 * s, stage_tx);
             const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
             tma_load_2d(sa, &map_a, kb * kBK, m0, full0 + 8 * s);
             tma_load_2d(sa + kABytes, &map_b, kb * kBK, n0, full0 + 8 * s);
@@ -129,7 +132,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kABytes);
 #pragma unroll
             for (int k = 0; k < kBK / kUmmaK; ++k)
-                umma_bf16(tmem_base, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+                umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
             umma_commit(empty0 + 8 * s);              // frees the ring slot when these MMAs have read it
         }
         umma_commit(tfull);                           // accumulators complete (or nothing pending)
@@ -139,8 +142,9 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int q = warp & 3;
         const int row = m0 + q * 32 + lane;
+        const bool vec_ok = ((ldo | ncols) & 3) == 0;
         if (ok) {
-            for (int c = 0; c < kBN / 32; ++c) {
+            for (int c = 0; c * 32 < bn; ++c) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32);
                 asm volatile(
@@ -155,11 +159,18 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int col = n0 + c * 32;
                 if (row < rows && col < ncols) {
-                    float4* dst = reinterpret_cast<float4*>(out + (long long)row * ldo + col);
+                    float* dr = out + (long long)row * ldo + col;
+                    if (vec_ok) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                             __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                        for (int j = 0; j < 8; ++j)
+                            if (col + 4 * j < ncols)
+                                reinterpret_cast<float4*>(dr)[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                                                __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < ncols) dr[j] = __uint_as_float(r[j]);
+                    }
                 }
             }
         }
@@ -172,43 +183,86 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
 }
 
-// P[row][v] = bf16(exp(l_v - lse)), columns V..ldp-1 = 0.  One block per row.
+// P[row][v] = bf16(exp(l_v - lse)), columns V..ldp-1 = 0.  One block per row; 8 logits per thread
+// and step when the row is 16-byte aligned.  exp is the fast intrinsic: its relative error (~1e-6)
+// is far below the 2^-9 of the bfloat16 result.
+template <bool VEC>
 __global__ void __launch_bounds__(256) softmax_bf16_kernel(const __half* __restrict__ logits, long long rows, int V, int ldp,
                                                            __nv_bfloat16* __restrict__ P) {
     __shared__ float red_m[8], red_s[8];
-    __shared__ float sh_lse;
+    __shared__ float sh_max, sh_lse;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
         const __half* lr = logits + row * V;
-        float m = -INFINITY, s = 0.f;
-        for (int v = tid; v < V; v += 256) {
-            const float x = __half2float(lr[v]);
-            if (x > m) { s = s * expf(m - x) + 1.f; m = x; } else if (x > -INFINITY) s += expf(x - m);
+        // pass 1: maximum
+        float m = -INFINITY;
+        if (VEC) {
+            for (int v = tid * 8; v < V; v += 256 * 8) {
+                const uint4 r = *reinterpret_cast<const uint4*>(lr + v);
+                const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(hp[j]); m = fmaxf(m, fmaxf(f.x, f.y)); }
+            }
+        } else {
+            for (int v = tid; v < V; v += 256) m = fmaxf(m, __half2float(lr[v]));
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float m2 = __shfl_xor_sync(kFull, m, o), s2 = __shfl_xor_sync(kFull, s, o);
-            const float mm = fmaxf(m, m2);
-            s = ((m > -INFINITY) ? s * expf(m - mm) : 0.f) + ((m2 > -INFINITY) ? s2 * expf(m2 - mm) : 0.f);
-            m = mm;
-        }
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
         __syncthreads();
-        if (lane == 0) { red_m[wid] = m; red_s[wid] = s; }
+        if (lane == 0) red_m[wid] = m;
         __syncthreads();
         if (tid == 0) {
-            float mm = red_m[0], ss = red_s[0];
-            for (int w = 1; w < 8; ++w) {
-                const float m2 = red_m[w], s2 = red_s[w], nm = fmaxf(mm, m2);
-                ss = ((mm > -INFINITY) ? ss * expf(mm - nm) : 0.f) + ((m2 > -INFINITY) ? s2 * expf(m2 - nm) : 0.f);
-                mm = nm;
+            float mm = red_m[0];
+            for (int w = 1; w < 8; ++w) mm = fmaxf(mm, red_m[w]);
+            sh_max = mm;
+        }
+        __syncthreads();
+        const float mx = sh_max;
+        // pass 2: sum of exponentials (row is in L2 now)
+        float s = 0.f;
+        if (VEC) {
+            for (int v = tid * 8; v < V; v += 256 * 8) {
+                const uint4 r = *reinterpret_cast<const uint4*>(lr + v);
+                const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(hp[j]); s += __expf(f.x - mx) + __expf(f.y - mx); }
             }
-            sh_lse = mm + logf(ss);
+        } else {
+            for (int v = tid; v < V; v += 256) s += __expf(__half2float(lr[v]) - mx);
+        }
+        s = warp_sum(s);
+        if (lane == 0) red_s[wid] = s;
+        __syncthreads();
+        if (tid == 0) {
+            float ss = 0.f;
+            for (int w = 0; w < 8; ++w) ss += red_s[w];
+            sh_lse = mx + __logf(ss);
         }
         __syncthreads();
         const float lse = sh_lse;
         __nv_bfloat16* pr = P + row * ldp;
-        for (int v = tid; v < ldp; v += 256)
-            pr[v] = v < V ? __float2bfloat16_rn(expf(__half2float(lr[v]) - lse)) : __float2bfloat16_rn(0.f);
+        if (VEC) {
+            for (int v = tid * 8; v < ldp; v += 256 * 8) {          // ldp is a multiple of 64
+                __nv_bfloat162 o[4];
+                if (v < V) {
+                    const uint4 r = *reinterpret_cast<const uint4*>(lr + v);
+                    const __half2* hp = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 f = __half22float2(hp[j]);
+                        o[j] = __floats2bfloat162_rn(__expf(f.x - lse), __expf(f.y - lse));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o[j] = __floats2bfloat162_rn(0.f, 0.f);
+                }
+                *reinterpret_cast<uint4*>(pr + v) = *reinterpret_cast<const uint4*>(o);
+            }
+        } else {
+            for (int v = tid; v < ldp; v += 256)
+                pr[v] = __float2bfloat16_rn(v < V ? __expf(__half2float(lr[v]) - lse) : 0.f);
+        }
+        __syncthreads();
     }
 }
 
@@ -230,8 +284,9 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __half* __res
     }
 }
 
-// n2b[t][v] = bf16(sum_j bf16(T[t][v][j])^2 / d), kept as float.  One warp per row.
-__global__ void __launch_bounds__(256) rownorm_bf16_kernel(const __half* __restrict__ Tl, long long nrows, int d, float* __restrict__ out) {
+// Nb[t][v] = bf16(sum_j bf16(T[t][v][j])^2 / d) (row pitch ldv).  One warp per row of T.
+__global__ void __launch_bounds__(256) rownorm_bf16_kernel(const __half* __restrict__ Tl, long long nrows, int V, int d, int ldv,
+                                                           __nv_bfloat16* __restrict__ out) {
     const int lane = threadIdx.x & 31;
     const long long warp = (long long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long long)gridDim.x * 8;
     for (long long r = warp; r < nrows; r += nw) {
@@ -241,40 +296,7 @@ __global__ void __launch_bounds__(256) rownorm_bf16_kernel(const __half* __restr
             s = __fmaf_rn(x, x, s);
         }
         s = warp_sum(s);
-        if (lane == 0) out[r] = __bfloat162float(__float2bfloat16_rn(s / (float)d));
-    }
-}
-
-// s1[row][t] = sum_v P[row][v] * n2b[t][v].  One block per row, 8 tables at a time.
-__global__ void __launch_bounds__(256) s1_kernel(const __nv_bfloat16* __restrict__ P, int ldp, const float* __restrict__ n2b,
-                                                 long long rows, int V, int tables, float* __restrict__ s1) {
-    __shared__ float red[8][8];
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
-        const __nv_bfloat16* pr = P + row * ldp;
-        for (int t0 = 0; t0 < tables; t0 += 8) {
-            float acc[8];
-#pragma unroll
-            for (int g = 0; g < 8; ++g) acc[g] = 0.f;
-            for (int v = tid; v < V; v += 256) {
-                const float p = __bfloat162float(pr[v]);
-#pragma unroll
-                for (int g = 0; g < 8; ++g)
-                    if (t0 + g < tables) acc[g] = __fmaf_rn(p, __ldg(n2b + (size_t)(t0 + g) * V + v), acc[g]);
-            }
-#pragma unroll
-            for (int g = 0; g < 8; ++g) acc[g] = warp_sum(acc[g]);
-            __syncthreads();
-            if (lane == 0)
-#pragma unroll
-                for (int g = 0; g < 8; ++g) red[wid][g] = acc[g];
-            __syncthreads();
-            if (tid < 8 && t0 + tid < tables) {
-                float s = 0.f;
-                for (int w = 0; w < 8; ++w) s += red[w][tid];
-                s1[row * tables + t0 + tid] = s;
-            }
-        }
+        if (lane == 0) out[(r / V) * ldv + (r % V)] = __float2bfloat16_rn(s / (float)d);
     }
 }
 
@@ -313,7 +335,7 @@ size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
     size_t o = 0;
     off[0] = o; o += up((size_t)sh.rows * sh.ldv * 2);                 // P
     off[1] = o; o += up((size_t)sh.ncols_pad * sh.ldv * 2);            // Tb
-    off[2] = o; o += up((size_t)sh.tables * sh.V * 4);                 // n2b
+    off[2] = o; o += up((size_t)((sh.tables + 15) / 16 * 16) * sh.ldv * 2);   // Nb (row norms, bf16)
     off[3] = o; o += up((size_t)sh.rows * sh.ncols * 4);               // mu
     off[4] = o; o += up((size_t)sh.rows * sh.tables * 4);              // s1
     return o;
@@ -321,18 +343,21 @@ size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
 
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st) {
     long long blocks = sh.rows < 148 * 8 ? sh.rows : 148 * 8;
-    softmax_bf16_kernel<<<(unsigned)blocks, 256, 0, st>>>(logits, sh.rows, sh.V, sh.ldv,
-                                                          reinterpret_cast<__nv_bfloat16*>(scratch + off[0]));
+    __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(scratch + off[0]);
+    if (sh.V % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0)
+        softmax_bf16_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(logits, sh.rows, sh.V, sh.ldv, P);
+    else
+        softmax_bf16_kernel<false><<<(unsigned)blocks, 256, 0, st>>>(logits, sh.rows, sh.V, sh.ldv, P);
     count_launch();
     return cudaGetLastError();
 }
 
 // Prediction of one layer: fills mu [rows][ncols] and s1 [rows][tables] in the scratch.
 cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
-                        unsigned int* status, cudaStream_t st) {
+                        unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(scratch + off[0]);
     __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(scratch + off[1]);
-    float* n2b = reinterpret_cast<float*>(scratch + off[2]);
+    __nv_bfloat16* Nb = reinterpret_cast<__nv_bfloat16*>(scratch + off[2]);
     float* mu = reinterpret_cast<float*>(scratch + off[3]);
     float* s1 = reinterpret_cast<float*>(scratch + off[4]);
     cudaError_t e;
@@ -343,17 +368,26 @@ cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* sc
     dim3 tg((sh.ldv + 31) / 32, sh.d / 32, sh.tables);
     transpose_bf16_kernel<<<tg, 256, 0, st>>>(T_layer, sh.tables, sh.V, sh.d, sh.ldv, Tb);
     const long long nrows = (long long)sh.tables * sh.V;
-    rownorm_bf16_kernel<<<(unsigned)((nrows + 7) / 8 < 148 * 16 ? (nrows + 7) / 8 : 148 * 16), 256, 0, st>>>(T_layer, nrows, sh.d, n2b);
+    e = cudaMemsetAsync(Nb, 0, (size_t)((sh.tables + 15) / 16 * 16) * sh.ldv * 2, st);     // padding rows / columns read as zero
+    if (e != cudaSuccess) return e;
+    rownorm_bf16_kernel<<<(unsigned)((nrows + 7) / 8 < 148 * 16 ? (nrows + 7) / 8 : 148 * 16), 256, 0, st>>>(T_layer, nrows, sh.V, sh.d, sh.ldv, Nb);
     CUtensorMap ma, mb;
+    const int nb_rows = (sh.tables + 15) / 16 * 16;                     // norm matrix rows, <= 256
+    CUtensorMap mn;
     if (!make_map(&ma, P, (uint64_t)sh.ldv, (uint64_t)sh.rows, (uint64_t)sh.ldv, kBM)) return cudaErrorUnknown;
     if (!make_map(&mb, Tb, (uint64_t)sh.ldv, (uint64_t)sh.ncols_pad, (uint64_t)sh.ldv, kBN)) return cudaErrorUnknown;
+    if (!make_map(&mn, Nb, (uint64_t)sh.ldv, (uint64_t)nb_rows, (uint64_t)sh.ldv, (uint32_t)nb_rows)) return cudaErrorUnknown;
     e = cudaFuncSetAttribute(dense_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
     if (e != cudaSuccess) return e;
     dim3 gg((unsigned)((sh.rows + kBM - 1) / kBM), (unsigned)(sh.ncols_pad / kBN));
+    if (ev0) cudaEventRecord(ev0, st);
     dense_gemm_kernel<<<gg, kGemmThreads, kGemmSmem, st>>>(ma, mb, mu, (long long)sh.ncols, (int)sh.rows, sh.ncols,
-                                                           sh.ldv / kBK, status);
-    long long blocks = sh.rows < 148 * 8 ? sh.rows : 148 * 8;
-    s1_kernel<<<(unsigned)blocks, 256, 0, st>>>(P, sh.ldv, n2b, sh.rows, sh.V, sh.tables, s1);
+                                                           sh.ldv / kBK, kBN, status);
+    if (ev1) cudaEventRecord(ev1, st);
+    // variance term: s1 = P * Nb^T, the same kernel with an N tile of nb_rows columns
+    dim3 gn(gg.x, 1);
+    dense_gemm_kernel<<<gn, kGemmThreads, kGemmSmem, st>>>(ma, mn, s1, (long long)sh.tables, (int)sh.rows, sh.tables,
+                                                           sh.ldv / kBK, nb_rows, status);
     count_launch(4);
     return cudaGetLastError();
 }
