@@ -147,6 +147,8 @@ def main():
     plc.build()
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    if args.workload == "append":
+        return append_arm(args, torch, plc, workloads, dev)
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -299,6 +301,63 @@ def main():
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+    return 0
+
+
+def append_arm(args, torch, plc, workloads, dev):
+    """Decode-time append: B sessions grow by one token per plc_append_step; per-step latency.
+    `--steps` counts groups of 32 append steps (one chunk seal per group)."""
+    from paper_2604_15356_b200 import synth
+    over = {}
+    for kvs in args.set:
+        k, v = kvs.split("=")
+        over[k] = float(v) if "." in v else int(v)
+    cfg = dict(workloads.CONFIGS["append"]); cfg.update(over)
+    B, L, H, d, V, K, CP = cfg["S"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"], cfg["chunk_pos"]
+    nsteps = CP * max(args.steps, 1)
+    W = 2 * L * H
+    seed = 20260419
+    table = synth.markov_table(V, cfg["pp"], seed, device=dev)
+    tokens = synth.sample_tokens(table, B, nsteps, seed + 1)
+    logits = synth.position_logits(table, tokens)                       # [B][nsteps][V]
+    T = synth.make_tables(L, H, V, d, seed + 2, device=dev)
+    ctx = plc.Context(T, K, cfg["delta"], chunk_pos=CP)
+    sb = ctx.new_session_batch(B, nsteps // CP + 1, int(nsteps * B * W * d * 1.4) + (1 << 20))
+    g = torch.Generator(device=dev); g.manual_seed(seed + 3)
+    lat = []
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nsteps)]
+    launches0 = plc.launch_count()
+    for i in range(nsteps):
+        tok = tokens[:, i].to(torch.int64)
+        kv_step = (T[:, :, :, tok, :].permute(0, 1, 3, 2, 4).float() +
+                   cfg["sigma"] * torch.randn(L, 2, B, H, d, device=dev, generator=g)).to(torch.float16).contiguous()
+        lg = logits[:, i, :].contiguous()
+        torch.cuda.synchronize()
+        ev[i][0].record()
+        ctx.append_step(sb, kv_step, lg)
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    assert ctx.sync_status() == plc.OK
+    lat = sorted(a.elapsed_time(b) for a, b in ev[CP:])                 # first chunk = warm-up
+    seal = sorted(ev[i][0].elapsed_time(ev[i][1]) for i in range(CP, nsteps) if (i + 1) % CP == 0)
+    st = ctx.stats()
+    mean_ms = sum(lat) / len(lat)
+    peak, kind = measured_peaks()
+    gathered = B * W * K * d * 2
+    line = {"metric": METRIC, "value": B / (mean_ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": nsteps - CP, "warmup": CP,
+            "ms_per_step": mean_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "append", "B": B, "L": L, "H": H, "d": d, "V": V, "K": K, "delta": cfg["delta"],
+                       "chunk_pos": CP, "perplexity": cfg["pp"], "encode_only": True},
+            "latency_ms": {"p50": lat[len(lat) // 2], "p99": lat[int(len(lat) * 0.99)], "max": lat[-1],
+                           "seal_steps_mean": sum(seal) / max(len(seal), 1)},
+            "bits_per_token": 8 * (st.payload_bytes + 12 * st.n_chunks) / max(st.coded_vectors / W, 1),
+            "roofline": {"kernel": "append_quantise_kernel", "bound": "hbm", "achieved": gathered / (lat[len(lat) // 2] / 1e3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": gathered / (lat[len(lat) // 2] / 1e3) / 1e9 / peak,
+                         "traffic": None, "peak_kind": kind,
+                         "accounting": "random 256-byte T rows per step (B*W*K*d*2 bytes) over the median whole-step time"},
+            "gpu_launches": plc.launch_count() - launches0}
+    print(json.dumps(line))
     return 0
 
 
