@@ -31,7 +31,8 @@ struct Smem {
     uint32_t cand_key[kCandCap];
     int32_t cand_idx[kCandCap];
     float ek[kCandCap];
-    float red_m[kWarps], red_s[kWarps];
+    uint32_t red_k[kWarps];
+    float red_s[kWarps];
     int scan[kWarps];
     int nsel, ncand, bstar, count_above, cstar, thr, need, neq, running;
     float row_max, row_sum, sum_k;
@@ -101,36 +102,22 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
         if (tid == 0) { sm.nsel = 0; sm.ncand = 0; sm.running = 0; }
         __syncthreads();
 
-        // Pass A: histogram of the top 12 key bits, running max and sum of exponentials.
-        float m = -INFINITY, s = 0.f;
+        // Pass A: histogram of the top 12 key bits and the largest key (keys order like the logits).
+        uint32_t kmax = 0;
         for (int t = 0; t < ntiles; ++t)
             for_tile<VEC>(row, V, t, [&](int, uint32_t bits) {
-                uint32_t key = key_of(bits);
+                const uint32_t key = key_of(bits);
                 atomicAdd(&sm.hist[key >> 4], 1u);
-                float x = val_of_key(key);
-                if (x > m) { s = s * expf(m - x) + 1.f; m = x; }
-                else if (x > -INFINITY) s += expf(x - m);
+                kmax = max(kmax, key);
             });
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            float m2 = __shfl_xor_sync(kFull, m, o), s2 = __shfl_xor_sync(kFull, s, o);
-            float mm = fmaxf(m, m2);
-            float a1 = (m > -INFINITY) ? s * expf(m - mm) : 0.f, a2 = (m2 > -INFINITY) ? s2 * expf(m2 - mm) : 0.f;
-            // fixed operand order by lane parity keeps both partners bit-identical
-            s = (lane & o) ? (a2 + a1) : (a1 + a2);
-            m = mm;
-        }
-        if (lane == 0) { sm.red_m[wid] = m; sm.red_s[wid] = s; }
+        for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
+        if (lane == 0) sm.red_k[wid] = kmax;
         __syncthreads();
         if (tid == 0) {
-            float mm = sm.red_m[0], ss = sm.red_s[0];
-            for (int w = 1; w < kWarps; ++w) {
-                float m2 = sm.red_m[w], s2 = sm.red_s[w];
-                float nm = fmaxf(mm, m2);
-                ss = ((mm > -INFINITY) ? ss * expf(mm - nm) : 0.f) + ((m2 > -INFINITY) ? s2 * expf(m2 - nm) : 0.f);
-                mm = nm;
-            }
-            sm.row_max = mm; sm.row_sum = ss;
+            uint32_t km = sm.red_k[0];
+            for (int w = 1; w < kWarps; ++w) km = max(km, sm.red_k[w]);
+            sm.row_max = val_of_key(km);
         }
 
         // Bin that holds the K-th largest key: thread t owns bins 4095-16t ... 4095-16t-15.
@@ -155,9 +142,14 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
         const bool use_cand = cstar <= kCandCap;
 
         // Pass B: everything above the bin is selected; inside the bin refine on the low 4 key bits.
+        // The same pass sums exp(l - l_max) over the row (fast exponential: its relative error of
+        // about 2e-6 at the arguments that matter is inside the tolerance of lse and Z_k).
+        const float lmax_b = sm.row_max;
+        float s = 0.f;
         for (int t = 0; t < ntiles; ++t)
             for_tile<VEC>(row, V, t, [&](int i, uint32_t bits) {
                 uint32_t key = key_of(bits);
+                s += __expf(__half2float(__ushort_as_half((unsigned short)bits)) - lmax_b);
                 int bin = (int)(key >> 4);
                 if (bin > bstar) {
                     int slot = atomicAdd(&sm.nsel, 1);
@@ -170,8 +162,13 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
                     }
                 }
             });
+        s = warp_sum(s);
+        if (lane == 0) sm.red_s[wid] = s;
         __syncthreads();
         if (tid == 0) {
+            float ss = 0.f;
+            for (int w = 0; w < kWarps; ++w) ss += sm.red_s[w];
+            sm.row_sum = ss;
             int need1 = K - count_above, cum = 0;
             for (int j = 15; j >= 0; --j) {
                 int c = (int)sm.sub[j];
