@@ -30,7 +30,8 @@ def build(force=False):
 
 class Config(C.Structure):
     _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("K", C.c_int32),
-                ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32), ("dense", C.c_int32)]
+                ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32), ("dense", C.c_int32),
+                ("adaptive_b0", C.c_int32), ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float)]
 
 
 class KVStrides(C.Structure):
@@ -120,6 +121,12 @@ def class_params(q):
     s, qp = C.c_int(), C.c_int()
     lib().plo_class_params(int(q), C.byref(s), C.byref(qp))
     return s.value, qp.value
+
+
+def adaptive_bits(h, b0, hbar, extra):
+    """Def. 7: bits per component at surprisal h (bits), capped at b0 + extra."""
+    lib().plo_adaptive_bits.argtypes = [C.c_float, C.c_int, C.c_float, C.c_int]
+    return lib().plo_adaptive_bits(C.c_float(h), int(b0), C.c_float(hbar), int(extra))
 
 
 def quantise(kv, mu, delta):
@@ -232,6 +239,7 @@ def encode(cfg, T, kv, logits, tokens, pos_begin=None, pos_end=None, export=Fals
     nby = np.zeros(nslots, np.uint32)
     stats = Stats()
     sym = q = mu = None
+    bits = np.zeros((S, n), np.int32) if cfg.adaptive_b0 > 0 else None
     if export:
         sym = np.zeros((S, n, L, 2, H, d), np.int32)
         q = np.zeros((S, n, L, 2, H), np.int32)
@@ -239,15 +247,15 @@ def encode(cfg, T, kv, logits, tokens, pos_begin=None, pos_end=None, export=Fals
     st = _strides(kv)
     rc = lib().plo_encode(C.byref(cfg), _p(Tb), C.c_void_p(kvv.ctypes.data), C.byref(st), _p(lg), _p(tk), S, n,
                           _p(pb), _p(pe), mc, _p(payload), C.c_uint64(cap), _p(off), _p(nby), C.byref(stats),
-                          _p(sym), _p(q), _p(mu))
+                          _p(sym), _p(q), _p(mu), _p(bits))
     if rc:
         raise ValueError(f"plo_encode rc={rc}")
     shape = (S, L, 2, H, mc)
     return dict(payload=payload, chunk_offset=off.reshape(shape), chunk_bytes=nby.reshape(shape), stats=stats,
-                sym=sym, q=q, mu=mu, max_chunks=mc)
+                sym=sym, q=q, mu=mu, bits=bits, max_chunks=mc)
 
 
-def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=False):
+def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=False, tokens=None):
     """Whole-path decode of the dict ``encode`` returned.  kv_shape = (L,2,S,H,n,d); returns float32 KV'."""
     Tb = _h(T)
     lg = _h(logits)
@@ -260,6 +268,7 @@ def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=F
     sym = np.zeros((S, n, L, 2, H, d), np.int32) if export else None
     off = np.ascontiguousarray(enc["chunk_offset"]).reshape(-1)
     nby = np.ascontiguousarray(enc["chunk_bytes"]).reshape(-1)
-    rc = lib().plo_decode(C.byref(cfg), _p(Tb), _p(lg), S, n, _p(pb), _p(pe), enc["max_chunks"], _p(enc["payload"]),
+    tk = None if tokens is None else np.ascontiguousarray(tokens, dtype=np.int32)
+    rc = lib().plo_decode(C.byref(cfg), _p(Tb), _p(lg), _p(tk), S, n, _p(pb), _p(pe), enc["max_chunks"], _p(enc["payload"]),
                           _p(off), _p(nby), _p(out), C.byref(st), _p(sym))
     return rc, out, sym

@@ -475,6 +475,22 @@ void plo_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* l
     }
 }
 
+/* ---------------------------------------------------------------- adaptive step */
+
+/* Def. 7 (surprisal-adaptive quantiser): at a position of surprisal h = -log2 P(x_i | x_<i) the
+ * residual gets b = max(1, floor(b0 h / hbar)) bits per component.  With an entropy coder behind
+ * the quantiser a bit more means half the step, so the position's step is delta 2^(b0 - b): b = b0
+ * reproduces the fixed-step coder.  The paper puts no upper limit on b; the symbol range is
+ * finite, so b is capped at b0 + extra.  The floor is an integer decided by floating point: it is
+ * taken in binary32 on h rounded to binary32. */
+int plo_adaptive_bits(float h, int b0, float hbar, int extra) {
+    float r = (float)b0 * (h / hbar);
+    int b = (int)floorf(r);
+    if (!(r >= 1.0f)) b = 1;
+    if (b > b0 + extra) b = b0 + extra;
+    return b;
+}
+
 /* ---------------------------------------------------------------- whole path */
 
 /* Strides, in elements, of a KV tensor whose last dimension (d) is contiguous. */
@@ -485,6 +501,9 @@ typedef struct {
     float delta, sigma_floor;
     int32_t chunk_pos;
     int32_t dense;          /* 0: top-K mixture, 1: full-vocabulary bf16 mixture */
+    int32_t adaptive_b0;    /* > 0: surprisal-adaptive step (Def. 7) with target depth b0 */
+    int32_t adaptive_extra; /* cap: b_i <= b0 + adaptive_extra */
+    float adaptive_hbar;    /* average surprisal h-bar, bits */
 } plo_config;
 
 typedef struct {
@@ -508,9 +527,11 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
                const uint16_t* logits /*[S][n][V]*/, const int32_t* tokens /*[S][n]*/, int S, int n,
                const int32_t* pos_begin, const int32_t* pos_end, int max_chunks,
                uint8_t* payload, uint64_t cap, uint64_t* chunk_offset, uint32_t* chunk_bytes,
-               plo_stats* stats, int32_t* sym_out, int32_t* q_out, float* mu_out) {
+               plo_stats* stats, int32_t* sym_out, int32_t* q_out, float* mu_out, int32_t* bits_out /*[S][n]*/) {
     int L = cfg->L, H = cfg->H, d = cfg->d, V = cfg->V, K = cfg->K, CP = cfg->chunk_pos;
     if (!valid_d(d) || CP < 1) return PLO_E_INVALID;
+    if (cfg->adaptive_b0 > 0 && !tokens) return PLO_E_INVALID;
+    float* pdelta = (float*)malloc(sizeof(float) * (size_t)n);   /* step of each position of the session */
     memset(stats, 0, sizeof(*stats));
     int32_t* idx = (int32_t*)malloc(sizeof(int32_t) * (size_t)n * K);
     double* w = (double*)malloc(sizeof(double) * (size_t)n * K);
@@ -529,6 +550,12 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
             plo_topk_softmax_row(logits + ((size_t)s * n + i) * V, V, K, tokens ? tokens[(size_t)s * n + i] : -1,
                                  idx + (size_t)i * K, w + (size_t)i * K, lse + i, zk + i, lp + i);
             if (tokens) stats->token_bits -= lp[i];
+            pdelta[i] = cfg->delta;
+            if (cfg->adaptive_b0 > 0) {
+                int bi = plo_adaptive_bits((float)(-lp[i]), cfg->adaptive_b0, cfg->adaptive_hbar, cfg->adaptive_extra);
+                pdelta[i] = ldexpf(cfg->delta, cfg->adaptive_b0 - bi);
+                if (bits_out) bits_out[(size_t)s * n + i] = bi;
+            }
         }
         stats->coded_positions += (uint64_t)(e - b);
         for (int l = 0; l < L && !rc; ++l) for (int a = 0; a < 2 && !rc; ++a) for (int h = 0; h < H && !rc; ++h) {
@@ -539,9 +566,9 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
                     int i = p0 + p; double s2;
                     if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mu, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mu, &s2);
-                    cq[p] = plo_class(s2, cfg->sigma_floor, cfg->delta);
+                    cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
                     const uint16_t* x = kv + l * st->layer + a * st->kv + s * st->session + h * st->head + (int64_t)i * st->pos;
-                    plo_quantise(x, mu, d, cfg->delta, csym + (size_t)p * d);
+                    plo_quantise(x, mu, d, pdelta[i], csym + (size_t)p * d);
                     size_t o = ((((size_t)s * n + i) * L + l) * 2 + a) * H + h;
                     if (sym_out) memcpy(sym_out + o * d, csym + (size_t)p * d, sizeof(int32_t) * d);
                     if (q_out) q_out[o] = cq[p];
@@ -558,14 +585,14 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
             }
         }
     }
-    free(idx); free(w); free(lse); free(zk); free(lp); free(csym); free(cq); free(mu);
+    free(idx); free(w); free(lse); free(zk); free(lp); free(csym); free(cq); free(mu); free(pdelta);
     return rc;
 }
 
 /* Decode (Sec. 7.2, integration point 2): the prediction and its class are recomputed from the
  * logits exactly as in the encoder, the symbols come from the chunk, KV' = mu + sym delta.
  * kv_out is float with the same strides; positions outside [pos_begin, pos_end) are not written. */
-int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits, int S, int n,
+int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits, const int32_t* tokens, int S, int n,
                const int32_t* pos_begin, const int32_t* pos_end, int max_chunks,
                const uint8_t* payload, const uint64_t* chunk_offset, const uint32_t* chunk_bytes,
                float* kv_out, const plo_kv_strides* st, int32_t* sym_out) {
@@ -578,12 +605,21 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
     int32_t* csym = (int32_t*)malloc(sizeof(int32_t) * (size_t)CP * d);
     int32_t* cq = (int32_t*)malloc(sizeof(int32_t) * (size_t)CP);
     double* mus = (double*)malloc(sizeof(double) * (size_t)CP * d);
+    float* pdelta = (float*)malloc(sizeof(float) * (size_t)n);
     int rc = PLO_OK;
+    if (cfg->adaptive_b0 > 0 && !tokens) rc = PLO_E_INVALID;
     for (int s = 0; s < S && !rc; ++s) {
         int b = pos_begin ? pos_begin[s] : 0, e = pos_end ? pos_end[s] : n;
         if (b < 0 || e > n || b > e) { rc = PLO_E_INVALID; break; }
-        for (int i = b; i < e; ++i)
-            plo_topk_softmax_row(logits + ((size_t)s * n + i) * V, V, K, -1, idx + (size_t)i * K, w + (size_t)i * K, lse + i, &zk, &lp);
+        for (int i = b; i < e; ++i) {
+            plo_topk_softmax_row(logits + ((size_t)s * n + i) * V, V, K, tokens ? tokens[(size_t)s * n + i] : -1,
+                                 idx + (size_t)i * K, w + (size_t)i * K, lse + i, &zk, &lp);
+            pdelta[i] = cfg->delta;
+            if (cfg->adaptive_b0 > 0) {
+                int bi = plo_adaptive_bits((float)(-lp), cfg->adaptive_b0, cfg->adaptive_hbar, cfg->adaptive_extra);
+                pdelta[i] = ldexpf(cfg->delta, cfg->adaptive_b0 - bi);
+            }
+        }
         for (int l = 0; l < L && !rc; ++l) for (int a = 0; a < 2 && !rc; ++a) for (int h = 0; h < H && !rc; ++h) {
             const uint16_t* table = T + ((((size_t)l * 2 + a) * H + h) * (size_t)V) * d;
             for (int ch = 0; b + ch * CP < e; ++ch) {
@@ -592,7 +628,7 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                     int i = p0 + p; double s2;
                     if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mus + (size_t)p * d, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mus + (size_t)p * d, &s2);
-                    cq[p] = plo_class(s2, cfg->sigma_floor, cfg->delta);
+                    cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
                 }
                 int64_t slot = chunk_slot(cfg, S, max_chunks, s, l, a, h, ch);
                 int r = plo_rans_decode_chunk(payload + chunk_offset[slot], chunk_bytes[slot], cq, P, d, csym);
@@ -600,7 +636,7 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                 for (int p = 0; p < P; ++p) {
                     int i = p0 + p;
                     float* o = kv_out + l * st->layer + a * st->kv + s * st->session + h * st->head + (int64_t)i * st->pos;
-                    plo_reconstruct(mus + (size_t)p * d, csym + (size_t)p * d, d, cfg->delta, o);
+                    plo_reconstruct(mus + (size_t)p * d, csym + (size_t)p * d, d, pdelta[i], o);
                     if (sym_out) {
                         size_t oo = ((((size_t)s * n + i) * L + l) * 2 + a) * H + h;
                         memcpy(sym_out + oo * d, csym + (size_t)p * d, sizeof(int32_t) * d);
@@ -609,6 +645,6 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
             }
         }
     }
-    free(idx); free(w); free(lse); free(csym); free(cq); free(mus);
+    free(idx); free(w); free(lse); free(csym); free(cq); free(mus); free(pdelta);
     return rc;
 }
