@@ -127,6 +127,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--set", action="append", default=[], help="override a workload field, e.g. --set L=4")
+    ap.add_argument("--adaptive", type=int, default=0,
+                    help="b0 > 0: surprisal-adaptive step (Def. 7) with hbar = log2(perplexity), cap b0 + 4")
     ap.add_argument("--variant", default="topk", choices=["topk", "dense"],
                     help="prediction: top-K gather (default) or full-vocabulary bf16 tensor-core contraction")
     args = ap.parse_args()
@@ -165,8 +167,11 @@ def main():
     S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
     W = 2 * L * H
     dense = args.variant == "dense"
+    import math
+    adaptive = (args.adaptive, 4, math.log2(cfg["pp"])) if args.adaptive > 0 else None
+    tok = w["tokens"] if adaptive else None
     ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                      variant=plc.PRED_DENSE if dense else plc.PRED_TOPK)
+                      variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive)
     ctx.reserve(S * n)
     ctx.set_profiling(True)
     mc = ctx.max_chunks(n)
@@ -177,8 +182,8 @@ def main():
 
     def step():
         st.total_bytes.zero_()
-        ctx.encode(w["kv"], w["logits"], st)
-        ctx.decode(st, w["logits"], out)
+        ctx.encode(w["kv"], w["logits"], st, tokens=tok)
+        ctx.decode(st, w["logits"], out, tokens=tok)
 
     def barrier():
         if dist is not None:
@@ -202,9 +207,9 @@ def main():
     for i in range(args.steps):
         st.total_bytes.zero_()
         ev[3 * i].record()
-        ctx.encode(w["kv"], w["logits"], st)
+        ctx.encode(w["kv"], w["logits"], st, tokens=tok)
         ev[3 * i + 1].record()
-        ctx.decode(st, w["logits"], out)
+        ctx.decode(st, w["logits"], out, tokens=tok)
         ev[3 * i + 2].record()
         enc_k.append(ctx.last_kernel_ms(0)); dec_k.append(ctx.last_kernel_ms(1))
         if dense:
@@ -227,7 +232,7 @@ def main():
     # spot check of the decoded batch (outside the timed region)
     sel = torch.randint(0, n, (64,), device=dev)
     err = float((out[:, :, :, :, sel].float() - w["kv"][:, :, :, :, sel].float()).abs().max())
-    assert err <= cfg["delta"] / 2 + 1e-3 + 8 * 2 ** -11, err
+    assert err <= cfg["delta"] * (2.0 ** (args.adaptive - 1) if adaptive else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
 
     peak, peak_kind = measured_peaks()
     vecs = S * n * W
@@ -242,7 +247,7 @@ def main():
     fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
     fma_ach = vecs * K * d / (dom_ms / 1e3)
     dom_name = "encode_kernel" if dom_enc else "decode_kernel"
-    default_cfg = args.workload == "llama2-7b" and not over and not dense
+    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive
     traffic = NCU_DRAM_BYTES_PER_VECTOR[dom_name] * vecs if default_cfg else None
     roofline = {"kernel": dom_name, "bound": "hbm",
                 "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
@@ -269,7 +274,7 @@ def main():
                     "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step)
+        e2e = run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step, tok)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -287,7 +292,7 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
                        "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
-                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant,
+                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant, "adaptive_b0": args.adaptive,
                        "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
             "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
             "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),
@@ -361,7 +366,7 @@ def append_arm(args, torch, plc, workloads, dev):
     return 0
 
 
-def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step):
+def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step, tok=None):
     """Same step with HOST buffers: pinned inputs are copied in, the coded bytes and index are
     copied out and back in, the decoded KV is copied out -- all inside the timed region."""
     kv_h = w["kv"].cpu().pin_memory()
@@ -376,7 +381,7 @@ def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step):
     def step():
         kv_d.copy_(kv_h, non_blocking=True); lg_d.copy_(lg_h, non_blocking=True)
         st.total_bytes.zero_()
-        ctx.encode(kv_d, lg_d, st)
+        ctx.encode(kv_d, lg_d, st, tokens=tok)
         tot_h.copy_(st.total_bytes, non_blocking=True)
         torch.cuda.current_stream().synchronize()           # the byte count decides how much to copy out
         used = int(tot_h[0])
@@ -384,7 +389,7 @@ def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step):
         off_h.copy_(st.chunk_offset, non_blocking=True); nby_h.copy_(st.chunk_bytes, non_blocking=True)
         st.payload[:used].copy_(pay_h[:used], non_blocking=True)
         st.chunk_offset.copy_(off_h, non_blocking=True); st.chunk_bytes.copy_(nby_h, non_blocking=True)
-        ctx.decode(st, lg_d, out)
+        ctx.decode(st, lg_d, out, tokens=tok)
         kvo_h.copy_(out, non_blocking=True)
         return used
 

@@ -58,6 +58,12 @@ typedef struct {
     int32_t chunk_pos;
     int32_t variant;
     int32_t out_dtype;   /* dtype plc_decode writes: PLC_OUT_F32 or PLC_OUT_F16 */
+    /* Surprisal-adaptive quantiser (Def. 7 of the paper), used by plc_encode_adaptive /
+     * plc_decode_adaptive: adaptive_b0 > 0 turns it on; a position of surprisal h_i = -log2 P(x_i | x_<i)
+     * gets b_i = min(adaptive_b0 + adaptive_extra, max(1, floor(adaptive_b0 * h_i / adaptive_hbar)))
+     * bits, i.e. the step delta * 2^(adaptive_b0 - b_i).  0 <= adaptive_extra <= 12, adaptive_b0 <= 16. */
+    int32_t adaptive_b0, adaptive_extra;
+    float adaptive_hbar;
 } plc_config;
 
 /* A KV tensor indexed [layer][kv][session][head][position][d]; strides in ELEMENTS, the d
@@ -90,6 +96,7 @@ typedef struct {
     int32_t* sym_dev;
     int32_t* q_dev;
     float* mu_dev;
+    int32_t* bits_dev;   /* [S][n] int32: b_i of the adaptive quantiser (adaptive calls only) */
 } plc_debug_buffers;
 
 typedef struct {
@@ -164,6 +171,18 @@ plc_status plc_encode(plc_ctx* ctx, const plc_kv_view* kv, const void* logits_de
 plc_status plc_decode(plc_ctx* ctx, const plc_streams* in, const void* logits_dev, int32_t S, int32_t n,
                       const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
                       const plc_debug_buffers* dbg, void* stream);
+
+/* The same two calls with the surprisal-adaptive step of Def. 7 (cfg.adaptive_b0 > 0, top-K variant).
+ * tokens_dev [S][n] int32: the token at every position; both directions need it, because the step
+ * of position i depends on the surprisal of the token that actually occurred there.  Calling these
+ * with adaptive_b0 = 0, or plc_encode / plc_decode / plc_append_step with adaptive_b0 > 0, returns
+ * PLC_E_STATE. */
+plc_status plc_encode_adaptive(plc_ctx* ctx, const plc_kv_view* kv, const void* logits_dev, const int32_t* tokens_dev,
+                               int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                               const plc_streams* out, const plc_debug_buffers* dbg, void* stream);
+plc_status plc_decode_adaptive(plc_ctx* ctx, const plc_streams* in, const void* logits_dev, const int32_t* tokens_dev,
+                               int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                               const plc_kv_view* kv_out, const plc_debug_buffers* dbg, void* stream);
 
 /* Decode-time append (integration point 1 for one new token per session).  kv_step_dev
  * [L][2][B][H][d] f16, logits_step_dev [B][V] f16.  The new position's symbols and class go to the

@@ -21,7 +21,7 @@ OUT_F32, OUT_F16 = 0, 1
 EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_prefix_dedup", "plc_encode",
            "plc_decode", "plc_append_step", "plc_append_flush", "plc_append_sizes", "plc_sync_status",
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
-           "plc_launch_count", "plc_rans_encode_static"]
+           "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive"]
 
 
 def sources():
@@ -45,7 +45,8 @@ def build(force=False, verbose=False):
 class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("vocab", C.c_int32),
                 ("top_k", C.c_int32), ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32),
-                ("variant", C.c_int32), ("out_dtype", C.c_int32)]
+                ("variant", C.c_int32), ("out_dtype", C.c_int32), ("adaptive_b0", C.c_int32),
+                ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float)]
 
 
 class KVView(C.Structure):
@@ -59,7 +60,7 @@ class Streams(C.Structure):
 
 
 class DebugBuffers(C.Structure):
-    _fields_ = [("sym_dev", C.c_void_p), ("q_dev", C.c_void_p), ("mu_dev", C.c_void_p)]
+    _fields_ = [("sym_dev", C.c_void_p), ("q_dev", C.c_void_p), ("mu_dev", C.c_void_p), ("bits_dev", C.c_void_p)]
 
 
 class Stats(C.Structure):
@@ -138,11 +139,15 @@ class StreamSet:
 class Context:
     """One parameter set + candidate table T ([L][2][H][V][d] float16 on the device)."""
 
-    def __init__(self, T, top_k, delta, chunk_pos=256, sigma_floor=0.0, variant=PRED_TOPK, out_dtype=OUT_F32):
+    def __init__(self, T, top_k, delta, chunk_pos=256, sigma_floor=0.0, variant=PRED_TOPK, out_dtype=OUT_F32,
+                 adaptive=None):
+        """adaptive = (b0, extra, hbar) turns on the surprisal-adaptive step (Def. 7); encode / decode
+        then need the tokens."""
         L, two, H, V, d = T.shape
         assert two == 2 and T.is_cuda and T.is_contiguous()
         self.T = T
-        self.cfg = Config(L, H, d, V, top_k, delta, sigma_floor, chunk_pos, variant, out_dtype)
+        b0, extra, hbar = adaptive if adaptive else (0, 0, 0.0)
+        self.cfg = Config(L, H, d, V, top_k, delta, sigma_floor, chunk_pos, variant, out_dtype, b0, extra, hbar)
         self.W = 2 * L * H
         self._h = C.c_void_p()
         _check(lib().plc_create(C.byref(self._h), C.byref(self.cfg), _ptr(T)), "plc_create")
@@ -196,17 +201,27 @@ class Context:
                                       _ptr(dT), _ptr(parent), _ptr(shared), _stream()), "plc_prefix_dedup")
         return lcp, dT, parent, shared
 
-    def encode(self, kv, logits, streams, pos_begin=None, pos_end=None, debug=None):
+    def encode(self, kv, logits, streams, pos_begin=None, pos_end=None, debug=None, tokens=None):
         S, n = logits.shape[0], logits.shape[1]
         view = kv if isinstance(kv, KVView) else kv_view(kv)
         st = streams.c()
+        if tokens is not None:
+            _check(lib().plc_encode_adaptive(self._h, C.byref(view), _ptr(logits), _ptr(tokens), S, n, _ptr(pos_begin),
+                                             _ptr(pos_end), C.byref(st), None if debug is None else C.byref(debug),
+                                             _stream()), "plc_encode_adaptive")
+            return
         _check(lib().plc_encode(self._h, C.byref(view), _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end),
                                 C.byref(st), None if debug is None else C.byref(debug), _stream()), "plc_encode")
 
-    def decode(self, streams, logits, kv_out, pos_begin=None, pos_end=None, debug=None):
+    def decode(self, streams, logits, kv_out, pos_begin=None, pos_end=None, debug=None, tokens=None):
         S, n = logits.shape[0], logits.shape[1]
         view = kv_out if isinstance(kv_out, KVView) else kv_view(kv_out)
         st = streams.c()
+        if tokens is not None:
+            _check(lib().plc_decode_adaptive(self._h, C.byref(st), _ptr(logits), _ptr(tokens), S, n, _ptr(pos_begin),
+                                             _ptr(pos_end), C.byref(view), None if debug is None else C.byref(debug),
+                                             _stream()), "plc_decode_adaptive")
+            return
         _check(lib().plc_decode(self._h, C.byref(st), _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end),
                                 C.byref(view), None if debug is None else C.byref(debug), _stream()), "plc_decode")
 

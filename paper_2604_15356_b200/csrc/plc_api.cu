@@ -16,6 +16,7 @@ struct plc_ctx {
     const __half* T;
     float* rownorm2;
     int2* pairs;
+    int* step_exp;                  // [positions] adaptive step exponents
     long long pairs_cap;            // positions
     uint16_t* staging;
     unsigned long long staging_words_per_warp;
@@ -60,8 +61,10 @@ int padded_k(const plc_config& cfg) {
 plc_status ensure_pairs(plc_ctx* c, long long positions) {
     if (positions <= c->pairs_cap) return PLC_OK;
     if (c->pairs) cudaFree(c->pairs);
-    c->pairs = nullptr; c->pairs_cap = 0;
+    if (c->step_exp) cudaFree(c->step_exp);
+    c->pairs = nullptr; c->step_exp = nullptr; c->pairs_cap = 0;
     if (cudaMalloc(&c->pairs, sizeof(int2) * (size_t)positions * padded_k(c->cfg)) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaMalloc(&c->step_exp, sizeof(int) * (size_t)positions) != cudaSuccess) return PLC_E_CUDA;
     c->pairs_cap = positions;
     return PLC_OK;
 }
@@ -124,6 +127,9 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
     if (!(cfg->delta >= 1.0f / 4096.0f) || !(cfg->delta < 65536.0f) || !(cfg->sigma_floor >= 0.0f)) return PLC_E_INVALID;
     if (cfg->variant != PLC_PRED_TOPK && cfg->variant != PLC_PRED_DENSE) return PLC_E_INVALID;
     if (cfg->out_dtype != PLC_OUT_F32 && cfg->out_dtype != PLC_OUT_F16) return PLC_E_INVALID;
+    if (cfg->adaptive_b0 < 0 || cfg->adaptive_b0 > 16 || cfg->adaptive_extra < 0 || cfg->adaptive_extra > 12) return PLC_E_INVALID;
+    if (cfg->adaptive_b0 > 0 && !(cfg->adaptive_hbar > 0.0f)) return PLC_E_INVALID;
+    if (cfg->adaptive_b0 > 0 && cfg->variant != PLC_PRED_TOPK) return PLC_E_STATE;
     if (!aligned16(T_dev)) return PLC_E_ALIGN;
     plc_ctx* c = new (std::nothrow) plc_ctx();
     if (!c) return PLC_E_CUDA;
@@ -149,7 +155,7 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
 
 plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
-    cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->staging);
+    cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->step_exp); cudaFree(c->staging);
     cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch);
     for (int i = 0; i < 6; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
@@ -184,12 +190,16 @@ plc_status plc_prefix_dedup(plc_ctx* c, const int32_t* tokens_dev, const int32_t
 }
 
 static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n, const int32_t* pb, const int32_t* pe,
-                               cudaStream_t st) {
+                               cudaStream_t st, const int32_t* tokens = nullptr, int32_t* bits_out = nullptr) {
     plc_status rc = ensure_pairs(c, (long long)S * n);
     if (rc) return rc;
     TopkArgs a{};
     a.logits = static_cast<const __half*>(logits_dev); a.N = (long long)S * n; a.V = c->cfg.vocab; a.K = c->cfg.top_k;
     a.pairs = c->pairs; a.Kp = padded_k(c->cfg); a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
+    if (tokens) {
+        a.tokens = tokens; a.step_exp = c->step_exp; a.bits_out = bits_out;
+        a.b0 = c->cfg.adaptive_b0; a.extra = c->cfg.adaptive_extra; a.hbar = c->cfg.adaptive_hbar;
+    }
     return launch_topk(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
@@ -219,10 +229,12 @@ static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, boo
     return PLC_OK;
 }
 
-plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
-                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_streams* out,
-                      const plc_debug_buffers* dbg, void* stream) {
+// tokens_dev non-null <=> adaptive call
+static plc_status encode_impl(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, const int32_t* tokens_dev,
+                              int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                              const plc_streams* out, const plc_debug_buffers* dbg, void* stream) {
     if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
+    if ((c->cfg.adaptive_b0 > 0) != (tokens_dev != nullptr)) return PLC_E_STATE;
     plc_status rc = check_view(kv, c->cfg.head_dim, 2);
     if (rc) return rc;
     const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
@@ -237,19 +249,34 @@ plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev,
     a.st = to_dev(out);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, true, st);
-    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;
+    a.step_exp = tokens_dev ? c->step_exp : nullptr;
     if (c->profiling) cudaEventRecord(c->ev[0], st);
     cudaError_t e = launch_encode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[1], st); c->ev_valid[0] = 1; }
     return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
-plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev, int32_t S, int32_t n,
-                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
+plc_status plc_encode(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_streams* out,
                       const plc_debug_buffers* dbg, void* stream) {
+    return encode_impl(c, kv, logits_dev, nullptr, S, n, pos_begin_dev, pos_end_dev, out, dbg, stream);
+}
+
+plc_status plc_encode_adaptive(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, const int32_t* tokens_dev,
+                               int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                               const plc_streams* out, const plc_debug_buffers* dbg, void* stream) {
+    if (!tokens_dev) return PLC_E_INVALID;
+    return encode_impl(c, kv, logits_dev, tokens_dev, S, n, pos_begin_dev, pos_end_dev, out, dbg, stream);
+}
+
+static plc_status decode_impl(plc_ctx* c, const plc_streams* in, const void* logits_dev, const int32_t* tokens_dev,
+                              int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                              const plc_kv_view* kv_out, const plc_debug_buffers* dbg, void* stream) {
     if (!c || !logits_dev || S < 0 || n < 0) return PLC_E_INVALID;
+    if ((c->cfg.adaptive_b0 > 0) != (tokens_dev != nullptr)) return PLC_E_STATE;
     plc_status rc = check_view(kv_out, c->cfg.head_dim, c->cfg.out_dtype == PLC_OUT_F16 ? 2 : 4);
     if (rc) return rc;
     const int need = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
@@ -264,13 +291,27 @@ plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev,
     a.st = to_dev(in);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, false, st);
-    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st);
+    rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;
+    a.step_exp = tokens_dev ? c->step_exp : nullptr;
     if (c->profiling) cudaEventRecord(c->ev[2], st);
     cudaError_t e = launch_decode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[3], st); c->ev_valid[1] = 1; }
     return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_decode(plc_ctx* c, const plc_streams* in, const void* logits_dev, int32_t S, int32_t n,
+                      const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_kv_view* kv_out,
+                      const plc_debug_buffers* dbg, void* stream) {
+    return decode_impl(c, in, logits_dev, nullptr, S, n, pos_begin_dev, pos_end_dev, kv_out, dbg, stream);
+}
+
+plc_status plc_decode_adaptive(plc_ctx* c, const plc_streams* in, const void* logits_dev, const int32_t* tokens_dev,
+                               int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                               const plc_kv_view* kv_out, const plc_debug_buffers* dbg, void* stream) {
+    if (!tokens_dev) return PLC_E_INVALID;
+    return decode_impl(c, in, logits_dev, tokens_dev, S, n, pos_begin_dev, pos_end_dev, kv_out, dbg, stream);
 }
 
 plc_status plc_append_sizes(const plc_ctx* c, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes) {
@@ -292,7 +333,7 @@ static plc_status seal(plc_ctx* c, plc_session_batch* sb, int chunk_index, int c
 plc_status plc_append_step(plc_ctx* c, plc_session_batch* sb, const void* kv_step_dev, const void* logits_step_dev,
                            void* stream) {
     if (!c || !sb || !kv_step_dev || !logits_step_dev || !sb->open_sym_dev || !sb->open_q_dev) return PLC_E_INVALID;
-    if (c->cfg.variant != PLC_PRED_TOPK) return PLC_E_STATE;
+    if (c->cfg.variant != PLC_PRED_TOPK || c->cfg.adaptive_b0 > 0) return PLC_E_STATE;
     if (sb->B < 1 || sb->steps < 0) return PLC_E_INVALID;
     if (!aligned16(kv_step_dev)) return PLC_E_ALIGN;
     const int CP = c->cfg.chunk_pos;

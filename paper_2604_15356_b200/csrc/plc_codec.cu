@@ -509,12 +509,18 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                     buf ^= 1;
                     predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
                 }
-                q = scale_class(sigma2, floor2, inv_delta2);
+                float inv_delta_p = inv_delta, inv_delta2_p = inv_delta2;
+                if (a.step_exp) {                                                  // adaptive step delta * 2^e
+                    const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
+                    inv_delta_p = ldexpf(inv_delta, -e);
+                    inv_delta2_p = ldexpf(inv_delta2, -2 * e);
+                }
+                q = scale_class(sigma2, floor2, inv_delta2_p);
                 float kvv[G];
                 load_half_vec<G>(kvp, kvv);
                 kvp -= a.kv.sp;
 #pragma unroll
-                for (int g = 0; g < G; ++g) sym[g] = quantise(kvv[g], mu[g], inv_delta);
+                for (int g = 0; g < G; ++g) sym[g] = quantise(kvv[g], mu[g], inv_delta_p);
                 __syncwarp();                                                     // readers of this slot are done
                 if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
                     const long long o = ((long long)it.s * a.n + it.p0 + p) * Wt + it.t;
@@ -592,7 +598,13 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
                 buf ^= 1;
                 predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
             }
-            const int q = scale_class(sigma2, floor2, inv_delta2);
+            float delta_p = delta, inv_delta2_p = inv_delta2;
+            if (a.step_exp) {
+                const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
+                delta_p = ldexpf(delta, e);
+                inv_delta2_p = ldexpf(inv_delta2, -2 * e);
+            }
+            const int q = scale_class(sigma2, floor2, inv_delta2_p);
             __syncwarp();                                                         // readers of this slot are done
             int s, qp;
             class_params(q, s, qp);
@@ -604,7 +616,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 sym[g] = decode_step(pc, cum, fcs, x, words, rp, nwords, lane, lt, bad);
-                out[g] = __fmaf_rn((float)sym[g], delta, mu[g]);
+                out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
             }
             store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
             kvo += a.kv.sp;

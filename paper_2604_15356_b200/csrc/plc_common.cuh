@@ -151,6 +151,8 @@ struct TopkArgs {
     int2* pairs;            // [N][Kp] {idx, float bits of w}, or null; entries K..Kp-1 get {idx_0, 0}
     int Kp;
     int32_t* idx; float* w; float* lse; float* zk; float* logp2;   // optional user outputs
+    // Adaptive step (needs tokens): step_exp[row] = b0 - b_i, bits_out[row] = b_i (both optional).
+    int* step_exp; int* bits_out; int b0, extra; float hbar;
     // Rows are skipped (nothing written) when pos ranges are given and the row is outside them.
     int n_per_session; const int32_t* pos_begin; const int32_t* pos_end;
 };
@@ -181,7 +183,8 @@ struct DebugDev {
 struct CodecArgs {
     CodecShape sh;
     const __half* T; const float* rownorm2;        // [tables][V][d], [tables][V]
-    const int2* pairs;                             // [S*n][K]
+    const int2* pairs;                             // [S*n][Kp]
+    const int* step_exp;                           // [S*n] adaptive step exponent, or null
     KvView kv;                                     // encode: input f16; decode: output
     int S, n; const int32_t* pos_begin; const int32_t* pos_end;
     StreamsDev st; DebugDev dbg;

@@ -266,10 +266,18 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
             float lse = lmax + logf(sum_all);
             if (a.lse) a.lse[rowi] = lse;
             if (a.zk) a.zk[rowi] = sum_k / sum_all;
-            if (a.logp2 && a.tokens) {
-                int tk = a.tokens[rowi];
-                float v = (tk >= 0 && tk < V) ? (__half2float(row[tk]) - lse) * 1.44269504088896341f : __int_as_float(0x7fc00000);
-                a.logp2[rowi] = v;
+            if (a.tokens && (a.logp2 || a.step_exp || a.bits_out)) {
+                const int tk = a.tokens[rowi];
+                const float v = (tk >= 0 && tk < V) ? (__half2float(row[tk]) - lse) * 1.44269504088896341f : __int_as_float(0x7fc00000);
+                if (a.logp2) a.logp2[rowi] = v;
+                if (a.step_exp || a.bits_out) {
+                    // Def. 7: b = max(1, floor(b0 h / hbar)), capped at b0 + extra; decided in binary32
+                    const float r = __fmul_rn((float)a.b0, __fdiv_rn(-v, a.hbar));
+                    int b = (r >= 1.0f) ? (int)floorf(r) : 1;
+                    b = min(b, a.b0 + a.extra);
+                    if (a.step_exp) a.step_exp[rowi] = a.b0 - b;
+                    if (a.bits_out) a.bits_out[rowi] = b;
+                }
             }
         }
         __syncthreads();

@@ -420,3 +420,64 @@ def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
     assert ctx.sync_status() == plc.OK
     assert torch.equal(sym2, sym)
     assert float((out.cpu() - kv.float()).abs().max()) <= delta / 2 + 1e-3
+
+
+def test_adaptive_quantiser_parity(dev, orc):
+    """Def. 7: per-position step delta * 2^(b0 - b_i), b_i from the surprisal of the actual token.
+    b_i is an integer decided in binary32 from a binary32 surprisal, so a position may get a different
+    depth than the oracle's only where b0 h / hbar is within 1e-4 of an integer; positions whose depth
+    agrees are held to the usual tolerances."""
+    S, n, L, H, d, V, K, CP, delta = 2, 150, 1, 2, 128, 1024, 32, 64, 0.02
+    tokens, logits, T, kv = make_workload(501, S, n, L, H, d, V, K, pp=10.0)
+    _, _, _, _, lp = orc.topk_softmax(logits.numpy().reshape(S * n, V), tokens.numpy().reshape(-1), K)
+    b0, extra, hbar = 6, 5, float(-lp.mean())
+    ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, adaptive=(b0, extra, hbar))
+    W, mc = ctx.W, ctx.max_chunks(n)
+    st = plc.StreamSet(S * W, mc, S * W * mc * 160 + 4 * S * n * W * d + 4096, dev)
+    sym = torch.zeros(S, n, W, d, dtype=torch.int32, device=dev)
+    q = torch.zeros(S, n, W, dtype=torch.int32, device=dev)
+    mu = torch.zeros(S, n, W, d, dtype=torch.float32, device=dev)
+    bits = torch.zeros(S, n, dtype=torch.int32, device=dev)
+    kvd, lgd, tkd = kv.to(dev), logits.to(dev), tokens.to(dev)
+    dbg = plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr(), bits.data_ptr())
+    with pytest.raises(plc.PlcError):
+        ctx.encode(kvd, lgd, st, debug=dbg)                       # adaptive context needs the tokens
+    ctx.encode(kvd, lgd, st, debug=dbg, tokens=tkd)
+    assert ctx.sync_status() == plc.OK
+    cfg = orc.Config(L, H, d, V, K, delta, 0.0, CP, 0, b0, extra, hbar)
+    enc = orc.encode(cfg, T.numpy(), kv.numpy(), logits.numpy(), tokens.numpy(), export=True)
+    bits_g, bits_o = bits.cpu().numpy(), enc["bits"]
+    same = bits_g == bits_o
+    assert same.mean() > 0.99 and len(set(bits_o.reshape(-1).tolist())) > 4
+    if not same.all():
+        r = b0 * (-lp.reshape(S, n)) / hbar
+        assert np.abs(r - np.rint(r))[~same].max() < 1e-4 and np.abs(bits_g - bits_o).max() == 1
+    sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W); mu_o = enc["mu"].reshape(S, n, W, d)
+    sym_g, q_g, mu_g = sym.cpu().numpy(), q.cpu().numpy(), mu.cpu().numpy()
+    scale = np.maximum(np.abs(mu_o).max(-1), 1e-3)
+    assert (np.abs(mu_g - mu_o).max(-1) <= 1e-3 * scale).all()
+    assert (sym_g[same] != sym_o[same]).mean() < 1e-4
+    assert (q_g[same] != q_o[same]).mean() < 1e-2
+    total = 0
+    for s_ in range(S):
+        for t_ in range(W):
+            for c in range(mc):
+                P = min(CP, n - c * CP)
+                ref, _, _ = orc.rans_encode_chunk(sym_g[s_, c * CP:c * CP + P, t_], q_g[s_, c * CP:c * CP + P, t_])
+                assert np.array_equal(st.chunk((s_ * W + t_) * mc + c), ref), (s_, t_, c)
+                total += len(ref)
+    if same.all():
+        assert abs(total / enc["stats"].payload_bytes - 1) < 1e-3
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    sym2 = torch.zeros_like(sym)
+    with pytest.raises(plc.PlcError):
+        ctx.decode(st, lgd, out)
+    ctx.decode(st, lgd, out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None, None), tokens=tkd)
+    assert ctx.sync_status() == plc.OK and torch.equal(sym2, sym)
+    err = (out.cpu() - kv.float()).abs().permute(2, 4, 0, 1, 3, 5).reshape(S, n, -1).max(-1).values.numpy()
+    step = delta * 2.0 ** (b0 - bits_g)
+    assert np.all(err <= step / 2 + 1e-3)                         # Prop. 3 with each position's own step
+    # a fixed-step context refuses the adaptive calls
+    plain = plc.Context(T.to(dev), K, delta, chunk_pos=CP)
+    with pytest.raises(plc.PlcError):
+        plain.encode(kvd, lgd, st, tokens=tkd)
