@@ -124,6 +124,7 @@ def main():
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--chunk-pos", type=int, default=None)
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-groups", type=int, default=4, help="layer groups (streams) of the host-buffer step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--set", action="append", default=[], help="override a workload field, e.g. --set L=4")
@@ -274,7 +275,13 @@ def main():
                     "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step, tok)
+        del out, st
+        torch.cuda.empty_cache()
+
+        def make_ctx(Tslice):
+            return plc.Context(Tslice, K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                               variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive)
+        e2e = run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok, args.e2e_groups)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -366,34 +373,68 @@ def append_arm(args, torch, plc, workloads, dev):
     return 0
 
 
-def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step, tok=None):
+def run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None, groups=4):
     """Same step with HOST buffers: pinned inputs are copied in, the coded bytes and index are
-    copied out and back in, the decoded KV is copied out -- all inside the timed region."""
+    copied out and back in, the decoded KV is copied out -- all inside the timed region.  The
+    layers are cut into groups, each with its own context and CUDA stream, so that the copies of
+    one group overlap the kernels and the opposite-direction copies of the others."""
+    cfg = w["cfg"]
+    S, n, L, H, d = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"]
+    G = groups if (L % groups == 0 and args.variant == "topk") else 1
+    Lg = L // G
     kv_h = w["kv"].cpu().pin_memory()
     lg_h = w["logits"].cpu().pin_memory()
-    pay_h = torch.empty(st.payload.numel(), dtype=torch.uint8).pin_memory()
-    off_h = torch.empty_like(st.chunk_offset, device="cpu").pin_memory()
-    nby_h = torch.empty_like(st.chunk_bytes, device="cpu").pin_memory()
-    tot_h = torch.zeros(1, dtype=torch.int64).pin_memory()
     kvo_h = torch.empty_like(kv_h).pin_memory()
-    kv_d, lg_d = torch.empty_like(w["kv"]), torch.empty_like(w["logits"])
+    kv_d, lg_d, out_d = torch.empty_like(w["kv"]), torch.empty_like(w["logits"]), torch.empty_like(w["kv"])
+    ctxs, sts, pay_h, off_h, nby_h, tot_h, streams = [], [], [], [], [], [], []
+    for g in range(G):
+        c = make_ctx(w["T"][g * Lg:(g + 1) * Lg])
+        c.reserve(S * n)
+        ctxs.append(c)
+        st = plc.StreamSet(S * c.W, c.max_chunks(n), int(0.70 * kv_h.numel() * 2 / G) + (1 << 20), dev)
+        sts.append(st)
+        pay_h.append(torch.empty(st.payload.numel(), dtype=torch.uint8).pin_memory())
+        off_h.append(torch.empty_like(st.chunk_offset, device="cpu").pin_memory())
+        nby_h.append(torch.empty_like(st.chunk_bytes, device="cpu").pin_memory())
+        tot_h.append(torch.zeros(1, dtype=torch.int64).pin_memory())
+        streams.append(torch.cuda.Stream(device=dev))
+    ev0 = torch.cuda.Event()
 
     def step():
-        kv_d.copy_(kv_h, non_blocking=True); lg_d.copy_(lg_h, non_blocking=True)
-        st.total_bytes.zero_()
-        ctx.encode(kv_d, lg_d, st, tokens=tok)
-        tot_h.copy_(st.total_bytes, non_blocking=True)
-        torch.cuda.current_stream().synchronize()           # the byte count decides how much to copy out
-        used = int(tot_h[0])
-        pay_h[:used].copy_(st.payload[:used], non_blocking=True)
-        off_h.copy_(st.chunk_offset, non_blocking=True); nby_h.copy_(st.chunk_bytes, non_blocking=True)
-        st.payload[:used].copy_(pay_h[:used], non_blocking=True)
-        st.chunk_offset.copy_(off_h, non_blocking=True); st.chunk_bytes.copy_(nby_h, non_blocking=True)
-        ctx.decode(st, lg_d, out, tokens=tok)
-        kvo_h.copy_(out, non_blocking=True)
-        return used
+        main = torch.cuda.current_stream()
+        lg_d.copy_(lg_h, non_blocking=True)
+        ev0.record(main)
+        for g in range(G):
+            lo, hi = g * Lg, (g + 1) * Lg
+            with torch.cuda.stream(streams[g]):
+                streams[g].wait_event(ev0)
+                kv_d[lo:hi].copy_(kv_h[lo:hi], non_blocking=True)
+                sts[g].total_bytes.zero_()
+                ctxs[g].encode(kv_d[lo:hi], lg_d, sts[g], tokens=tok)
+                tot_h[g].copy_(sts[g].total_bytes, non_blocking=True)
+        used_all = 0
+        for g in range(G):
+            lo, hi = g * Lg, (g + 1) * Lg
+            streams[g].synchronize()                          # the byte count decides how much to copy out
+            used = int(tot_h[g][0]); used_all += used
+            st = sts[g]
+            with torch.cuda.stream(streams[g]):
+                pay_h[g][:used].copy_(st.payload[:used], non_blocking=True)
+                off_h[g].copy_(st.chunk_offset, non_blocking=True); nby_h[g].copy_(st.chunk_bytes, non_blocking=True)
+                st.payload[:used].copy_(pay_h[g][:used], non_blocking=True)
+                st.chunk_offset.copy_(off_h[g], non_blocking=True); st.chunk_bytes.copy_(nby_h[g], non_blocking=True)
+                ctxs[g].decode(st, lg_d, out_d[lo:hi], tokens=tok)
+                kvo_h[lo:hi].copy_(out_d[lo:hi], non_blocking=True)
+        for g in range(G):
+            main.wait_stream(streams[g])
+        return used_all
 
     used = step()
+    torch.cuda.synchronize()
+    for c in ctxs:
+        assert c.sync_status() == plc.OK
+    err = float((kvo_h[:, :, :, :, :64].float() - kv_h[:, :, :, :, :64].float()).abs().max())
+    assert err <= cfg["delta"] * (2.0 ** (args.adaptive - 1) if args.adaptive > 0 else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
@@ -404,10 +445,11 @@ def run_e2e(args, torch, ctx, st, w, out, dev, world, dist, tokens_per_step, tok
     t1.record()
     torch.cuda.synchronize()
     ms = max_over_ranks(t0.elapsed_time(t1) / args.e2e_steps, dist, dev)
-    idx_bytes = off_h.numel() * 8 + nby_h.numel() * 4
+    idx_bytes = sum(o.numel() * 8 + b.numel() * 4 for o, b in zip(off_h, nby_h))
     return {"value": job_value(world, tokens_per_step, ms), "unit": UNIT, "ms_per_step": ms,
             "h2d_bytes_per_step": kv_h.numel() * 2 + lg_h.numel() * 2 + used + idx_bytes,
-            "d2h_bytes_per_step": used + idx_bytes + 8 + kvo_h.numel() * 2, "steps": args.e2e_steps}
+            "d2h_bytes_per_step": used + idx_bytes + 8 * G + kvo_h.numel() * 2, "steps": args.e2e_steps,
+            "layer_groups": G}
 
 
 def reference_arm(args, workloads):
