@@ -191,7 +191,7 @@ def test_tiny_config_full_parity(dev, orc):
 
 
 @pytest.mark.parametrize("d,K,V,n,CP", [(128, 64, 2000, 300, 128), (32, 7, 64, 70, 32), (256, 20, 512, 45, 16),
-                                        (64, 64, 4096, 130, 64)])
+                                        (64, 64, 4096, 130, 64), (64, 301, 512, 40, 16), (128, 1024, 1024, 20, 8)])
 def test_multi_stream_ragged_parity(dev, orc, d, K, V, n, CP):
     tokens, logits, T, kv = make_workload(100 + d, 2, n, 2, 2, d, V, K, pp=15.0, alpha=1.1 if d == 128 else 0.0)
     g = gpu_encode(dev, T, kv, logits, K, 0.02, CP)
