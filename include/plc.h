@@ -153,6 +153,27 @@ plc_status plc_prefix_dedup(plc_ctx* ctx, const int32_t* tokens_dev, const int32
                             int32_t S, int64_t token_stride, int32_t* lcp_dev, float* dT_dev, int32_t* parent_dev,
                             int32_t* shared_len_dev, void* stream);
 
+/* Trie-based prefix index of Sec. 7.3 (host side; all pointers are HOST memory): stored session
+ * prefixes with insert, best-match lookup and evict, each one walk along a root-to-node path.
+ * epsilon > 0 prunes the trie at nodes whose probability P(prefix) = prod_j P(x_j | x_<j) (Def. 1)
+ * is below epsilon: a prefix is kept only down to its deepest node with P >= epsilon.
+ *   insert: id must be new (PLC_E_STATE otherwise); logp2[j] = log2 P(tokens[j] | tokens[<j]);
+ *           *stored_len (optional) = number of tokens kept.
+ *   best_match: follows the query until it leaves all stored paths and reports the deepest stored
+ *           ancestor: *lcp its depth, *dT = -log2 P of that common prefix (Def. 2), *id one stored
+ *           prefix passing through it (the lexicographically smallest stored continuation, then the
+ *           smallest id); *id = -1 when nothing is stored.
+ *   evict: removes a stored prefix and the nodes no other prefix uses (PLC_E_INVALID if unknown). */
+typedef struct plc_trie plc_trie;
+plc_status plc_trie_create(plc_trie** out, float epsilon);
+plc_status plc_trie_destroy(plc_trie* trie);
+plc_status plc_trie_insert(plc_trie* trie, int32_t id, const int32_t* tokens, const float* logp2, int32_t len,
+                           int32_t* stored_len);
+plc_status plc_trie_best_match(const plc_trie* trie, const int32_t* tokens, int32_t len, int32_t* id, int32_t* lcp,
+                               float* dT);
+plc_status plc_trie_evict(plc_trie* trie, int32_t id);
+plc_status plc_trie_stats(const plc_trie* trie, int64_t* n_nodes, int64_t* n_prefixes);
+
 /* Integration point 1 of Sec. 7.2: before KV_i is written, predict it, subtract (Def. 6), quantise
  * and code the residual -- for every position in [pos_begin[s], pos_end[s]) of every session and
  * every stream.  logits_dev [S][n][V] f16, logits[s][i] being the distribution over token i.

@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INC = os.path.join(os.path.dirname(_HERE), "include")
 _SO = os.path.join(_HERE, "libplc.so")
-_SOURCES = ["plc_api.cu", "plc_topk.cu", "plc_prefix.cu", "plc_codec.cu", "plc_dense.cu", "plc_static.cu"]
+_SOURCES = ["plc_api.cu", "plc_topk.cu", "plc_prefix.cu", "plc_codec.cu", "plc_dense.cu", "plc_static.cu", "plc_trie.cu"]
 
 OK, E_INVALID, E_SHAPE, E_ALIGN, E_CAPACITY, E_CORRUPT, E_STATE, E_CUDA = range(8)
 PRED_TOPK, PRED_DENSE = 0, 1
@@ -21,7 +21,9 @@ OUT_F32, OUT_F16 = 0, 1
 EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_prefix_dedup", "plc_encode",
            "plc_decode", "plc_append_step", "plc_append_flush", "plc_append_sizes", "plc_sync_status",
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
-           "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive"]
+           "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
+           "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
+           "plc_trie_stats"]
 
 
 def sources():
@@ -275,6 +277,46 @@ def rans_encode_static(sym, q, n_pos, chunk_index, streams, status):
     st = streams.c()
     return lib().plc_rans_encode_static(_ptr(sym), _ptr(q), n_streams, int(n_pos), d, cap, int(chunk_index),
                                         C.byref(st), _ptr(status), _stream())
+
+
+class TrieIndex:
+    """Host-side prefix index (Sec. 7.3): insert / best_match / evict over numpy int32 token arrays."""
+
+    def __init__(self, epsilon=0.0):
+        self._h = C.c_void_p()
+        _check(lib().plc_trie_create(C.byref(self._h), C.c_float(epsilon)), "plc_trie_create")
+
+    def __del__(self):
+        try:
+            if self._h:
+                lib().plc_trie_destroy(self._h)
+                self._h = C.c_void_p()
+        except Exception:
+            pass
+
+    def insert(self, ident, tokens, logp2):
+        import numpy as np
+        tk = np.ascontiguousarray(tokens, dtype=np.int32); lp = np.ascontiguousarray(logp2, dtype=np.float32)
+        kept = C.c_int32()
+        _check(lib().plc_trie_insert(self._h, int(ident), tk.ctypes.data_as(C.c_void_p), lp.ctypes.data_as(C.c_void_p),
+                                     len(tk), C.byref(kept)), "plc_trie_insert")
+        return kept.value
+
+    def best_match(self, tokens):
+        import numpy as np
+        tk = np.ascontiguousarray(tokens, dtype=np.int32)
+        ident, lcp, dT = C.c_int32(), C.c_int32(), C.c_float()
+        _check(lib().plc_trie_best_match(self._h, tk.ctypes.data_as(C.c_void_p), len(tk), C.byref(ident), C.byref(lcp),
+                                         C.byref(dT)), "plc_trie_best_match")
+        return ident.value, lcp.value, dT.value
+
+    def evict(self, ident):
+        _check(lib().plc_trie_evict(self._h, int(ident)), "plc_trie_evict")
+
+    def stats(self):
+        a, b = C.c_int64(), C.c_int64()
+        _check(lib().plc_trie_stats(self._h, C.byref(a), C.byref(b)), "plc_trie_stats")
+        return a.value, b.value
 
 
 def table_constants(qp):
