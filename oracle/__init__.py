@@ -31,7 +31,8 @@ def build(force=False):
 class Config(C.Structure):
     _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("K", C.c_int32),
                 ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32), ("dense", C.c_int32),
-                ("adaptive_b0", C.c_int32), ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float)]
+                ("adaptive_b0", C.c_int32), ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float),
+                ("lin_dm", C.c_int32), ("lin_E", C.c_void_p), ("lin_A", C.c_void_p), ("lin_c", C.c_void_p)]
 
 
 class KVStrides(C.Structure):
@@ -129,6 +130,40 @@ def adaptive_bits(h, b0, hbar, extra):
     return lib().plo_adaptive_bits(C.c_float(h), int(b0), C.c_float(hbar), int(extra))
 
 
+def linear_config(L, H, d, V, K, delta, chunk_pos, E, A, c):
+    """Config of the linear-embedding predictor (Sec. 7.1): E [V,dm], A [L,2,H,d,dm], c [L,2,H,d], all float16.
+    The arrays are kept alive on the returned object."""
+    Eb, Ab, cb = _h(E), _h(A), _h(c)
+    cfg = Config(L, H, d, V, K, delta, 0.0, chunk_pos, 2, 0, 0, 0.0, Eb.shape[1], Eb.ctypes.data, Ab.ctypes.data, cb.ctypes.data)
+    cfg._keep = (Eb, Ab, cb)
+    return cfg
+
+
+def expected_embedding(E, logits_row, lse):
+    Eb = _h(E); lg = _h(logits_row)
+    V, dm = Eb.shape
+    out = np.zeros(dm, np.float64)
+    lib().plo_expected_embedding(_p(Eb), V, dm, _p(lg), C.c_double(lse), _p(out))
+    return out
+
+
+def linear_apply(A, c, x):
+    Ab, cb = _h(A), _h(c)
+    d, dm = Ab.shape
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.zeros(d, np.float64)
+    lib().plo_linear_apply(_p(Ab), _p(cb), d, dm, _p(x), _p(out))
+    return out
+
+
+def linear_rownorms(E, A, c):
+    Eb, Ab, cb = _h(E), _h(A), _h(c)
+    V, dm = Eb.shape
+    out = np.zeros(V, np.float64)
+    lib().plo_linear_rownorms(_p(Eb), _p(Ab), _p(cb), V, Ab.shape[0], dm, _p(out))
+    return out
+
+
 def quantise(kv, mu, delta):
     x = _h(kv)
     mu = np.ascontiguousarray(mu, dtype=np.float64)
@@ -222,8 +257,12 @@ def encode(cfg, T, kv, logits, tokens, pos_begin=None, pos_end=None, export=Fals
     logits [S,n,V] f16; tokens [S,n] i32 or None.  Returns a dict with payload, chunk_offset,
     chunk_bytes ([S,L,2,H,max_chunks]), stats and, with export=True, sym/q/mu ([S,n,L,2,H(,d)]).
     """
-    Tb = _h(T)
-    L, _, H, V, d = Tb.shape
+    if T is None:                                   # linear-embedding predictor: shapes come from the config
+        Tb = None
+        L, H, V, d = cfg.L, cfg.H, cfg.V, cfg.d
+    else:
+        Tb = _h(T)
+        L, _, H, V, d = Tb.shape
     assert kv.dtype == np.float16 and kv.strides[-1] == 2
     kvv = kv.view(np.uint16)
     lg = _h(logits)
@@ -257,7 +296,7 @@ def encode(cfg, T, kv, logits, tokens, pos_begin=None, pos_end=None, export=Fals
 
 def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=False, tokens=None):
     """Whole-path decode of the dict ``encode`` returned.  kv_shape = (L,2,S,H,n,d); returns float32 KV'."""
-    Tb = _h(T)
+    Tb = None if T is None else _h(T)
     lg = _h(logits)
     S, n, _ = lg.shape
     pb = None if pos_begin is None else np.ascontiguousarray(pos_begin, dtype=np.int32)

@@ -176,6 +176,56 @@ void plo_dense_mixture(const uint16_t* table /*[V][d]*/, int V, int d, const uin
     *sigma2 = r > 0.0 ? r : 0.0;
 }
 
+/* Linear embedding approximation (Sec. 7.1): F(t_<i, t) ~ c + A E(t), hence
+ *   KV^ ~ c + A Ebar,  Ebar = E_{t ~ P}[E(t)] = sum_v p_v E(v),
+ * "a single weighted sum over the vocabulary using the softmax output".  In the arithmetic of two
+ * chained bf16 contractions: p_v, E and A are rounded to bfloat16, Ebar is summed exactly and then
+ * rounded to bfloat16 itself (it is the input of the second contraction), mu = c + A Ebar exactly. */
+void plo_expected_embedding(const uint16_t* E /*[V][dm]*/, int V, int dm, const uint16_t* logits, double lse, double* ebar) {
+    for (int k = 0; k < dm; ++k) ebar[k] = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double p = round_bf16(exp(half_to_double(logits[v]) - lse));
+        const uint16_t* row = E + (size_t)v * dm;
+        for (int k = 0; k < dm; ++k) ebar[k] += p * round_bf16(half_to_double(row[k]));
+    }
+    for (int k = 0; k < dm; ++k) ebar[k] = round_bf16(ebar[k]);
+}
+
+/* out[j] = c[j] + sum_k bf16(A[j][k]) x[k]   (x already on the bf16 grid) */
+void plo_linear_apply(const uint16_t* A /*[d][dm]*/, const uint16_t* c /*[d]*/, int d, int dm, const double* x, double* out) {
+    for (int j = 0; j < d; ++j) {
+        double s = half_to_double(c[j]);
+        for (int k = 0; k < dm; ++k) s += round_bf16(half_to_double(A[(size_t)j * dm + k])) * x[k];
+        out[j] = s;
+    }
+}
+
+/* n2b[v] = bf16(||c + A E(v)||^2 / d): squared norm of the linear model's own candidate vector. */
+void plo_linear_rownorms(const uint16_t* E, const uint16_t* A, const uint16_t* c, int V, int d, int dm, double* n2b) {
+    double* x = (double*)malloc(sizeof(double) * (size_t)dm);
+    double* t = (double*)malloc(sizeof(double) * (size_t)d);
+    for (int v = 0; v < V; ++v) {
+        for (int k = 0; k < dm; ++k) x[k] = round_bf16(half_to_double(E[(size_t)v * dm + k]));
+        plo_linear_apply(A, c, d, dm, x, t);
+        double n2 = 0.0;
+        for (int j = 0; j < d; ++j) n2 += t[j] * t[j];
+        n2b[v] = round_bf16(n2 / d);
+    }
+    free(x); free(t);
+}
+
+/* Prediction and variance of one (table, position) under the linear model:
+ *   sigma2 = max(0, sum_v bf16(p_v) n2b[v] - ||mu||^2 / d)   (Thm. 2 with F := c + A E) */
+void plo_linear_mixture(const uint16_t* A, const uint16_t* c, int V, int d, int dm, const uint16_t* logits, double lse,
+                        const double* ebar, const double* n2b, double* mu, double* sigma2) {
+    plo_linear_apply(A, c, d, dm, ebar, mu);
+    double s = 0.0, m2 = 0.0;
+    for (int v = 0; v < V; ++v) s += round_bf16(exp(half_to_double(logits[v]) - lse)) * n2b[v];
+    for (int j = 0; j < d; ++j) m2 += mu[j] * mu[j];
+    double r = s - m2 / d;
+    *sigma2 = r > 0.0 ? r : 0.0;
+}
+
 /* ---------------------------------------------------------------- scale class */
 
 /* Class of the per-position scale: q = clamp(round(8 log2(sigma_tot / delta)), -24, 135) with
@@ -504,6 +554,11 @@ typedef struct {
     int32_t adaptive_b0;    /* > 0: surprisal-adaptive step (Def. 7) with target depth b0 */
     int32_t adaptive_extra; /* cap: b_i <= b0 + adaptive_extra */
     float adaptive_hbar;    /* average surprisal h-bar, bits */
+    /* dense == 2: linear-embedding predictor F(t) ~ c + A E(t) (Sec. 7.1); T is not used */
+    int32_t lin_dm;               /* embedding width d_model */
+    const uint16_t* lin_E;        /* [V][dm] f16 token embeddings */
+    const uint16_t* lin_A;        /* [L][2][H][d][dm] f16 */
+    const uint16_t* lin_c;        /* [L][2][H][d] f16 */
 } plo_config;
 
 typedef struct {
@@ -558,13 +613,26 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
             }
         }
         stats->coded_positions += (uint64_t)(e - b);
+        const int lin = cfg->dense == 2, dm = cfg->lin_dm;
+        double* ebar = NULL; double* n2b = NULL;
+        if (lin) {
+            ebar = (double*)malloc(sizeof(double) * (size_t)n * dm);
+            n2b = (double*)malloc(sizeof(double) * (size_t)V);
+            for (int i = b; i < e; ++i)
+                plo_expected_embedding(cfg->lin_E, V, dm, logits + ((size_t)s * n + i) * V, lse[i], ebar + (size_t)i * dm);
+        }
         for (int l = 0; l < L && !rc; ++l) for (int a = 0; a < 2 && !rc; ++a) for (int h = 0; h < H && !rc; ++h) {
-            const uint16_t* table = T + ((((size_t)l * 2 + a) * H + h) * (size_t)V) * d;
+            const size_t tix = ((size_t)l * 2 + a) * H + h;
+            const uint16_t* table = lin ? NULL : T + (tix * (size_t)V) * d;
+            const uint16_t* At = lin ? cfg->lin_A + tix * (size_t)d * dm : NULL;
+            const uint16_t* ct = lin ? cfg->lin_c + tix * (size_t)d : NULL;
+            if (lin) plo_linear_rownorms(cfg->lin_E, At, ct, V, d, dm, n2b);
             for (int ch = 0; b + ch * CP < e; ++ch) {
                 int p0 = b + ch * CP, P = e - p0 < CP ? e - p0 : CP;
                 for (int p = 0; p < P; ++p) {
                     int i = p0 + p; double s2;
-                    if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mu, &s2);
+                    if (lin) plo_linear_mixture(At, ct, V, d, dm, logits + ((size_t)s * n + i) * V, lse[i], ebar + (size_t)i * dm, n2b, mu, &s2);
+                    else if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mu, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mu, &s2);
                     cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
                     const uint16_t* x = kv + l * st->layer + a * st->kv + s * st->session + h * st->head + (int64_t)i * st->pos;
@@ -584,6 +652,7 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
                 stats->ideal_bits += ideal; stats->payload_bytes += nb; stats->n_chunks++; stats->n_escapes += nesc;
             }
         }
+        free(ebar); free(n2b);
     }
     free(idx); free(w); free(lse); free(zk); free(lp); free(csym); free(cq); free(mu); free(pdelta);
     return rc;
@@ -620,13 +689,26 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                 pdelta[i] = ldexpf(cfg->delta, cfg->adaptive_b0 - bi);
             }
         }
+        const int lin = cfg->dense == 2, dm = cfg->lin_dm;
+        double* ebar = NULL; double* n2b = NULL;
+        if (lin) {
+            ebar = (double*)malloc(sizeof(double) * (size_t)n * dm);
+            n2b = (double*)malloc(sizeof(double) * (size_t)V);
+            for (int i = b; i < e; ++i)
+                plo_expected_embedding(cfg->lin_E, V, dm, logits + ((size_t)s * n + i) * V, lse[i], ebar + (size_t)i * dm);
+        }
         for (int l = 0; l < L && !rc; ++l) for (int a = 0; a < 2 && !rc; ++a) for (int h = 0; h < H && !rc; ++h) {
-            const uint16_t* table = T + ((((size_t)l * 2 + a) * H + h) * (size_t)V) * d;
+            const size_t tix = ((size_t)l * 2 + a) * H + h;
+            const uint16_t* table = lin ? NULL : T + (tix * (size_t)V) * d;
+            const uint16_t* At = lin ? cfg->lin_A + tix * (size_t)d * dm : NULL;
+            const uint16_t* ct = lin ? cfg->lin_c + tix * (size_t)d : NULL;
+            if (lin) plo_linear_rownorms(cfg->lin_E, At, ct, V, d, dm, n2b);
             for (int ch = 0; b + ch * CP < e; ++ch) {
                 int p0 = b + ch * CP, P = e - p0 < CP ? e - p0 : CP;
                 for (int p = 0; p < P; ++p) {
                     int i = p0 + p; double s2;
-                    if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mus + (size_t)p * d, &s2);
+                    if (lin) plo_linear_mixture(At, ct, V, d, dm, logits + ((size_t)s * n + i) * V, lse[i], ebar + (size_t)i * dm, n2b, mus + (size_t)p * d, &s2);
+                    else if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mus + (size_t)p * d, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mus + (size_t)p * d, &s2);
                     cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
                 }
@@ -644,6 +726,7 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                 }
             }
         }
+        free(ebar); free(n2b);
     }
     free(idx); free(w); free(lse); free(csym); free(cq); free(mus); free(pdelta);
     return rc;

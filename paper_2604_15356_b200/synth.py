@@ -191,3 +191,32 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
             start = tokens[s, pos - 1:pos].to(torch.int64)
             tokens[s, pos:] = sample_tokens(table, 1, n - pos, seed * 1000 + 500 + s, start=start)[0]
     return tokens, prefix_keys(tokens), leaf, plen
+
+
+def make_linear_model(L, H, V, d, dm, seed, device="cpu"):
+    """Parameters of a KV function that is linear in the token embedding, F(t) = c + A E(t):
+    E [V][dm] ~ N(0,1), A [L][2][H][d][dm] ~ N(0, 1/dm), c [L][2][H][d] ~ N(0, 0.01), all float16."""
+    g = _gen(seed, device)
+    E = torch.randn(V, dm, generator=g, device=device, dtype=torch.float32).to(torch.float16)
+    A = (torch.randn(L, 2, H, d, dm, generator=g, device=device, dtype=torch.float32) / dm ** 0.5).to(torch.float16)
+    c = (0.1 * torch.randn(L, 2, H, d, generator=g, device=device, dtype=torch.float32)).to(torch.float16)
+    return E, A, c
+
+
+def make_kv_linear(E, A, c, tokens, sigma, seed, keys=None):
+    """KV [L][2][S][H][n][d] float16 = c + A E[x_i] + sigma * noise(key[s][i]) (computed in float32)."""
+    L, _, H, d, dm = A.shape
+    S, n = tokens.shape
+    dev = A.device
+    if keys is None:
+        keys = torch.arange(S * n, device=dev, dtype=torch.int64).view(S, n)
+    out = torch.empty(L, 2, S, H, n, d, dtype=torch.float16, device=dev)
+    emb = E[tokens.to(torch.int64)].to(torch.float32)                         # [S][n][dm]
+    for l in range(L):
+        for a in range(2):
+            for h in range(H):
+                rows = emb @ A[l, a, h].to(torch.float32).t() + c[l, a, h].to(torch.float32)   # [S][n][d]
+                if sigma:
+                    rows = rows + sigma * hashed_normal(keys, (l * 2 + a) * H + h, d, seed)
+                out[l, a, :, h] = rows.to(torch.float16)
+    return out
