@@ -130,8 +130,10 @@ def main():
     ap.add_argument("--set", action="append", default=[], help="override a workload field, e.g. --set L=4")
     ap.add_argument("--adaptive", type=int, default=0,
                     help="b0 > 0: surprisal-adaptive step (Def. 7) with hbar = log2(perplexity), cap b0 + 4")
-    ap.add_argument("--variant", default="topk", choices=["topk", "dense"],
-                    help="prediction: top-K gather (default) or full-vocabulary bf16 tensor-core contraction")
+    ap.add_argument("--variant", default="topk", choices=["topk", "dense", "linear"],
+                    help="prediction: top-K gather (default), full-vocabulary bf16 tensor-core contraction, or the "
+                         "linear-embedding model of Sec. 7.1 (two chained contractions; see --d-model)")
+    ap.add_argument("--d-model", type=int, default=4096, help="embedding width of --variant linear")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -163,6 +165,9 @@ def main():
         over[k] = float(v) if "." in v else int(v)
     if args.chunk_pos:
         over["chunk_pos"] = args.chunk_pos
+    linear = args.variant == "linear"
+    if linear:
+        over["dm"] = args.d_model
     w = workloads.build(args.workload, dev, seed=20260415 + 1000 * rank, **over)
     cfg = w["cfg"]
     S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
@@ -171,9 +176,12 @@ def main():
     import math
     adaptive = (args.adaptive, 4, math.log2(cfg["pp"])) if args.adaptive > 0 else None
     tok = w["tokens"] if adaptive else None
-    ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                      variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive)
-    ctx.reserve(S * n)
+    if linear:
+        ctx = plc.Context.linear(w["E"], w["A"], w["c"], cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16)
+    else:
+        ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                          variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive)
+        ctx.reserve(S * n)
     ctx.set_profiling(True)
     mc = ctx.max_chunks(n)
     kv_bytes = w["kv"].numel() * 2
@@ -213,7 +221,7 @@ def main():
         ctx.decode(st, w["logits"], out, tokens=tok)
         ev[3 * i + 2].record()
         enc_k.append(ctx.last_kernel_ms(0)); dec_k.append(ctx.last_kernel_ms(1))
-        if dense:
+        if dense or linear:
             gemm_k.append(ctx.last_kernel_ms(2))
     t_end.record()
     barrier()
@@ -240,7 +248,7 @@ def main():
     ek, dk = statistics.mean(enc_k), statistics.mean(dec_k)
     gathered = vecs * K * d * 2
     bytes_ns = vecs * d * 2 + gathered + payload_per_step    # KV + T rows read + bitstream (either direction)
-    bytes_c = vecs * d * 2 + w["T"].numel() * 2 + payload_per_step
+    bytes_c = vecs * d * 2 + (0 if linear else w["T"].numel() * 2) + payload_per_step
     dom_enc = ek >= dk
     dom_ms = ek if dom_enc else dk
     sm_mhz = clocks.get("sm_mhz") or 1965.0
@@ -248,7 +256,7 @@ def main():
     fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
     fma_ach = vecs * K * d / (dom_ms / 1e3)
     dom_name = "encode_kernel" if dom_enc else "decode_kernel"
-    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive
+    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive and not linear
     traffic = NCU_DRAM_BYTES_PER_VECTOR[dom_name] * vecs if default_cfg else None
     roofline = {"kernel": dom_name, "bound": "hbm",
                 "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
@@ -273,8 +281,21 @@ def main():
                     "peak_kind": "measured sustained bf16" if pk else "fallback", "ms_per_launch": gm,
                     "flop_per_launch": flop, "launches_per_step": 2 * L,
                     "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
+    if linear:
+        # per layer: rows x (2H*d) x d_model; once per call: rows x d_model x V (Ebar) and rows x (L*2H) x V (variance)
+        gm = statistics.mean(gemm_k)
+        dm = args.d_model
+        flop = 2.0 * S * n * dm * (2 * H * d)
+        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+        tpeak = float(pk.get("bf16_tflops_sustained", 1400.0))
+        roofline = {"kernel": "dense_gemm_kernel", "bound": "tensor", "achieved": flop / (gm / 1e3) / 1e12, "peak": tpeak,
+                    "unit": "TFLOP/s", "frac": flop / (gm / 1e3) / 1e12 / tpeak, "traffic": None,
+                    "peak_kind": "measured sustained bf16" if pk else "fallback", "ms_per_launch": gm,
+                    "flop_per_launch": flop, "launches_per_step": 2 * L,
+                    "flop_per_step_all_contractions": 2 * (L * flop + 2.0 * S * n * V * dm + 2.0 * S * n * V * 256 * ((W + 255) // 256)),
+                    "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not linear:
         del out, st
         torch.cuda.empty_cache()
 
@@ -284,7 +305,7 @@ def main():
         e2e = run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok, args.e2e_groups)
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not linear:
         layers, pos = min(L, 2), min(n, 256)
         r = oracle_sample_rate(w, pos, layers)
         cpu = {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle",

@@ -45,13 +45,14 @@ enum {
     PLC_E_CUDA = 7       /* a CUDA runtime call failed (allocation, launch) */
 };
 
-enum { PLC_PRED_TOPK = 0, PLC_PRED_DENSE = 1 };
+enum { PLC_PRED_TOPK = 0, PLC_PRED_DENSE = 1, PLC_PRED_LINEAR = 2 };
 enum { PLC_OUT_F32 = 0, PLC_OUT_F16 = 1 };
 
 /* Codec parameters.  delta: quantiser step (>= 2^-12).  sigma_floor: added in quadrature to the
  * mixture's standard deviation before the scale class is taken (0 = none).  chunk_pos: positions
  * per independently coded chunk.  variant: PLC_PRED_TOPK (Sec. 7.1 of the paper, top-k
- * approximation) or PLC_PRED_DENSE (Def. 5, sum over the whole vocabulary as a bf16 contraction). */
+ * approximation), PLC_PRED_DENSE (Def. 5, sum over the whole vocabulary as a bf16 contraction) or
+ * PLC_PRED_LINEAR (Sec. 7.1, linear-embedding approximation; contexts made by plc_create_linear). */
 typedef struct {
     int32_t n_layers, n_kv_heads, head_dim, vocab, top_k;
     float delta, sigma_floor;
@@ -126,6 +127,29 @@ typedef struct plc_ctx plc_ctx;
  * Synchronises the device once (it pre-computes the squared norm of every row of T).
  * Errors: PLC_E_INVALID / PLC_E_SHAPE / PLC_E_ALIGN on bad arguments, PLC_E_CUDA. */
 plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev);
+
+/* Linear-embedding predictor (Sec. 7.1 of the paper: the KV function taken as affine in the token
+ * embedding, so that the expectation over the next token moves inside it):
+ *     KV^ = c + A * Ebar,   Ebar = sum_v P(v) E(v)   over the whole vocabulary,
+ *     sigma_mix^2 = sum_v P(v) ||c + A E(v)||^2 / d - ||KV^||^2 / d          (Thm. 2 with F := c + A E).
+ * E_dev [V][d_model], A_dev [L][2][H][d][d_model], c_dev [L][2][H][d], all f16, 16-byte aligned, not
+ * copied (they must outlive the context).  d_model: a multiple of 64, at most 16384.
+ * Arithmetic: P, E, A and Ebar are rounded to bfloat16 and contracted on the tensor cores with
+ * binary32 accumulation; c is added in binary32. */
+typedef struct {
+    const void* E_dev;
+    const void* A_dev;
+    const void* c_dev;
+    int32_t d_model;
+} plc_linear_model;
+
+/* Creates a context whose predictor is the linear-embedding model; cfg->variant must be
+ * PLC_PRED_LINEAR (top_k is ignored by encode / decode, adaptive_b0 must be 0).  Builds, once, the
+ * bf16 transpose of E and the table of candidate norms ||c + A E(v)||^2 / d of every layer (L
+ * contractions of V x 2Hd x d_model), allocating and freeing its temporaries; synchronises the device.
+ * plc_encode / plc_decode then work as for the other variants; plc_append_step returns PLC_E_STATE.
+ * Errors: PLC_E_INVALID / PLC_E_SHAPE / PLC_E_ALIGN on bad arguments, PLC_E_CUDA. */
+plc_status plc_create_linear(plc_ctx** out, const plc_config* cfg, const plc_linear_model* model);
 plc_status plc_destroy(plc_ctx* ctx);
 
 /* Grows the context's scratch so that calls over up to max_positions = S*n positions allocate

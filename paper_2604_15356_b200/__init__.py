@@ -15,7 +15,7 @@ _SO = os.path.join(_HERE, "libplc.so")
 _SOURCES = ["plc_api.cu", "plc_topk.cu", "plc_prefix.cu", "plc_codec.cu", "plc_dense.cu", "plc_static.cu", "plc_trie.cu"]
 
 OK, E_INVALID, E_SHAPE, E_ALIGN, E_CAPACITY, E_CORRUPT, E_STATE, E_CUDA = range(8)
-PRED_TOPK, PRED_DENSE = 0, 1
+PRED_TOPK, PRED_DENSE, PRED_LINEAR = 0, 1, 2
 OUT_F32, OUT_F16 = 0, 1
 
 EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_prefix_dedup", "plc_encode",
@@ -23,7 +23,7 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
-           "plc_trie_stats"]
+           "plc_trie_stats", "plc_create_linear"]
 
 
 def sources():
@@ -68,6 +68,10 @@ class DebugBuffers(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("payload_bytes", C.c_uint64), ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64),
                 ("coded_vectors", C.c_uint64)]
+
+
+class LinearModel(C.Structure):
+    _fields_ = [("E_dev", C.c_void_p), ("A_dev", C.c_void_p), ("c_dev", C.c_void_p), ("d_model", C.c_int32)]
 
 
 class SessionBatch(C.Structure):
@@ -154,8 +158,26 @@ class Context:
         self._h = C.c_void_p()
         _check(lib().plc_create(C.byref(self._h), C.byref(self.cfg), _ptr(T)), "plc_create")
 
+    @classmethod
+    def linear(cls, E, A, c, delta, chunk_pos=256, sigma_floor=0.0, out_dtype=OUT_F32):
+        """Context of the linear-embedding predictor (Sec. 7.1): E [V][dm], A [L][2][H][d][dm],
+        c [L][2][H][d], float16 on the device."""
+        V, dm = E.shape
+        L, two, H, d, dm2 = A.shape
+        assert two == 2 and dm2 == dm and tuple(c.shape) == (L, 2, H, d)
+        assert all(t.is_cuda and t.is_contiguous() for t in (E, A, c))
+        self = cls.__new__(cls)
+        self.T = None
+        self._model = (E, A, c)
+        self.cfg = Config(L, H, d, V, 1, delta, sigma_floor, chunk_pos, PRED_LINEAR, out_dtype, 0, 0, 0.0)
+        self.W = 2 * L * H
+        self._h = C.c_void_p()
+        m = LinearModel(E.data_ptr(), A.data_ptr(), c.data_ptr(), dm)
+        _check(lib().plc_create_linear(C.byref(self._h), C.byref(self.cfg), C.byref(m)), "plc_create_linear")
+        return self
+
     def close(self):
-        if self._h:
+        if getattr(self, "_h", None):
             lib().plc_destroy(self._h)
             self._h = C.c_void_p()
 

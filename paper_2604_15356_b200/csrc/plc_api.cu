@@ -23,8 +23,14 @@ struct plc_ctx {
     unsigned int* ticket;
     unsigned int* status;
     Counters* counters;
-    uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1
+    uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1; linear variant: P, Ebar, s1, A_layer, mu
     size_t dense_bytes;
+    const __half* lin_E;            // linear variant (Sec. 7.1): caller's E [V][dm], A [L][2H*d][dm], c [L][2H*d]
+    const __half* lin_A;
+    const __half* lin_c;
+    int lin_dm;
+    uint8_t* lin_model;             // E transposed (bf16) and the candidate-norm table of every (layer, table)
+    size_t lin_off[2];
     int profiling;                  // record events around the codec kernels
     cudaEvent_t ev[6];              // encode start/stop, decode start/stop, dense contraction start/stop
     int ev_valid[3];
@@ -90,6 +96,24 @@ DenseShape dense_shape(const plc_ctx* c, long long rows) {
     return sh;
 }
 
+LinearShape linear_shape(const plc_config& cfg, int dm, long long rows) {
+    LinearShape sh;
+    sh.rows = rows; sh.V = cfg.vocab; sh.d = cfg.head_dim; sh.dm = dm; sh.tables = 2 * cfg.n_kv_heads; sh.L = cfg.n_layers;
+    sh.ldv = (sh.V + 63) / 64 * 64;
+    sh.ncols = sh.tables * sh.d; sh.ncols_pad = (sh.ncols + 255) / 256 * 256;
+    sh.nt_all = sh.L * sh.tables; sh.nt_all_pad = (sh.nt_all + 255) / 256 * 256;
+    return sh;
+}
+
+plc_status ensure_scratch(plc_ctx* c, size_t need) {
+    if (need <= c->dense_bytes) return PLC_OK;
+    if (c->dense_scratch) cudaFree(c->dense_scratch);
+    c->dense_scratch = nullptr; c->dense_bytes = 0;
+    if (cudaMalloc(&c->dense_scratch, need) != cudaSuccess) return PLC_E_CUDA;
+    c->dense_bytes = need;
+    return PLC_OK;
+}
+
 plc_status ensure_dense(plc_ctx* c, const DenseShape& sh, size_t* off) {
     const size_t need = dense_scratch_bytes(sh, off);
     if (need <= c->dense_bytes) return PLC_OK;
@@ -118,19 +142,35 @@ KvView to_dev(const plc_kv_view* v) {
 
 extern "C" {
 
+static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void* T_dev, const plc_linear_model* lin);
+
 plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
     if (!out || !cfg || !T_dev) return PLC_E_INVALID;
+    if (cfg->variant != PLC_PRED_TOPK && cfg->variant != PLC_PRED_DENSE) return PLC_E_INVALID;
+    return create_common(out, cfg, T_dev, nullptr);
+}
+
+plc_status plc_create_linear(plc_ctx** out, const plc_config* cfg, const plc_linear_model* model) {
+    if (!out || !cfg || !model || !model->E_dev || !model->A_dev || !model->c_dev) return PLC_E_INVALID;
+    if (cfg->variant != PLC_PRED_LINEAR) return PLC_E_INVALID;
+    if (model->d_model < 64 || model->d_model % 64 || model->d_model > 16384) return PLC_E_SHAPE;
+    if ((long long)cfg->n_layers * 2 * cfg->n_kv_heads > 65536) return PLC_E_SHAPE;
+    if (!aligned16(model->E_dev) || !aligned16(model->A_dev) || !aligned16(model->c_dev)) return PLC_E_ALIGN;
+    return create_common(out, cfg, nullptr, model);
+}
+
+static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void* T_dev, const plc_linear_model* lin) {
     *out = nullptr;
     if (cfg->n_layers < 1 || cfg->n_kv_heads < 1 || cfg->vocab < 1) return PLC_E_INVALID;
     if (!valid_d(cfg->head_dim) || cfg->top_k < 1 || cfg->top_k > cfg->vocab || cfg->top_k > 1024) return PLC_E_SHAPE;
     if (cfg->chunk_pos < 1 || cfg->chunk_pos > 4096) return PLC_E_SHAPE;
     if (!(cfg->delta >= 1.0f / 4096.0f) || !(cfg->delta < 65536.0f) || !(cfg->sigma_floor >= 0.0f)) return PLC_E_INVALID;
-    if (cfg->variant != PLC_PRED_TOPK && cfg->variant != PLC_PRED_DENSE) return PLC_E_INVALID;
     if (cfg->out_dtype != PLC_OUT_F32 && cfg->out_dtype != PLC_OUT_F16) return PLC_E_INVALID;
     if (cfg->adaptive_b0 < 0 || cfg->adaptive_b0 > 16 || cfg->adaptive_extra < 0 || cfg->adaptive_extra > 12) return PLC_E_INVALID;
     if (cfg->adaptive_b0 > 0 && !(cfg->adaptive_hbar > 0.0f)) return PLC_E_INVALID;
     if (cfg->adaptive_b0 > 0 && cfg->variant != PLC_PRED_TOPK) return PLC_E_STATE;
-    if (!aligned16(T_dev)) return PLC_E_ALIGN;
+    if (cfg->variant != PLC_PRED_TOPK && 2 * cfg->n_kv_heads > 256) return PLC_E_SHAPE;
+    if (T_dev && !aligned16(T_dev)) return PLC_E_ALIGN;
     plc_ctx* c = new (std::nothrow) plc_ctx();
     if (!c) return PLC_E_CUDA;
     c->cfg = *cfg;
@@ -138,15 +178,23 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
     const long long rows = (long long)cfg->n_layers * 2 * cfg->n_kv_heads * cfg->vocab;
     c->staging_words_per_warp = 4ull * cfg->chunk_pos * cfg->head_dim + 64;
     const int warps = codec_grid_warps(0);
-    bool ok = cudaMalloc(&c->rownorm2, sizeof(float) * (size_t)rows) == cudaSuccess &&
+    bool ok = (!T_dev || cudaMalloc(&c->rownorm2, sizeof(float) * (size_t)rows) == cudaSuccess) &&
               cudaMalloc(&c->staging, sizeof(uint16_t) * c->staging_words_per_warp * warps) == cudaSuccess &&
               cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(unsigned int)) == cudaSuccess &&
               cudaMalloc(&c->counters, sizeof(Counters)) == cudaSuccess;
     if (ok) ok = cudaMemset(c->status, 0, sizeof(unsigned int)) == cudaSuccess &&
                  cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
-    if (ok) ok = launch_rownorm(c->T, c->rownorm2, rows, cfg->head_dim, 0) == cudaSuccess &&
-                 cudaDeviceSynchronize() == cudaSuccess;
+    if (ok && T_dev) ok = launch_rownorm(c->T, c->rownorm2, rows, cfg->head_dim, 0) == cudaSuccess &&
+                          cudaDeviceSynchronize() == cudaSuccess;
+    if (ok && lin) {
+        c->lin_E = static_cast<const __half*>(lin->E_dev); c->lin_A = static_cast<const __half*>(lin->A_dev);
+        c->lin_c = static_cast<const __half*>(lin->c_dev); c->lin_dm = lin->d_model;
+        const LinearShape sh = linear_shape(*cfg, lin->d_model, 0);
+        const size_t bytes = linear_model_bytes(sh, c->lin_off);
+        ok = cudaMalloc(&c->lin_model, bytes) == cudaSuccess &&
+             linear_prepare(c->lin_E, c->lin_A, c->lin_c, sh, c->lin_model, c->lin_off, c->status, 0) == cudaSuccess;
+    }
     for (int i = 0; i < 6 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
     if (!ok) { plc_destroy(c); return PLC_E_CUDA; }
     *out = c;
@@ -156,7 +204,7 @@ plc_status plc_create(plc_ctx** out, const plc_config* cfg, const void* T_dev) {
 plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
     cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->step_exp); cudaFree(c->staging);
-    cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch);
+    cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch); cudaFree(c->lin_model);
     for (int i = 0; i < 6; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
     return PLC_OK;
@@ -229,6 +277,32 @@ static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, boo
     return PLC_OK;
 }
 
+// Linear-embedding variant (Sec. 7.1): Ebar and the variance term once, then per layer mu = Ebar A^T and the coding.
+static plc_status run_linear(plc_ctx* c, CodecArgs a, const void* logits_dev, bool encode, cudaStream_t st) {
+    const LinearShape sh = linear_shape(c->cfg, c->lin_dm, (long long)a.S * a.n);
+    size_t off[6];
+    plc_status rc = ensure_scratch(c, linear_scratch_bytes(sh, off));
+    if (rc) return rc;
+    if (linear_begin(static_cast<const __half*>(logits_dev), sh, c->lin_model, c->lin_off, c->dense_scratch, off, c->status, st) !=
+        cudaSuccess) return PLC_E_CUDA;
+    a.mu_dense = reinterpret_cast<const float*>(c->dense_scratch + off[5]);
+    a.mu_ld = sh.ncols; a.s1_ld = sh.nt_all;
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        const bool prof = c->profiling != 0;
+        if (linear_layer(c->lin_A + (size_t)l * sh.ncols * sh.dm, sh, c->dense_scratch, off, c->status, st,
+                         prof ? c->ev[4] : nullptr, prof ? c->ev[5] : nullptr) != cudaSuccess) return PLC_E_CUDA;
+        if (prof) c->ev_valid[2] = 1;
+        a.dense_layer = l;
+        a.s1_dense = reinterpret_cast<const float*>(c->dense_scratch + off[3]) + (size_t)l * sh.tables;
+        a.mu_bias = c->lin_c + (size_t)l * sh.ncols;
+        const int w = encode ? 0 : 1;
+        if (prof) cudaEventRecord(c->ev[2 * w], st);
+        if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;
+        if (prof) { cudaEventRecord(c->ev[2 * w + 1], st); c->ev_valid[w] = 1; }
+    }
+    return PLC_OK;
+}
+
 // tokens_dev non-null <=> adaptive call
 static plc_status encode_impl(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, const int32_t* tokens_dev,
                               int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
@@ -249,6 +323,7 @@ static plc_status encode_impl(plc_ctx* c, const plc_kv_view* kv, const void* log
     a.st = to_dev(out);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, true, st);
+    if (c->cfg.variant == PLC_PRED_LINEAR) return run_linear(c, a, logits_dev, true, st);
     rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;
@@ -291,6 +366,7 @@ static plc_status decode_impl(plc_ctx* c, const plc_streams* in, const void* log
     a.st = to_dev(in);
     if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, false, st);
+    if (c->cfg.variant == PLC_PRED_LINEAR) return run_linear(c, a, logits_dev, false, st);
     rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;

@@ -428,6 +428,10 @@ __device__ __forceinline__ void predict_dense(const CodecArgs& a, long long row,
     const float* mp = a.mu_dense + row * a.mu_ld + (long long)t_local * D + c0;
 #pragma unroll
     for (int g = 0; g < G; ++g) mu[g] = __ldg(mp + g);
+    if (a.mu_bias) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) mu[g] = __fadd_rn(mu[g], __half2float(a.mu_bias[t_local * D + c0 + g]));
+    }
     const float s1 = __ldg(a.s1_dense + row * a.s1_ld + t_local);
     const float s2 = warp_norm2<G>(mu);
     sigma2 = fmaxf(0.f, s1 - s2 * inv_d);

@@ -193,6 +193,7 @@ struct CodecArgs {
     unsigned int* status; Counters* counters;
     // dense variant: prediction read from buffers; one launch covers the 2*H tables of dense_layer
     const float* mu_dense; const float* s1_dense; long long mu_ld, s1_ld; int dense_layer;
+    const __half* mu_bias;                         // optional [2*H][d] f16 added to mu (linear predictor's c), or null
     // append path: symbols come from / go to the open chunk
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
 };
@@ -207,6 +208,22 @@ struct DenseShape {
 };
 size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]: P, Tb, n2b, mu, s1*/);
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st);
+// Linear-embedding predictor (Sec. 7.1).
+struct LinearShape {
+    long long rows;
+    int V, d, dm, tables, L;   // tables = 2*H per layer, dm = d_model (multiple of 64)
+    int ldv;                   // V rounded up to 64
+    int ncols, ncols_pad;      // tables*d, rounded up to 256
+    int nt_all, nt_all_pad;    // L*tables, rounded up to 256
+};
+size_t linear_model_bytes(const LinearShape& sh, size_t* off /*[2]*/);
+size_t linear_scratch_bytes(const LinearShape& sh, size_t* off /*[6]*/);
+cudaError_t linear_prepare(const __half* E, const __half* A, const __half* c, const LinearShape& sh, uint8_t* model,
+                           const size_t* moff, unsigned int* status, cudaStream_t st);
+cudaError_t linear_begin(const __half* logits, const LinearShape& sh, const uint8_t* model, const size_t* moff,
+                         uint8_t* scratch, const size_t* off, unsigned int* status, cudaStream_t st);
+cudaError_t linear_layer(const __half* A_layer, const LinearShape& sh, uint8_t* scratch, const size_t* off,
+                         unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1);
 cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
                         unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1);   // events bracket the contraction
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st);

@@ -328,6 +328,51 @@ bool make_map(CUtensorMap* map, void* base, uint64_t inner, uint64_t outer, uint
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// out[rows x ncols] (fp32, pitch ldo) = A[rows x K] * B[nrows_b x K]^T, both bf16 with row pitch ldk (a
+// multiple of 64; K = ldk, zero padded); nrows_b is a multiple of the N tile bn.
+cudaError_t launch_gemm(const __nv_bfloat16* A, long long rows, const __nv_bfloat16* B, int nrows_b, int ldk, int bn,
+                        float* out, long long ldo, int ncols, unsigned int* status, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, const_cast<__nv_bfloat16*>(A), (uint64_t)ldk, (uint64_t)rows, (uint64_t)ldk, kBM)) return cudaErrorUnknown;
+    if (!make_map(&mb, const_cast<__nv_bfloat16*>(B), (uint64_t)ldk, (uint64_t)nrows_b, (uint64_t)ldk, (uint32_t)bn)) return cudaErrorUnknown;
+    cudaError_t e = cudaFuncSetAttribute(dense_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+    if (e != cudaSuccess) return e;
+    dim3 g((unsigned)((rows + kBM - 1) / kBM), (unsigned)(nrows_b / bn));
+    dense_gemm_kernel<<<g, kGemmThreads, kGemmSmem, st>>>(ma, mb, out, ldo, (int)rows, ncols, ldk / kBK, bn, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// dst[r][c] = bf16(src[r][c]) for c < cols, 0 for cols <= c < ld (row-major, f16 source pitch = cols).
+__global__ void __launch_bounds__(256) cvt_f16_bf16_kernel(const __half* __restrict__ src, long long rows, int cols, int ld,
+                                                           __nv_bfloat16* __restrict__ dst) {
+    const long long total = rows * ld;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+        const long long r = i / ld; const int c = (int)(i % ld);
+        dst[i] = __float2bfloat16_rn(c < cols ? __half2float(src[r * cols + c]) : 0.f);
+    }
+}
+__global__ void __launch_bounds__(256) cvt_f32_bf16_kernel(const float* __restrict__ src, long long n, __nv_bfloat16* __restrict__ dst) {
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256)
+        dst[i] = __float2bfloat16_rn(src[i]);
+}
+// Nb[t][v] = bf16(sum_j (tlin[v][t*d + j] + c[t][j])^2 / d): one warp per (v, t).
+__global__ void __launch_bounds__(256) tlin_norm_kernel(const float* __restrict__ tlin, long long ld_t, const __half* __restrict__ c,
+                                                        int V, int tables, int d, int ldv, __nv_bfloat16* __restrict__ Nb) {
+    const int lane = threadIdx.x & 31;
+    const long long warp = (long long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long long)gridDim.x * 8;
+    for (long long it = warp; it < (long long)V * tables; it += nw) {
+        const int v = (int)(it / tables), t = (int)(it % tables);
+        float s = 0.f;
+        for (int j = lane; j < d; j += 32) {
+            const float x = tlin[(long long)v * ld_t + t * d + j] + __half2float(c[t * d + j]);
+            s = __fmaf_rn(x, x, s);
+        }
+        s = warp_sum(s);
+        if (lane == 0) Nb[(size_t)t * ldv + v] = __float2bfloat16_rn(s / (float)d);
+    }
+}
+
 }  // namespace
 
 size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
@@ -390,6 +435,105 @@ cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* sc
                                                            sh.ldv / kBK, nb_rows, status);
     count_launch(4);
     return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Linear-embedding predictor (Sec. 7.1): KV^ ~ c + A Ebar, Ebar = sum_v p_v E(v).  Two chained
+// contractions on the same tensor-core kernel: Ebar = P * E (once per call, shared by all layers),
+// then per layer mu = Ebar * A_layer^T (K = d_model); the variance term of all layers is one more
+// contraction of P with the table of candidate norms ||c + A E(v)||^2 / d built at creation.
+
+size_t linear_model_bytes(const LinearShape& sh, size_t* off /*[2]: Ebt, NbAll*/) {
+    auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    size_t o = 0;
+    off[0] = o; o += up((size_t)sh.dm * sh.ldv * 2);
+    off[1] = o; o += up((size_t)sh.nt_all_pad * sh.ldv * 2);
+    return o;
+}
+
+size_t linear_scratch_bytes(const LinearShape& sh, size_t* off /*[6]: P, Ef, Eb16, s1, Ab, mu*/) {
+    auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    size_t o = 0;
+    off[0] = o; o += up((size_t)sh.rows * sh.ldv * 2);
+    off[1] = o; o += up((size_t)sh.rows * sh.dm * 4);
+    off[2] = o; o += up((size_t)sh.rows * sh.dm * 2);
+    off[3] = o; o += up((size_t)sh.rows * sh.nt_all * 4);
+    off[4] = o; o += up((size_t)sh.ncols_pad * sh.dm * 2);
+    off[5] = o; o += up((size_t)sh.rows * sh.ncols * 4);
+    return o;
+}
+
+static int tile_for(int n) { return n % 256 == 0 ? 256 : (n % 128 == 0 ? 128 : 64); }
+static unsigned blocks_for(long long n) { long long b = (n + 255) / 256; return (unsigned)(b < 148 * 16 ? (b > 0 ? b : 1) : 148 * 16); }
+
+// Creation: E transposed to bf16 and the norm table of every (layer, table).  Allocates (and
+// frees) its temporaries; synchronises the stream.
+cudaError_t linear_prepare(const __half* E, const __half* A, const __half* c, const LinearShape& sh, uint8_t* model,
+                           const size_t* moff, unsigned int* status, cudaStream_t st) {
+    __nv_bfloat16* Ebt = reinterpret_cast<__nv_bfloat16*>(model + moff[0]);
+    __nv_bfloat16* NbAll = reinterpret_cast<__nv_bfloat16*>(model + moff[1]);
+    __nv_bfloat16 *Eb = nullptr, *Ab = nullptr;
+    float* tlin = nullptr;
+    cudaError_t e = cudaMalloc(&Eb, (size_t)sh.V * sh.dm * 2);
+    if (e == cudaSuccess) e = cudaMalloc(&Ab, (size_t)sh.ncols_pad * sh.dm * 2);
+    if (e == cudaSuccess) e = cudaMalloc(&tlin, (size_t)sh.V * sh.ncols * 4);
+    if (e == cudaSuccess) e = cudaMemsetAsync(NbAll, 0, (size_t)sh.nt_all_pad * sh.ldv * 2, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(Ab, 0, (size_t)sh.ncols_pad * sh.dm * 2, st);
+    if (e == cudaSuccess) {
+        dim3 tg((sh.ldv + 31) / 32, sh.dm / 32, 1);
+        transpose_bf16_kernel<<<tg, 256, 0, st>>>(E, 1, sh.V, sh.dm, sh.ldv, Ebt);
+        cvt_f16_bf16_kernel<<<blocks_for((long long)sh.V * sh.dm), 256, 0, st>>>(E, sh.V, sh.dm, sh.dm, Eb);
+        count_launch(2);
+        for (int l = 0; l < sh.L && e == cudaSuccess; ++l) {
+            const __half* Al = A + (size_t)l * sh.ncols * sh.dm;
+            cvt_f16_bf16_kernel<<<blocks_for((long long)sh.ncols * sh.dm), 256, 0, st>>>(Al, sh.ncols, sh.dm, sh.dm, Ab);
+            e = launch_gemm(Eb, sh.V, Ab, sh.ncols_pad, sh.dm, 256, tlin, sh.ncols, sh.ncols, status, st);
+            if (e != cudaSuccess) break;
+            const long long pairs = (long long)sh.V * sh.tables;
+            tlin_norm_kernel<<<(unsigned)((pairs + 7) / 8 < 148 * 16 ? (pairs + 7) / 8 : 148 * 16), 256, 0, st>>>(
+                tlin, sh.ncols, c + (size_t)l * sh.ncols, sh.V, sh.tables, sh.d, sh.ldv, NbAll + (size_t)l * sh.tables * sh.ldv);
+            count_launch(2);
+            e = cudaGetLastError();
+        }
+    }
+    cudaError_t e2 = cudaStreamSynchronize(st);
+    cudaFree(Eb); cudaFree(Ab); cudaFree(tlin);
+    return e != cudaSuccess ? e : e2;
+}
+
+// Per call: P, Ebar (bf16) and the variance term of every layer.
+cudaError_t linear_begin(const __half* logits, const LinearShape& sh, const uint8_t* model, const size_t* moff,
+                         uint8_t* scratch, const size_t* off, unsigned int* status, cudaStream_t st) {
+    DenseShape ds{}; ds.rows = sh.rows; ds.V = sh.V; ds.ldv = sh.ldv;
+    cudaError_t e = dense_softmax(logits, ds, scratch, off, st);
+    if (e != cudaSuccess) return e;
+    const __nv_bfloat16* P = reinterpret_cast<const __nv_bfloat16*>(scratch + off[0]);
+    float* Ef = reinterpret_cast<float*>(scratch + off[1]);
+    __nv_bfloat16* Eb16 = reinterpret_cast<__nv_bfloat16*>(scratch + off[2]);
+    float* s1 = reinterpret_cast<float*>(scratch + off[3]);
+    e = launch_gemm(P, sh.rows, reinterpret_cast<const __nv_bfloat16*>(model + moff[0]), sh.dm, sh.ldv, tile_for(sh.dm),
+                    Ef, sh.dm, sh.dm, status, st);
+    if (e != cudaSuccess) return e;
+    cvt_f32_bf16_kernel<<<blocks_for(sh.rows * sh.dm), 256, 0, st>>>(Ef, sh.rows * sh.dm, Eb16);
+    count_launch();
+    return launch_gemm(P, sh.rows, reinterpret_cast<const __nv_bfloat16*>(model + moff[1]), sh.nt_all_pad, sh.ldv, 256,
+                       s1, sh.nt_all, sh.nt_all, status, st);
+}
+
+// Per layer: mu [rows][2H*d] = Ebar * A_layer^T (the bias c is added where mu is read).
+cudaError_t linear_layer(const __half* A_layer, const LinearShape& sh, uint8_t* scratch, const size_t* off,
+                         unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
+    __nv_bfloat16* Ab = reinterpret_cast<__nv_bfloat16*>(scratch + off[4]);
+    cudaError_t e = cudaSuccess;
+    if (sh.ncols_pad > sh.ncols) e = cudaMemsetAsync(Ab + (size_t)sh.ncols * sh.dm, 0, (size_t)(sh.ncols_pad - sh.ncols) * sh.dm * 2, st);
+    if (e != cudaSuccess) return e;
+    cvt_f16_bf16_kernel<<<blocks_for((long long)sh.ncols * sh.dm), 256, 0, st>>>(A_layer, sh.ncols, sh.dm, sh.dm, Ab);
+    count_launch();
+    if (ev0) cudaEventRecord(ev0, st);
+    e = launch_gemm(reinterpret_cast<const __nv_bfloat16*>(scratch + off[2]), sh.rows, Ab, sh.ncols_pad, sh.dm, 256,
+                    reinterpret_cast<float*>(scratch + off[5]), sh.ncols, sh.ncols, status, st);
+    if (ev1) cudaEventRecord(ev1, st);
+    return e;
 }
 
 }  // namespace plc

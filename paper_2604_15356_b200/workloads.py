@@ -24,7 +24,8 @@ CONFIGS = {
 
 def build(name, device, seed=20260415, **override):
     """Returns dict(cfg, tokens [S][n] i32, logits [S][n][V] f16, T [L][2][H][V][d] f16,
-    kv [L][2][S][H][n][d] f16), all on ``device``."""
+    kv [L][2][S][H][n][d] f16), all on ``device``.  With the override ``dm`` the candidate table is
+    replaced by a linear model (E [V][dm], A [L][2][H][d][dm], c [L][2][H][d]) and T is None."""
     cfg = dict(CONFIGS[name])
     cfg.update(override)
     S, n, L, H, d, V = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"]
@@ -33,6 +34,12 @@ def build(name, device, seed=20260415, **override):
     tokens = synth.sample_tokens(table, S, n, seed + 1)
     logits = synth.position_logits(table, tokens)
     del table
+    if cfg.get("dm"):          # KV function linear in the token embedding (Sec. 7.1) instead of a candidate table
+        E, A, c = synth.make_linear_model(L, H, V, d, int(cfg["dm"]), seed + 2, device=device)
+        kv = synth.make_kv_linear(E, A, c, tokens, cfg["sigma"], seed + 3)
+        if torch.device(device).type == "cuda":
+            torch.cuda.empty_cache()
+        return dict(cfg=cfg, tokens=tokens, logits=logits, T=None, kv=kv, E=E, A=A, c=c)
     T = synth.make_tables(L, H, V, d, seed + 2, device=device)
     kv = synth.make_kv(T, tokens, cfg["sigma"], seed + 3)
     if torch.device(device).type == "cuda":
