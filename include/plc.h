@@ -65,6 +65,16 @@ typedef struct {
      * bits, i.e. the step delta * 2^(adaptive_b0 - b_i).  0 <= adaptive_extra <= 12, adaptive_b0 <= 16. */
     int32_t adaptive_b0, adaptive_extra;
     float adaptive_hbar;
+    /* Zero-rate rule (Thm. 3 / Cor. 6 of the paper: a position whose residual variance per component
+     * does not exceed the target distortion D needs no bits).  zero_rate_D > 0 turns it on: a
+     * (stream, position) whose scale class q = round(4 log2(sigma^2 / step^2)) satisfies
+     * q <= floor(4 log2(zero_rate_D / step^2) - 1/2) -- which implies sigma^2 <= zero_rate_D, sigma^2
+     * being the mixture variance plus sigma_floor^2 -- puts nothing in the stream and decodes to the
+     * prediction itself (symbols 0); the step/2 error bound does not hold there, the expected squared
+     * error per component is at most zero_rate_D if KV follows the predictor's distribution.  With
+     * the adaptive step the comparison uses the position's own step.  0 = off.  Works with every
+     * variant and with plc_append_step. */
+    float zero_rate_D;
 } plc_config;
 
 /* A KV tensor indexed [layer][kv][session][head][position][d]; strides in ELEMENTS, the d
@@ -104,7 +114,8 @@ typedef struct {
     uint64_t payload_bytes;   /* sum of exact chunk sizes written since the counters were last reset */
     uint64_t n_chunks;
     uint64_t n_escapes;       /* components whose magnitude left the 63-symbol alphabet */
-    uint64_t coded_vectors;   /* (stream, position) pairs coded */
+    uint64_t coded_vectors;   /* (stream, position) pairs covered by the chunks written */
+    uint64_t skipped_vectors; /* of those, pairs the zero-rate rule left out of the stream */
 } plc_stats;
 
 /* State of a batch of B sessions that grow by one position per plc_append_step (lock step).

@@ -32,7 +32,8 @@ class Config(C.Structure):
     _fields_ = [("L", C.c_int32), ("H", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("K", C.c_int32),
                 ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32), ("dense", C.c_int32),
                 ("adaptive_b0", C.c_int32), ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float),
-                ("lin_dm", C.c_int32), ("lin_E", C.c_void_p), ("lin_A", C.c_void_p), ("lin_c", C.c_void_p)]
+                ("lin_dm", C.c_int32), ("lin_E", C.c_void_p), ("lin_A", C.c_void_p), ("lin_c", C.c_void_p),
+                ("zero_D", C.c_float)]
 
 
 class KVStrides(C.Structure):
@@ -42,7 +43,8 @@ class KVStrides(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("ideal_bits", C.c_double), ("token_bits", C.c_double), ("payload_bytes", C.c_uint64),
-                ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64), ("coded_positions", C.c_uint64)]
+                ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64), ("coded_positions", C.c_uint64),
+                ("skipped_vectors", C.c_uint64)]
 
 
 _lib = None
@@ -137,6 +139,17 @@ def linear_config(L, H, d, V, K, delta, chunk_pos, E, A, c):
     cfg = Config(L, H, d, V, K, delta, 0.0, chunk_pos, 2, 0, 0, 0.0, Eb.shape[1], Eb.ctypes.data, Ab.ctypes.data, cb.ctypes.data)
     cfg._keep = (Eb, Ab, cb)
     return cfg
+
+
+def zero_class(D, step):
+    """Largest scale class the zero-rate rule (Thm. 3) skips at target distortion D and this step."""
+    lib().plo_zero_class.restype = C.c_int
+    return int(lib().plo_zero_class(C.c_double(D), C.c_double(step)))
+
+
+def q_skip():
+    """Class value that marks a position without symbols in rans_encode_chunk / rans_decode_chunk."""
+    return int(lib().plo_q_skip())
 
 
 def expected_embedding(E, logits_row, lse):

@@ -358,6 +358,10 @@ static int valid_d(int d) { return d == 32 || d == 64 || d == 128 || d == 256; }
 static int zigzag(int32_t hi) { return hi > 0 ? 2 * hi - 1 : -2 * hi; }
 static int32_t unzigzag(int zz) { return (zz & 1) ? (zz + 1) / 2 : -(zz / 2); }
 
+/* Class value that marks a position carrying no symbols at all (zero-rate rule, Thm. 3). */
+#define PLO_Q_SKIP (-100000)
+int plo_q_skip(void) { return PLO_Q_SKIP; }
+
 /* A chunk is P consecutive positions of one stream (one d-vector per position); d = 32 G, d in
  * {32, 64, 128, 256}.  The vector is cut into R = d/8 groups of 8 components (16 bytes of f16);
  * lane l (0..31) owns, in group l mod R, the G components starting at G*(l div R):
@@ -396,6 +400,7 @@ int plo_rans_encode_chunk(const int32_t* sym /*[P][d]*/, const int32_t* q /*[P]*
     int cur_qp = 1000;
     for (int p = P - 1; p >= 0; --p) {
         int s, qp;
+        if (q[p] == PLO_Q_SKIP) continue;              /* zero-rate position: nothing in the stream */
         if (q[p] < Q_MIN || q[p] > Q_MAX) { free(words); return PLO_E_INVALID; }
         plo_class_params(q[p], &s, &qp);
         if (qp != cur_qp) { plo_build_table(qp, f, c); cur_qp = qp; }
@@ -466,6 +471,7 @@ int plo_rans_decode_chunk(const uint8_t* in, uint64_t nbytes, const int32_t* q /
     int cur_qp = 1000;
     for (int p = 0; p < P; ++p) {
         int s, qp;
+        if (q[p] == PLO_Q_SKIP) { for (int j = 0; j < d; ++j) sym[(size_t)p * d + j] = 0; continue; }
         if (q[p] < Q_MIN || q[p] > Q_MAX) return PLO_E_INVALID;
         plo_class_params(q[p], &s, &qp);
         if (qp != cur_qp) { plo_build_table(qp, f, c); cur_qp = qp; }
@@ -541,6 +547,19 @@ int plo_adaptive_bits(float h, int b0, float hbar, int extra) {
     return b;
 }
 
+/* ---------------------------------------------------------------- zero-rate rule */
+
+/* Thm. 3 / Cor. 6 (reverse water-filling): a position whose residual variance per component does
+ * not exceed the target distortion D needs no bits; the decoder then takes KV' = KV^.  The
+ * variance the coder knows is the mixture's (plus the optional floor), and its comparison with D
+ * is taken on the integer scale class q = round(4 log2(sigma^2 / step^2)), so that both sides
+ * decide alike: a position is skipped iff q <= floor(4 log2(D / step^2) - 1/2), which implies
+ * sigma^2 <= D (the rounding of q is at most 1/2).  D <= 0 switches the rule off. */
+int plo_zero_class(double D, double step) {
+    if (!(D > 0.0)) return -1000000;
+    return (int)floor(4.0 * log2(D / (step * step)) - 0.5);
+}
+
 /* ---------------------------------------------------------------- whole path */
 
 /* Strides, in elements, of a KV tensor whose last dimension (d) is contiguous. */
@@ -559,6 +578,7 @@ typedef struct {
     const uint16_t* lin_E;        /* [V][dm] f16 token embeddings */
     const uint16_t* lin_A;        /* [L][2][H][d][dm] f16 */
     const uint16_t* lin_c;        /* [L][2][H][d] f16 */
+    float zero_D;                 /* > 0: zero-rate rule (Thm. 3) at target distortion D per component */
 } plo_config;
 
 typedef struct {
@@ -566,6 +586,7 @@ typedef struct {
     double token_bits;      /* sum of -log2 P(x_i | x_<i) over coded positions */
     uint64_t payload_bytes; /* sum of exact chunk sizes */
     uint64_t n_chunks, n_escapes, coded_positions;
+    uint64_t skipped_vectors; /* (stream, position) pairs left out by the zero-rate rule */
 } plo_stats;
 
 static int64_t chunk_slot(const plo_config* c, int S, int max_chunks, int s, int l, int kv, int h, int ch) {
@@ -635,11 +656,14 @@ int plo_encode(const plo_config* cfg, const uint16_t* T, const uint16_t* kv, con
                     else if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mu, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mu, &s2);
                     cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
+                    const int skip = cq[p] <= plo_zero_class((double)cfg->zero_D, (double)pdelta[i]);
                     const uint16_t* x = kv + l * st->layer + a * st->kv + s * st->session + h * st->head + (int64_t)i * st->pos;
                     plo_quantise(x, mu, d, pdelta[i], csym + (size_t)p * d);
+                    if (skip) memset(csym + (size_t)p * d, 0, sizeof(int32_t) * (size_t)d);
                     size_t o = ((((size_t)s * n + i) * L + l) * 2 + a) * H + h;
                     if (sym_out) memcpy(sym_out + o * d, csym + (size_t)p * d, sizeof(int32_t) * d);
                     if (q_out) q_out[o] = cq[p];
+                    if (skip) { cq[p] = PLO_Q_SKIP; stats->skipped_vectors++; }
                     if (mu_out) for (int j = 0; j < d; ++j) mu_out[o * d + j] = (float)mu[j];
                 }
                 uint64_t nb = 0, nesc = 0; double ideal = 0.0;
@@ -711,6 +735,7 @@ int plo_decode(const plo_config* cfg, const uint16_t* T, const uint16_t* logits,
                     else if (cfg->dense) plo_dense_mixture(table, V, d, logits + ((size_t)s * n + i) * V, lse[i], mus + (size_t)p * d, &s2);
                     else plo_mixture(table, d, idx + (size_t)i * K, w + (size_t)i * K, K, mus + (size_t)p * d, &s2);
                     cq[p] = plo_class(s2, cfg->sigma_floor, pdelta[i]);
+                    if (cq[p] <= plo_zero_class((double)cfg->zero_D, (double)pdelta[i])) cq[p] = PLO_Q_SKIP;
                 }
                 int64_t slot = chunk_slot(cfg, S, max_chunks, s, l, a, h, ch);
                 int r = plo_rans_decode_chunk(payload + chunk_offset[slot], chunk_bytes[slot], cq, P, d, csym);

@@ -48,7 +48,7 @@ class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("vocab", C.c_int32),
                 ("top_k", C.c_int32), ("delta", C.c_float), ("sigma_floor", C.c_float), ("chunk_pos", C.c_int32),
                 ("variant", C.c_int32), ("out_dtype", C.c_int32), ("adaptive_b0", C.c_int32),
-                ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float)]
+                ("adaptive_extra", C.c_int32), ("adaptive_hbar", C.c_float), ("zero_rate_D", C.c_float)]
 
 
 class KVView(C.Structure):
@@ -67,7 +67,7 @@ class DebugBuffers(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("payload_bytes", C.c_uint64), ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64),
-                ("coded_vectors", C.c_uint64)]
+                ("coded_vectors", C.c_uint64), ("skipped_vectors", C.c_uint64)]
 
 
 class LinearModel(C.Structure):
@@ -146,20 +146,20 @@ class Context:
     """One parameter set + candidate table T ([L][2][H][V][d] float16 on the device)."""
 
     def __init__(self, T, top_k, delta, chunk_pos=256, sigma_floor=0.0, variant=PRED_TOPK, out_dtype=OUT_F32,
-                 adaptive=None):
+                 adaptive=None, zero_rate_D=0.0):
         """adaptive = (b0, extra, hbar) turns on the surprisal-adaptive step (Def. 7); encode / decode
-        then need the tokens."""
+        then need the tokens.  zero_rate_D > 0 turns on the zero-rate rule (Thm. 3)."""
         L, two, H, V, d = T.shape
         assert two == 2 and T.is_cuda and T.is_contiguous()
         self.T = T
         b0, extra, hbar = adaptive if adaptive else (0, 0, 0.0)
-        self.cfg = Config(L, H, d, V, top_k, delta, sigma_floor, chunk_pos, variant, out_dtype, b0, extra, hbar)
+        self.cfg = Config(L, H, d, V, top_k, delta, sigma_floor, chunk_pos, variant, out_dtype, b0, extra, hbar, zero_rate_D)
         self.W = 2 * L * H
         self._h = C.c_void_p()
         _check(lib().plc_create(C.byref(self._h), C.byref(self.cfg), _ptr(T)), "plc_create")
 
     @classmethod
-    def linear(cls, E, A, c, delta, chunk_pos=256, sigma_floor=0.0, out_dtype=OUT_F32):
+    def linear(cls, E, A, c, delta, chunk_pos=256, sigma_floor=0.0, out_dtype=OUT_F32, zero_rate_D=0.0):
         """Context of the linear-embedding predictor (Sec. 7.1): E [V][dm], A [L][2][H][d][dm],
         c [L][2][H][d], float16 on the device."""
         V, dm = E.shape
@@ -169,7 +169,7 @@ class Context:
         self = cls.__new__(cls)
         self.T = None
         self._model = (E, A, c)
-        self.cfg = Config(L, H, d, V, 1, delta, sigma_floor, chunk_pos, PRED_LINEAR, out_dtype, 0, 0, 0.0)
+        self.cfg = Config(L, H, d, V, 1, delta, sigma_floor, chunk_pos, PRED_LINEAR, out_dtype, 0, 0, 0.0, zero_rate_D)
         self.W = 2 * L * H
         self._h = C.c_void_p()
         m = LinearModel(E.data_ptr(), A.data_ptr(), c.data_ptr(), dm)

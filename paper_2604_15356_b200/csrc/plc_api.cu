@@ -3,6 +3,7 @@
 #include <new>
 
 #include "plc_common.cuh"
+#include <cmath>
 
 namespace plc {
 static std::atomic<unsigned long long> g_launches{0};
@@ -82,6 +83,10 @@ CodecArgs base_args(const plc_ctx* c) {
     a.sh.delta = c->cfg.delta; a.sh.sigma_floor = c->cfg.sigma_floor;
     a.sh.inv_delta = 1.0f / c->cfg.delta;
     a.sh.inv_delta2 = (float)(1.0 / ((double)c->cfg.delta * (double)c->cfg.delta));
+    // zero-rate rule (Thm. 3): skip iff q <= floor(4 log2(D / delta^2) - 1/2), which implies sigma^2 <= D
+    a.sh.zero_q = c->cfg.zero_rate_D > 0.0f
+        ? (int)floor(4.0 * log2((double)c->cfg.zero_rate_D / ((double)c->cfg.delta * (double)c->cfg.delta)) - 0.5)
+        : kZeroOff;
     a.T = c->T; a.rownorm2 = c->rownorm2; a.pairs = c->pairs;
     a.staging = c->staging; a.staging_words_per_warp = c->staging_words_per_warp;
     a.ticket = c->ticket; a.status = c->status; a.counters = c->counters;
@@ -168,6 +173,7 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
     if (cfg->out_dtype != PLC_OUT_F32 && cfg->out_dtype != PLC_OUT_F16) return PLC_E_INVALID;
     if (cfg->adaptive_b0 < 0 || cfg->adaptive_b0 > 16 || cfg->adaptive_extra < 0 || cfg->adaptive_extra > 12) return PLC_E_INVALID;
     if (cfg->adaptive_b0 > 0 && !(cfg->adaptive_hbar > 0.0f)) return PLC_E_INVALID;
+    if (!(cfg->zero_rate_D >= 0.0f) || !(cfg->zero_rate_D < 1e30f)) return PLC_E_INVALID;
     if (cfg->adaptive_b0 > 0 && cfg->variant != PLC_PRED_TOPK) return PLC_E_STATE;
     if (cfg->variant != PLC_PRED_TOPK && 2 * cfg->n_kv_heads > 256) return PLC_E_SHAPE;
     if (T_dev && !aligned16(T_dev)) return PLC_E_ALIGN;
@@ -459,7 +465,7 @@ plc_status plc_get_stats(plc_ctx* c, plc_stats* out, int32_t reset, void* stream
     if (reset && cudaMemsetAsync(c->counters, 0, sizeof(h), st) != cudaSuccess) return PLC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
     out->payload_bytes = h.payload_bytes; out->n_chunks = h.n_chunks; out->n_escapes = h.n_escapes;
-    out->coded_vectors = h.coded_vectors;
+    out->coded_vectors = h.coded_vectors; out->skipped_vectors = h.skipped_vectors;
     return PLC_OK;
 }
 

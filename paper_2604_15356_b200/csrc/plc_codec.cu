@@ -384,7 +384,7 @@ __device__ __forceinline__ long long kv_elem(const KvView& v, int t, int H, int 
 
 // Finishes an encoded chunk: reserves its place, writes states and words, index and counters.
 __device__ __forceinline__ void commit_chunk(const CodecArgs& a, long long slot, uint32_t x, const uint16_t* stage,
-                                             int wp, int cap_words, int lane, int P, unsigned n_escapes) {
+                                             int wp, int cap_words, int lane, int P, unsigned n_escapes, int n_skipped = 0) {
     __syncwarp();
     const int n_words = cap_words - wp;
     const unsigned nbytes = 128u + 2u * (unsigned)n_words;
@@ -394,6 +394,7 @@ __device__ __forceinline__ void commit_chunk(const CodecArgs& a, long long slot,
         atomicAdd(&a.counters->payload_bytes, (unsigned long long)nbytes);
         atomicAdd(&a.counters->n_chunks, 1ull);
         atomicAdd(&a.counters->coded_vectors, (unsigned long long)P);
+        if (n_skipped) atomicAdd(&a.counters->skipped_vectors, (unsigned long long)n_skipped);
     }
     off = __shfl_sync(kFull, off, 0);
     if (lane == 0 && n_escapes) atomicAdd(&a.counters->n_escapes, (unsigned long long)n_escapes);
@@ -439,7 +440,8 @@ __device__ __forceinline__ void predict_dense(const CodecArgs& a, long long row,
 
 enum { kSrcGather = 0, kSrcOpen = 1, kSrcDense = 2 };
 
-template <int D, int SRC>
+// ZR: the zero-rate rule (Thm. 3) is on; a separate instantiation keeps the plain coder's loop free of it.
+template <int D, int SRC, bool ZR>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     constexpr bool FROM_OPEN = SRC == kSrcOpen;
@@ -478,6 +480,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
         uint32_t x = kRansL;
         int wp = cap_words;
         unsigned n_escapes = 0;
+        int n_skipped = 0;
         const int2* gp = nullptr;
         const __half* kvp = nullptr;
         int buf = 0;
@@ -492,9 +495,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
         for (int p = it.P - 1; p >= 0; --p) {
             int sym[G];
             int q;
+            bool skip;                                                             // zero-rate position (Thm. 3)
             if (FROM_OPEN) {
                 const long long o = ((long long)it.s * Wt + it.t) * a.sh.chunk_pos + p;
                 q = a.open_q[o];
+                skip = ZR && q <= a.sh.zero_q;
 #pragma unroll
                 for (int g = 0; g < G; ++g) sym[g] = a.open_sym[o * D + c0 + g];
             } else {
@@ -514,12 +519,15 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                     predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
                 }
                 float inv_delta_p = inv_delta, inv_delta2_p = inv_delta2;
+                int zero_q = ZR ? a.sh.zero_q : 0;
                 if (a.step_exp) {                                                  // adaptive step delta * 2^e
                     const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
                     inv_delta_p = ldexpf(inv_delta, -e);
                     inv_delta2_p = ldexpf(inv_delta2, -2 * e);
+                    if (ZR) zero_q -= 8 * e;                                       // same D against a step 2^e times larger
                 }
                 q = scale_class(sigma2, floor2, inv_delta2_p);
+                skip = ZR && q <= zero_q;
                 float kvv[G];
                 load_half_vec<G>(kvp, kvv);
                 kvp -= a.kv.sp;
@@ -531,11 +539,12 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                     if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        if (a.dbg.sym) a.dbg.sym[o * D + c0 + g] = sym[g];
+                        if (a.dbg.sym) a.dbg.sym[o * D + c0 + g] = skip ? 0 : sym[g];
                         if (a.dbg.mu) a.dbg.mu[o * D + c0 + g] = mu[g];
                     }
                 }
             }
+            if (ZR && skip) { ++n_skipped; continue; }                             // nothing is coded
             int s, qp;
             class_params(q, s, qp);
             const PosCode pc = pos_code(s);
@@ -543,12 +552,12 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
 #pragma unroll
             for (int g = G - 1; g >= 0; --g) wp = encode_step(sym[g], pc, tbl, x, stage, wp, lane, lt, n_escapes);
         }
-        commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes);
+        commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes, n_skipped);
         __syncwarp();
     }
 }
 
-template <int D, bool DENSE>
+template <int D, bool DENSE, bool ZR>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     __shared__ DecTables tb;
@@ -603,24 +612,31 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
                 predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
             }
             float delta_p = delta, inv_delta2_p = inv_delta2;
+            int zero_q = ZR ? a.sh.zero_q : 0;
             if (a.step_exp) {
                 const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
                 delta_p = ldexpf(delta, e);
                 inv_delta2_p = ldexpf(inv_delta2, -2 * e);
+                if (ZR) zero_q -= 8 * e;
             }
             const int q = scale_class(sigma2, floor2, inv_delta2_p);
             __syncwarp();                                                         // readers of this slot are done
-            int s, qp;
-            class_params(q, s, qp);
-            const PosCode pc = pos_code(s);
-            const uint16_t* cum = tb.cum[qp - kQMin];
-            const uint32_t* fcs = tb.fc[qp - kQMin];
             int sym[G];
             float out[G];
+            if (ZR && q <= zero_q) {                                              // zero-rate position: KV' = KV^
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                sym[g] = decode_step(pc, cum, fcs, x, words, rp, nwords, lane, lt, bad);
-                out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
+                for (int g = 0; g < G; ++g) { sym[g] = 0; out[g] = mu[g]; }
+            } else {
+                int s, qp;
+                class_params(q, s, qp);
+                const PosCode pc = pos_code(s);
+                const uint16_t* cum = tb.cum[qp - kQMin];
+                const uint32_t* fcs = tb.fc[qp - kQMin];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    sym[g] = decode_step(pc, cum, fcs, x, words, rp, nwords, lane, lt, bad);
+                    out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
+                }
             }
             store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
             kvo += a.kv.sp;
@@ -667,7 +683,7 @@ __global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecAr
         const long long o = ((long long)b * Wt + t) * a.sh.chunk_pos + a.open_slot;
         if (lane == 0) a.open_q[o] = q;
 #pragma unroll
-        for (int g = 0; g < G; ++g) a.open_sym[o * D + c0 + g] = quantise(kvv[g], mu[g], inv_delta);
+        for (int g = 0; g < G; ++g) a.open_sym[o * D + c0 + g] = q <= a.sh.zero_q ? 0 : quantise(kvv[g], mu[g], inv_delta);
     }
 }
 
@@ -714,13 +730,15 @@ cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, c
 cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
+    const bool zr = a.sh.zero_q != kZeroOff;
     return dispatch_d(a.sh.d, [&](auto D) {
         if (a.mu_dense) {
-            encode_kernel<decltype(D)::value, kSrcDense><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+            auto kd = zr ? encode_kernel<decltype(D)::value, kSrcDense, true> : encode_kernel<decltype(D)::value, kSrcDense, false>;
+            kd<<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
             count_launch();
             return cudaGetLastError();
         }
-        auto kern = encode_kernel<decltype(D)::value, kSrcGather>;
+        auto kern = zr ? encode_kernel<decltype(D)::value, kSrcGather, true> : encode_kernel<decltype(D)::value, kSrcGather, false>;
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
@@ -737,7 +755,8 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
         long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (long long)sm_count() * kBlocksPerSM) blocks = (long long)sm_count() * kBlocksPerSM;
-        encode_kernel<decltype(D)::value, kSrcOpen><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        auto ko = a.sh.zero_q != kZeroOff ? encode_kernel<decltype(D)::value, kSrcOpen, true> : encode_kernel<decltype(D)::value, kSrcOpen, false>;
+        ko<<<(unsigned)blocks, kThreads, 0, st>>>(a);
         count_launch();
         return cudaGetLastError();
     });
@@ -746,13 +765,15 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
 cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
+    const bool zr = a.sh.zero_q != kZeroOff;
     return dispatch_d(a.sh.d, [&](auto D) {
         if (a.mu_dense) {
-            decode_kernel<decltype(D)::value, true><<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
+            auto kd = zr ? decode_kernel<decltype(D)::value, true, true> : decode_kernel<decltype(D)::value, true, false>;
+            kd<<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
             count_launch();
             return cudaGetLastError();
         }
-        auto kern = decode_kernel<decltype(D)::value, false>;
+        auto kern = zr ? decode_kernel<decltype(D)::value, false, true> : decode_kernel<decltype(D)::value, false, false>;
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;

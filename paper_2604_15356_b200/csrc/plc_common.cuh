@@ -25,7 +25,7 @@ constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u, kStTimeout = 8u;
 
 // Device counters (plc_stats).
 struct Counters {
-    unsigned long long payload_bytes, n_chunks, n_escapes, coded_vectors;
+    unsigned long long payload_bytes, n_chunks, n_escapes, coded_vectors, skipped_vectors;
 };
 
 // Frequency-table entry used by the encoder: rcp = floor(2^32 / f) (2^32-1 for f = 1),
@@ -161,10 +161,13 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st);
 cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,
                                 int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st);
 
+constexpr int kZeroOff = -1000000;
+
 struct CodecShape {
     int L, H, d, V, K, Kp, chunk_pos, out_dtype;   // Kp: K rounded up to the rows one warp-wide load fetches
     float delta, sigma_floor;
     float inv_delta, inv_delta2;   // fl(1/delta), fl(1/(delta*delta)), rounded once on the host
+    int zero_q;                    // zero-rate rule (Thm. 3): positions of class <= zero_q carry no symbols (kZeroOff = never)
 };
 
 struct KvView {

@@ -193,6 +193,16 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
     return tokens, prefix_keys(tokens), leaf, plen
 
 
+def peaked_logits(S, n, V, seed, lo=0.5, hi=40.0, device="cpu"):
+    """Logits [S][n][V] float16 whose entropy differs widely from position to position:
+    row = scale * N(0,1)^V with scale log-uniform in [lo, hi] (near-uniform rows up to point masses)."""
+    g = _gen(seed, device)
+    base = torch.randn(S, n, V, generator=g, device=device, dtype=torch.float32)
+    u = torch.rand(S, n, generator=g, device=device, dtype=torch.float32)
+    scale = torch.exp(math.log(lo) + u * (math.log(hi) - math.log(lo)))
+    return (base * scale[..., None]).to(torch.float16)
+
+
 def make_linear_model(L, H, V, d, dm, seed, device="cpu"):
     """Parameters of a KV function that is linear in the token embedding, F(t) = c + A E(t):
     E [V][dm] ~ N(0,1), A [L][2][H][d][dm] ~ N(0, 1/dm), c [L][2][H][d] ~ N(0, 0.01), all float16."""

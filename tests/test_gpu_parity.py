@@ -481,6 +481,124 @@ def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
     assert total < 0.8 * S * n * W * d * 2
 
 
+@pytest.mark.parametrize("adaptive", [False, True])
+def test_zero_rate_rule_parity(dev, orc, adaptive):
+    """Thm. 3 / Cor. 6: positions whose class is at most floor(4 log2(D / step^2) - 1/2) carry no
+    symbols and decode to the prediction.  The decision is the integer class, so wherever the GPU's
+    class equals the oracle's the same positions are skipped; the stream of a chunk is the oracle
+    coder's stream of the kept positions; counters agree; the rule follows the adaptive step."""
+    S, n, L, H, d, V, K, CP, delta, D = 2, 150, 1, 2, 128, 512, 32, 64, 0.02, 0.05
+    logits = synth.peaked_logits(S, n, V, 811)
+    g = torch.Generator().manual_seed(812)
+    tokens = torch.randint(0, V, (S, n), generator=g, dtype=torch.int32)
+    T = synth.make_tables(L, H, V, d, 813)
+    kv = synth.make_kv(T, tokens, 0.05, 814)
+    b0, extra = 6, 4
+    _, _, _, _, lp = orc.topk_softmax(logits.numpy().reshape(S * n, V), tokens.numpy().reshape(-1), K)
+    hbar = float(-lp.mean())
+    ad = (b0, extra, hbar) if adaptive else None
+    ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, adaptive=ad, zero_rate_D=D)
+    W, mc = ctx.W, ctx.max_chunks(n)
+    st = plc.StreamSet(S * W, mc, S * W * mc * 160 + 4 * S * n * W * d + 4096, dev)
+    sym = torch.full((S, n, W, d), 7, dtype=torch.int32, device=dev)
+    q = torch.zeros(S, n, W, dtype=torch.int32, device=dev)
+    mu = torch.zeros(S, n, W, d, dtype=torch.float32, device=dev)
+    bits = torch.zeros(S, n, dtype=torch.int32, device=dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    tkd = tokens.to(dev) if adaptive else None
+    ctx.encode(kvd, lgd, st, debug=plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr(), bits.data_ptr()), tokens=tkd)
+    assert ctx.sync_status() == plc.OK
+    stats = ctx.stats()
+    cfg = orc.Config(L, H, d, V, K, delta, 0.0, CP, 0, *((b0, extra, hbar) if adaptive else (0, 0, 0.0)))
+    cfg.zero_D = D
+    enc = orc.encode(cfg, T.numpy(), kv.numpy(), logits.numpy(), tokens.numpy() if adaptive else None, export=True)
+    sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W)
+    sym_g, q_g, mu_g = sym.cpu().numpy(), q.cpu().numpy(), mu.cpu().numpy()
+    if adaptive:
+        bits_g = bits.cpu().numpy()
+        assert (bits_g == enc["bits"]).mean() > 0.99
+        step = delta * 2.0 ** (b0 - bits_g.astype(np.float64))                   # [S][n]
+    else:
+        step = np.full((S, n), delta)
+    zc = np.array([[orc.zero_class(D, float(step[s_, i])) for i in range(n)] for s_ in range(S)])
+    skip_g = q_g <= zc[:, :, None]
+    assert 0.1 < skip_g.mean() < 0.9                                         # both branches are exercised
+    bsame = (bits_g == enc["bits"]) if adaptive else np.ones((S, n), bool)      # a different depth moves q by 8
+    # sigma^2 = s1 - ||mu||^2/d cancels for peaked distributions (s1 = O(1)): its binary32 error, 1e-7 absolute, is
+    # relatively small only where sigma^2 itself is not tiny, so the classes are compared where sigma^2 >= 1e-3
+    s2_o = (step[:, :, None] ** 2) * 2.0 ** (q_o / 4.0)
+    big = bsame[:, :, None] & (s2_o >= 1e-3)
+    assert big.mean() > 0.3 and (q_g[big] != q_o[big]).mean() < 1e-2 and np.abs(q_g[big] - q_o[big]).max() <= 1
+    assert (q_g[bsame] != q_o[bsame]).mean() < 5e-2
+    same = (q_g == q_o) & bsame[:, :, None]
+    assert np.array_equal(skip_g[same], (q_o <= zc[:, :, None])[same])
+    assert not sym_g[skip_g].any()
+    assert (sym_g[same & ~skip_g] != sym_o[same & ~skip_g]).mean() < 1e-4
+    assert stats.skipped_vectors == int(skip_g.sum()) and stats.coded_vectors == S * n * W
+    total = 0
+    for s_ in range(S):
+        for t_ in range(W):
+            for c in range(mc):
+                P = min(CP, n - c * CP)
+                sl = slice(c * CP, c * CP + P)
+                qq = np.where(skip_g[s_, sl, t_], orc.q_skip(), q_g[s_, sl, t_]).astype(np.int32)
+                ref, _, _ = orc.rans_encode_chunk(sym_g[s_, sl, t_], qq)
+                assert np.array_equal(st.chunk((s_ * W + t_) * mc + c), ref), (s_, t_, c)
+                total += len(ref)
+    assert total == stats.payload_bytes
+    if (q_g == q_o).all() and (not adaptive or (bits_g == enc["bits"]).all()):
+        assert abs(total / enc["stats"].payload_bytes - 1) < 2e-3
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    sym2 = torch.full_like(sym, 9)
+    ctx.decode(st, lgd, out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None), tokens=tkd)
+    assert ctx.sync_status() == plc.OK
+    assert torch.equal(sym2, sym)
+    o = out.cpu().numpy()                                                     # [L][2][S][H][n][d]
+    o = np.transpose(o, (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)
+    kvv = np.transpose(kv.numpy().astype(np.float64), (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)
+    assert np.array_equal(o[skip_g], mu_g[skip_g])                            # KV' = KV^ bit for bit
+    err = np.abs(o - kvv).max(-1)
+    assert (err[~skip_g] <= (step[:, :, None] * np.ones((1, 1, W)))[~skip_g] / 2 + 1e-3).all()
+    # and the rule off reproduces the plain coder's size, which is larger
+    ctx0 = plc.Context(T.to(dev), K, delta, chunk_pos=CP, adaptive=ad)
+    st0 = plc.StreamSet(S * W, mc, S * W * mc * 160 + 4 * S * n * W * d + 4096, dev)
+    ctx0.encode(kvd, lgd, st0, tokens=tkd)
+    assert ctx0.sync_status() == plc.OK
+    s0 = ctx0.stats()
+    assert s0.skipped_vectors == 0 and s0.payload_bytes > stats.payload_bytes
+
+
+def test_zero_rate_rule_on_the_append_path(dev, orc):
+    """The append path stores zero symbols for skipped positions and seals chunks without them:
+    chunk for chunk the bytes of a bulk encode with the same rule."""
+    B, steps, L, H, d, V, K, CP, delta, D = 3, 70, 1, 2, 64, 512, 32, 32, 0.02, 0.05
+    logits = synth.peaked_logits(B, steps, V, 821)
+    g = torch.Generator().manual_seed(822)
+    tokens = torch.randint(0, V, (B, steps), generator=g, dtype=torch.int32)
+    T = synth.make_tables(L, H, V, d, 823)
+    kv = synth.make_kv(T, tokens, 0.05, 824)
+    ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, zero_rate_D=D)
+    W, mc = ctx.W, 3
+    st = plc.StreamSet(B * W, mc, 3 * B * steps * W * d + 4096, dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    ctx.encode(kvd, lgd, st)
+    assert ctx.sync_status() == plc.OK
+    bulk = ctx.stats(reset=True)
+    assert 0 < bulk.skipped_vectors < B * steps * W
+    sb = ctx.new_session_batch(B, mc, 3 * B * steps * W * d + 4096)
+    for i in range(steps):
+        ctx.append_step(sb, kvd[:, :, :, :, i, :].contiguous(), lgd[:, i, :].contiguous())
+    ctx.append_flush(sb)
+    assert ctx.sync_status() == plc.OK
+    app = ctx.stats()
+    assert app.skipped_vectors == bulk.skipped_vectors and app.payload_bytes == bulk.payload_bytes
+    for slot in range(B * W * mc):
+        assert np.array_equal(sb.streams.chunk(slot), st.chunk(slot)), slot
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    ctx.decode(sb.streams, lgd, out)
+    assert ctx.sync_status() == plc.OK
+
+
 def test_adaptive_quantiser_parity(dev, orc):
     """Def. 7: per-position step delta * 2^(b0 - b_i), b_i from the surprisal of the actual token.
     b_i is an integer decided in binary32 from a binary32 surprisal, so a position may get a different
