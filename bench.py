@@ -134,6 +134,8 @@ def main():
                     help="prediction: top-K gather (default), full-vocabulary bf16 tensor-core contraction, or the "
                          "linear-embedding model of Sec. 7.1 (two chained contractions; see --d-model)")
     ap.add_argument("--d-model", type=int, default=4096, help="embedding width of --variant linear")
+    ap.add_argument("--sigma-floor", type=float, default=0.0,
+                    help="standard deviation added in quadrature to the mixture's before the scale class is taken")
     ap.add_argument("--zero-rate", type=float, default=0.0,
                     help="D > 0: zero-rate rule (Thm. 3), positions with mixture variance <= D carry no symbols")
     args = ap.parse_args()
@@ -180,10 +182,11 @@ def main():
     tok = w["tokens"] if adaptive else None
     if linear:
         ctx = plc.Context.linear(w["E"], w["A"], w["c"], cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                                 zero_rate_D=args.zero_rate)
+                                 zero_rate_D=args.zero_rate, sigma_floor=args.sigma_floor)
     else:
         ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                          variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive, zero_rate_D=args.zero_rate)
+                          variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive, zero_rate_D=args.zero_rate,
+                          sigma_floor=args.sigma_floor)
         ctx.reserve(S * n)
     ctx.set_profiling(True)
     mc = ctx.max_chunks(n)
@@ -260,7 +263,7 @@ def main():
     fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
     fma_ach = vecs * K * d / (dom_ms / 1e3)
     dom_name = "encode_kernel" if dom_enc else "decode_kernel"
-    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive and not linear and not args.zero_rate
+    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive and not linear and not args.zero_rate and not args.sigma_floor
     traffic = NCU_DRAM_BYTES_PER_VECTOR[dom_name] * vecs if default_cfg else None
     roofline = {"kernel": dom_name, "bound": "hbm",
                 "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
@@ -306,7 +309,7 @@ def main():
         def make_ctx(Tslice):
             return plc.Context(Tslice, K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
                                variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive,
-                               zero_rate_D=args.zero_rate)
+                               zero_rate_D=args.zero_rate, sigma_floor=args.sigma_floor)
         e2e = run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok, args.e2e_groups)
 
     cpu = None
@@ -325,7 +328,7 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
                        "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
-                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant, "adaptive_b0": args.adaptive, "zero_rate_D": args.zero_rate,
+                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant, "adaptive_b0": args.adaptive, "zero_rate_D": args.zero_rate, "sigma_floor": args.sigma_floor,
                        "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
             "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
             "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),
