@@ -252,6 +252,16 @@ def prefix_dedup(tokens, lens, logp2):
     return lcp, dT, parent, shared
 
 
+def prefix_clusters(lcp, dT, delta):
+    """Def. 3 on the matrices of prefix_dedup -> cluster [S] (smallest member), centroid [S], begin [S]."""
+    lcp = np.ascontiguousarray(lcp, dtype=np.int32)
+    dT = np.ascontiguousarray(dT, dtype=np.float64)
+    S = lcp.shape[0]
+    cl, ce, be = (np.zeros(S, np.int32) for _ in range(3))
+    lib().plo_prefix_clusters(_p(lcp), _p(dT), S, C.c_double(delta), _p(cl), _p(ce), _p(be))
+    return cl, ce, be
+
+
 def _strides(kv):
     """kv laid out [L,2,S,H,n,d] (any permutation of a contiguous array works): element strides."""
     es = kv.itemsize

@@ -531,6 +531,30 @@ void plo_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* l
     }
 }
 
+/* Def. 3 (semantic prefix cluster at threshold delta; centroid = its most probable member) on the
+ * matrices of plo_prefix_dedup.  Reading taken: with d_T = -log2 P(s ^ s') (Def. 2) a LONGER shared
+ * prefix gives a LARGER d_T, and d_T(a,c) >= min(d_T(a,b), d_T(b,c)); the relation the definition
+ * needs -- one whose maximal subsets are unique -- is therefore "the shared prefix carries at least
+ * delta bits", d_T(s,s') >= delta, which is an equivalence by that inequality (the printed "<="
+ * is not: it would separate exactly the sessions that share the most).  A session is always a member
+ * of its own cluster.  cluster[s] = smallest member index; centroid[s] = member with the largest
+ * P(s') = 2^-d_T(s',s') (ties: smallest index); begin[s] = first position of s that is not covered by
+ * the centroid's cache (0 for the centroid itself): the tail Cor. 3 charges for. */
+void plo_prefix_clusters(const int32_t* lcp /*[S][S]*/, const double* dT /*[S][S]*/, int S, double delta,
+                         int32_t* cluster, int32_t* centroid, int32_t* begin) {
+    for (int a = 0; a < S; ++a) {
+        int first = a, best = a;
+        for (int b = 0; b < S; ++b) {
+            if (b != a && !(dT[(size_t)a * S + b] >= delta)) continue;
+            if (b < first) first = b;
+            double pb = dT[(size_t)b * S + b], pbest = dT[(size_t)best * S + best];
+            if (pb < pbest || (pb == pbest && b < best)) best = b;
+        }
+        cluster[a] = first; centroid[a] = best;
+        begin[a] = best == a ? 0 : lcp[(size_t)a * S + best];
+    }
+}
+
 /* ---------------------------------------------------------------- adaptive step */
 
 /* Def. 7 (surprisal-adaptive quantiser): at a position of surprisal h = -log2 P(x_i | x_<i) the
