@@ -36,7 +36,7 @@ def build(force=False, verbose=False):
     deps = srcs + [os.path.join(_CSRC, "plc_common.cuh"), os.path.join(_INC, "plc.h")]
     if not force and os.path.exists(_SO) and all(os.path.getmtime(_SO) >= os.path.getmtime(d) for d in deps):
         return _SO
-    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    cmd = ["nvcc", "-t", "0", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-shared", "-I" + _INC, "-o", _SO] + srcs
     if verbose:
         cmd.insert(1, "-Xptxas=-v")

@@ -186,7 +186,7 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
     const int warps = codec_grid_warps(0);
     bool ok = (!T_dev || cudaMalloc(&c->rownorm2, sizeof(float) * (size_t)rows) == cudaSuccess) &&
               cudaMalloc(&c->staging, sizeof(uint16_t) * c->staging_words_per_warp * warps) == cudaSuccess &&
-              cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->ticket, sizeof(unsigned int) * kTicketWords) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(unsigned int)) == cudaSuccess &&
               cudaMalloc(&c->counters, sizeof(Counters)) == cudaSuccess;
     if (ok) ok = cudaMemset(c->status, 0, sizeof(unsigned int)) == cudaSuccess &&

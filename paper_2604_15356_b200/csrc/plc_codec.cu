@@ -12,6 +12,7 @@
 // from chunk to chunk so it stays in L2), then reserves the chunk's final place with one atomicAdd
 // and copies it there.  Work items are handed out by an atomic ticket in table-major order so that
 // the warps running at any time gather from few tables.
+#include <algorithm>
 #include <type_traits>
 
 #include "plc_common.cuh"
@@ -25,7 +26,10 @@ namespace {
 #ifndef PLC_GATHER_UNROLL
 #define PLC_GATHER_UNROLL 8
 #endif
-constexpr int kWarpsPerBlock = 8;
+#ifndef PLC_WARPS_PER_BLOCK
+#define PLC_WARPS_PER_BLOCK 8
+#endif
+constexpr int kWarpsPerBlock = PLC_WARPS_PER_BLOCK;
 constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kBlocksPerSM = PLC_BLOCKS_PER_SM;
 constexpr int kGatherUnroll = PLC_GATHER_UNROLL;
@@ -101,12 +105,19 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const __half* __restrict__
     }
 }
 
-// Two binary32 fused multiply-adds in one instruction (sm_100 packed f32x2); each half is an
-// IEEE fma, so the result equals two scalar __fmaf_rn.
-__device__ __forceinline__ void ffma2(float& a0, float& a1, float w, float x0, float x1) {
-    asm("{ .reg .b64 ra, rb, rc;\n mov.b64 ra, {%2,%2};\n mov.b64 rb, {%3,%4};\n mov.b64 rc, {%0,%1};\n"
-        " fma.rn.f32x2 rc, ra, rb, rc;\n mov.b64 {%0,%1}, rc; }"
-        : "+f"(a0), "+f"(a1) : "f"(w), "f"(x0), "f"(x1));
+// Two binary32 fused multiply-adds in one instruction (sm_100 packed f32x2) on register pairs that
+// stay packed across the gather loop; each half is an IEEE fma, so the result equals two scalar
+// __fmaf_rn.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void ffma2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
 
 // Mixture of one position for one table.  sp: the position's Kp {idx, w} entries in shared memory,
@@ -123,9 +134,7 @@ __device__ __forceinline__ void predict(const char* __restrict__ col, const floa
         const int2 pr = sp[k];
         s1 = __fmaf_rn(__int_as_float(pr.y), __ldg(n2 + pr.x), s1);
     }
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    unsigned long long acc2[4] = {0ull, 0ull, 0ull, 0ull};   // four pairs of +0.f
     const int2* pl = sp + h;
     const int iters = Kp / ROWS;
 #pragma unroll kGatherUnroll
@@ -133,13 +142,17 @@ __device__ __forceinline__ void predict(const char* __restrict__ col, const floa
         const int2 pr = pl[it * ROWS];
         const float w = __int_as_float(pr.y);
         const uint4 r = __ldg(reinterpret_cast<const uint4*>(col + (long long)pr.x * (D * 2)));
+        const unsigned long long ww = pack2(w, w);
         const __half2* hp = reinterpret_cast<const __half2*>(&r);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float2 f = __half22float2(hp[j]);
-            ffma2(acc[2 * j], acc[2 * j + 1], w, f.x, f.y);
+            ffma2(acc2[j], ww, pack2(f.x, f.y));
         }
     }
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) unpack2(acc2[j], acc[2 * j], acc[2 * j + 1]);
     // reduce-scatter over the ROWS lanes that hold partial sums of the same 8 components
     int cnt = 8;
 #pragma unroll
@@ -185,128 +198,193 @@ __device__ __forceinline__ int scale_class(float sigma2, float floor2, float inv
     return class_from_v((sigma2 + floor2) * inv_delta2);
 }
 
-__device__ __forceinline__ int join_sym(int hi, uint32_t lo, int s) {
-    if (s == 0) return hi;
-    return (int)(((uint32_t)hi << s) + lo - (1u << (s - 1)));
-}
-
-// Values that are the same for all components of one position.
-struct PosCode {
-    int s;               // bit planes
-    uint32_t half;       // 2^(s-1), 0 when s = 0
-    uint32_t lomask;     // 2^s - 1
+// Per-lane constants of the coder steps.
+struct LaneCode {
+    uint32_t lt;         // lanes below this one
+    int sh;              // 16 * (lane & 1): which half of a bit-plane word lanes 0 / 1 store
+    int hs;              // lane >> 4: which half of a bit-plane word this lane's bit sits in
+    uint32_t bit;        // 1 << (lane & 15): this lane's bit in that half
+    int lane;
 };
-__device__ __forceinline__ PosCode pos_code(int s) {
-    PosCode pc;
-    pc.s = s;
-    pc.half = s ? (1u << (s - 1)) : 0u;
-    pc.lomask = (1u << s) - 1u;
-    return pc;
+__device__ __forceinline__ LaneCode lane_code(int lane) {
+    LaneCode lc;
+    lc.lt = lanemask_lt(); lc.sh = 16 * (lane & 1); lc.hs = lane >> 4; lc.bit = 1u << (lane & 15); lc.lane = lane;
+    return lc;
 }
 
-// One encoder step for the warp: every lane codes `sym`.  Words are written back to front at
-// stage[wp-1], stage[wp-2], ...; returns the new wp.
-__device__ __forceinline__ int encode_step(int sym, const PosCode pc, const EncEntry* tbl, uint32_t& x,
-                                           uint16_t* __restrict__ stage, int wp, int lane, uint32_t lt,
-                                           unsigned& n_escapes) {
-    const int u = sym + (int)pc.half;              // |sym| <= 2^30, s <= 15: no overflow
-    const int hi = u >> pc.s;
-    const uint32_t lo = (uint32_t)u & pc.lomask;
-    const bool esc = (uint32_t)(hi + kHiMax) > 2u * kHiMax;
+// One encoder step for the warp: every lane codes `sym` with S raw bit planes (S is the same in
+// all lanes).  Words are written back to front at stage[wp-1], stage[wp-2], ...; returns the new
+// wp.  In decoder order a step is: 2S plane words, the refill words of the lanes that renormalise
+// (lanes ascending), the raw high parts of escaped lanes (lanes ascending, low half first).
+template <int SC>
+__device__ __forceinline__ int encode_step(int sym, int s_dyn, const EncEntry* tbl, uint32_t& x, uint16_t* __restrict__ stage,
+                                           int wp, const LaneCode& lc, unsigned& n_escapes) {
+    const int S = SC >= 0 ? SC : s_dyn;                            // SC < 0: plane count known at run time only
+    const int S2 = 2 * S;
+    const int u = sym + (S ? (1 << (S - 1)) : 0);                  // |sym| <= 2^30, S <= 15: no overflow
+    const int hi = u >> S;                                         // bits below S of u are the raw part
     const int nh = -hi;
-    const int zz = esc ? kEsc : ((nh << 1) ^ (nh >> 31));     // 0, +1 -> 1, -1 -> 2, +2 -> 3, ...
-    const EncEntry e = tbl[zz];
-    const uint32_t f = e.fc & 0xffffu, c = e.fc >> 16;
+    const uint32_t zz0 = (uint32_t)((nh << 1) ^ (nh >> 31));       // 0, +1 -> 1, -1 -> 2, +2 -> 3, ...
+    const bool esc = zz0 > 2u * kHiMax;                            // |hi| > 31
+    const EncEntry e = tbl[min(zz0, (uint32_t)kEsc)];
+    const uint32_t f = e.fc & 0xffffu;
     const bool emit = x >= (f << 17);
     const uint32_t emask = __ballot_sync(kFull, emit);
-    const int s2 = 2 * pc.s;
-    int base = wp - s2 - __popc(emask);
+    int base = wp - S2 - __popc(emask);
     if (__any_sync(kFull, esc)) {                  // rare: raw 32-bit hi of the escaped lanes
         const uint32_t xmask = __ballot_sync(kFull, esc);
         const int n_esc = __popc(xmask);
         base -= 2 * n_esc;
         if (esc) {
-            const int at = base + s2 + __popc(emask) + 2 * __popc(xmask & lt);
+            const int at = base + S2 + __popc(emask) + 2 * __popc(xmask & lc.lt);
             stage[at] = (uint16_t)((uint32_t)hi & 0xffffu);
             stage[at + 1] = (uint16_t)((uint32_t)hi >> 16);
         }
         n_escapes += n_esc;
     }
-    if (emit) {
-        stage[base + s2 + __popc(emask & lt)] = (uint16_t)(x & 0xffffu);
-        x >>= 16;
-    }
-    uint32_t q = __umulhi(x, e.rcp);
-    uint32_t r = x - q * f;
+    uint16_t* out = stage + base;
+    if (emit) out[S2 + __popc(emask & lc.lt)] = (uint16_t)(x & 0xffffu);
+    const uint32_t xe = emit ? x >> 16 : x;
+    uint32_t q = __umulhi(xe, e.rcp);
+    uint32_t r = xe - q * f;
     if (r >= f) { ++q; r -= f; }
-    x = (q << kProbBits) + r + c;
-    if (pc.s) {
-        uint32_t mine = 0;
-        const int myb = lane >> 1;
-        for (int b = 0; b < pc.s; ++b) {
-            const uint32_t plane = __ballot_sync(kFull, (lo >> b) & 1u);
-            if (myb == b) mine = plane;
+    x = (q << kProbBits) + r + (e.fc >> 16);
+    if (S > 0) {
+        uint16_t* mine = out + lc.lane;            // lanes 0 and 1 store the two halves of every plane
+#pragma unroll
+        for (int b = 0; b < S; ++b) {
+            const uint32_t plane = __ballot_sync(kFull, (u >> b) & 1);
+            if (lc.lane < 2) mine[2 * b] = (uint16_t)(plane >> lc.sh);
         }
-        if (lane < s2) stage[base + lane] = (uint16_t)((lane & 1) ? (mine >> 16) : mine);
     }
     return base;
 }
 
-// One decoder step for the warp; words[0 .. nwords) are readable.
-__device__ __forceinline__ int decode_step(const PosCode pc, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
-                                           const uint16_t* __restrict__ words, int& rp, int nwords, int lane,
-                                           uint32_t lt, bool& bad) {
+// All G components of one position, last component first, dispatched on the number of planes.
+template <int G>
+__device__ __forceinline__ int encode_position(const int (&sym)[G], int s, const EncEntry* tbl, uint32_t& x,
+                                               uint16_t* __restrict__ stage, int wp, const LaneCode& lc, unsigned& n_escapes) {
+#define PLC_ENC_CASE(S_, LABEL)                                                                            \
+    LABEL:                                                                                                 \
+        _Pragma("unroll") for (int g = G - 1; g >= 0; --g)                                                 \
+            wp = encode_step<S_>(sym[g], s, tbl, x, stage, wp, lc, n_escapes);                             \
+        break;
+    switch (s) {       // the plane counts that occur in practice get code of their own
+        PLC_ENC_CASE(0, case 0) PLC_ENC_CASE(1, case 1) PLC_ENC_CASE(2, case 2) PLC_ENC_CASE(3, case 3)
+        PLC_ENC_CASE(4, case 4) PLC_ENC_CASE(5, case 5) PLC_ENC_CASE(6, case 6) PLC_ENC_CASE(7, case 7)
+        PLC_ENC_CASE(-1, default)
+    }
+#undef PLC_ENC_CASE
+    return wp;
+}
+
+// One decoder step for the warp; words[-1 .. nwords) are readable (words[-1] is the last half of
+// the chunk's state block).  A read past the end is redirected to the chunk's last word; rp still
+// advances, so the caller's final check rp == nwords reports it.
+template <int SC>
+__device__ __forceinline__ int decode_step(int s_dyn, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
+                                           const uint16_t* __restrict__ words, int& rp, int last, const LaneCode& lc) {
+    const int S = SC >= 0 ? SC : s_dyn;
     uint32_t lo = 0;
-    if (pc.s) {
-        const int s2 = 2 * pc.s;
+    if (S > 0) {
+        const int S2 = 2 * S;
         uint32_t v = 0;
-        if (lane < s2) {
-            const int at = rp + lane;
-            if (at < nwords) v = __ldg(words + at); else bad = true;
+        if (lc.lane < S2) v = __ldg(words + min(rp + lc.lane, last));
+#pragma unroll
+        for (int b = 0; b < S; ++b) {
+            const uint32_t hw = __shfl_sync(kFull, v, 2 * b + lc.hs);
+            if (hw & lc.bit) lo |= 1u << b;
         }
-        const int hs = lane >> 4, sh = lane & 15;    // which half of the plane word, which bit of it
-        for (int b = 0; b < pc.s; ++b) {
-            const uint32_t hw = __shfl_sync(kFull, v, 2 * b + hs);
-            lo |= ((hw >> sh) & 1u) << b;
-        }
-        rp += s2;
+        rp += S2;
     }
     const uint32_t slot = x & (kProbM - 1u);
-    int zz = 0;
+    const uint16_t* cp = cum;
 #pragma unroll
     for (int step = 32; step > 0; step >>= 1)
-        if (cum[zz + step] <= slot) zz += step;
+        if (cp[step] <= slot) cp += step;
+    const int zz = (int)(cp - cum);
     const uint32_t fc = fcs[zz];
-    const uint32_t f = fc & 0xffffu, c = fc >> 16;
-    x = f * (x >> kProbBits) + slot - c;
+    x = (fc & 0xffffu) * (x >> kProbBits) + slot - (fc >> 16);
     const bool need = x < kRansL;
     const uint32_t nmask = __ballot_sync(kFull, need);
-    if (need) {
-        const int at = rp + __popc(nmask & lt);
-        uint32_t w = 0;
-        if (at < nwords) w = __ldg(words + at); else bad = true;
-        x = (x << 16) | w;
-    }
+    if (need) x = (x << 16) | __ldg(words + min(rp + __popc(nmask & lc.lt), last));
     rp += __popc(nmask);
-    const bool esc = zz == kEsc;
-    int hi = (zz & 1) ? (zz + 1) >> 1 : -(zz >> 1);
-    if (__any_sync(kFull, esc)) {
+    const int t = (zz + 1) >> 1;
+    int hi = (zz & 1) ? t : -t;
+    if (__any_sync(kFull, zz == kEsc)) {
+        const bool esc = zz == kEsc;
         const uint32_t xmask = __ballot_sync(kFull, esc);
         if (esc) {
-            const int at = rp + 2 * __popc(xmask & lt);
-            uint32_t a = 0, b = 0;
-            if (at + 1 < nwords) { a = __ldg(words + at); b = __ldg(words + at + 1); } else bad = true;
-            hi = (int)(a | (b << 16));
+            const int at = rp + 2 * __popc(xmask & lc.lt);
+            hi = (int)((uint32_t)__ldg(words + min(at, last)) | ((uint32_t)__ldg(words + min(at + 1, last)) << 16));
         }
         rp += 2 * __popc(xmask);
     }
-    return join_sym(hi, lo, pc.s);
+    return S ? (int)(((uint32_t)hi << S) + lo - (1u << (S - 1))) : hi;
 }
 
+template <int G>
+__device__ __forceinline__ void decode_position(int (&sym)[G], int s, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
+                                                const uint16_t* __restrict__ words, int& rp, int last, const LaneCode& lc) {
+#define PLC_DEC_CASE(S_, LABEL)                                                                            \
+    LABEL:                                                                                                 \
+        _Pragma("unroll") for (int g = 0; g < G; ++g)                                                      \
+            sym[g] = decode_step<S_>(s, cum, fcs, x, words, rp, last, lc);                                 \
+        break;
+    switch (s) {
+        PLC_DEC_CASE(0, case 0) PLC_DEC_CASE(1, case 1) PLC_DEC_CASE(2, case 2) PLC_DEC_CASE(3, case 3)
+        PLC_DEC_CASE(4, case 4) PLC_DEC_CASE(5, case 5) PLC_DEC_CASE(6, case 6) PLC_DEC_CASE(7, case 7)
+        PLC_DEC_CASE(-1, default)
+    }
+#undef PLC_DEC_CASE
+}
+
+// Lane 0's value for the whole warp, through a warp reduction: the result is provably the same in
+// every lane, so everything derived from it (loop bounds, table addresses, branches) is kept out of
+// the per-lane registers and needs no divergence handling.
+__device__ __forceinline__ unsigned from_lane0(unsigned v, int lane) {
+    return __reduce_or_sync(kFull, lane == 0 ? v : 0u);
+}
 __device__ __forceinline__ unsigned next_ticket(unsigned int* ticket, int lane) {
     unsigned t = 0;
     if (lane == 0) t = atomicAdd(ticket, 1u);
-    return __shfl_sync(kFull, t, 0);
+    return from_lane0(t, lane);
+}
+
+// Work queues of the gather kernels.  The tables are dealt round-robin to nq queues (queue k owns
+// tables k, k + nq, ...), each queue lists its (table, session, chunk) items table-major, and the
+// g SMs with the same smid / g serve one queue.  The warps resident on an SM therefore gather from
+// one or two tables at a time, so candidate rows that several positions share are found in that
+// SM's L1, and the number of tables in flight on the whole GPU stays near nq.  A warp whose queue
+// is empty moves on to the next queue (and never returns), so the tail is balanced by stealing.
+// Returns the item in table-major numbering (table * per_table + rest), or ~0u when all is taken.
+__device__ __forceinline__ unsigned smid() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
+    return r;
+}
+struct QueueCursor { int q, tried; };
+__device__ __forceinline__ QueueCursor queue_of_this_sm(const CodecArgs& a) {
+    QueueCursor qc;
+    qc.q = min((int)(smid() / (unsigned)a.sched_g), a.sched_nq - 1);
+    qc.tried = 0;
+    return qc;
+}
+__device__ __forceinline__ unsigned next_queued(const CodecArgs& a, QueueCursor& qc, unsigned per_table, int n_tables, int lane) {
+    unsigned item = ~0u;
+    if (lane == 0) {
+        while (qc.tried < a.sched_nq) {
+            const unsigned nt = (unsigned)max(0, (n_tables - qc.q + a.sched_nq - 1) / a.sched_nq);
+            const unsigned j = atomicAdd(a.ticket + qc.q, 1u);
+            if (j < nt * per_table) {
+                item = ((unsigned)qc.q + (unsigned)a.sched_nq * (j / per_table)) * per_table + j % per_table;
+                break;
+            }
+            qc.q = qc.q + 1 == a.sched_nq ? 0 : qc.q + 1;
+            ++qc.tried;
+        }
+    }
+    return from_lane0(item, lane);
 }
 
 template <int G>
@@ -450,7 +528,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     build_enc_tables(&tb);
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const uint32_t lt = lanemask_lt();
+    const LaneCode lc = lane_code(lane);
     const long long gw = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     uint16_t* stage = a.staging + gw * a.staging_words_per_warp;
     const int cap_words = (int)a.staging_words_per_warp;
@@ -462,7 +540,11 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                 floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
 
-    for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
+    constexpr bool QUEUED = SRC == kSrcGather;
+    QueueCursor qc = QUEUED ? queue_of_this_sm(a) : QueueCursor{0, 0};
+    const unsigned per_table = (unsigned)a.S * (unsigned)a.st.max_chunks;
+    auto next = [&]() { return QUEUED ? next_queued(a, qc, per_table, Wl, lane) : next_ticket(a.ticket, lane); };
+    for (unsigned item = next(); item < total; item = next()) {
         Item it;
         if (FROM_OPEN) {
             it.t = (int)(item / a.S); it.s = (int)(item % a.S); it.c = a.chunk_index;
@@ -526,7 +608,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                     inv_delta2_p = ldexpf(inv_delta2, -2 * e);
                     if (ZR) zero_q -= 8 * e;                                       // same D against a step 2^e times larger
                 }
-                q = scale_class(sigma2, floor2, inv_delta2_p);
+                q = __reduce_max_sync(kFull, scale_class(sigma2, floor2, inv_delta2_p));   // same in all lanes
                 skip = ZR && q <= zero_q;
                 float kvv[G];
                 load_half_vec<G>(kvp, kvv);
@@ -547,10 +629,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             if (ZR && skip) { ++n_skipped; continue; }                             // nothing is coded
             int s, qp;
             class_params(q, s, qp);
-            const PosCode pc = pos_code(s);
-            const EncEntry* tbl = tb.enc[qp - kQMin];
-#pragma unroll
-            for (int g = G - 1; g >= 0; --g) wp = encode_step(sym[g], pc, tbl, x, stage, wp, lane, lt, n_escapes);
+            wp = encode_position<G>(sym, s, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
         }
         commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes, n_skipped);
         __syncwarp();
@@ -564,7 +643,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
     build_dec_tables(&tb);
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const uint32_t lt = lanemask_lt();
+    const LaneCode lc = lane_code(lane);
     const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
     int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
     const int Wl = DENSE ? 2 * H : Wt;
@@ -573,7 +652,10 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
                 floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
 
-    for (unsigned item = next_ticket(a.ticket, lane); item < total; item = next_ticket(a.ticket, lane)) {
+    QueueCursor qc = DENSE ? QueueCursor{0, 0} : queue_of_this_sm(a);
+    const unsigned per_table = (unsigned)a.S * (unsigned)a.st.max_chunks;
+    auto next = [&]() { return DENSE ? next_ticket(a.ticket, lane) : next_queued(a, qc, per_table, Wl, lane); };
+    for (unsigned item = next(); item < total; item = next()) {
         const Item it = bulk_item(a, item, DENSE ? a.dense_layer * Wl : 0);
         if (it.P <= 0) continue;
         const unsigned long long off = a.st.chunk_offset[it.slot];
@@ -587,6 +669,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
         bool bad = x < kRansL;
         const uint16_t* words = reinterpret_cast<const uint16_t*>(src + 128);
         const int nwords = (int)((nbytes - 128u) >> 1);
+        const int last = nwords - 1;                 // -1 for a chunk of states only: words[-1] is inside the chunk
         int rp = 0;
         const char* col = reinterpret_cast<const char*>(a.T + (size_t)it.t * a.sh.V * D + 8 * (lane % Geo<D>::R));
         const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
@@ -619,7 +702,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
                 inv_delta2_p = ldexpf(inv_delta2, -2 * e);
                 if (ZR) zero_q -= 8 * e;
             }
-            const int q = scale_class(sigma2, floor2, inv_delta2_p);
+            const int q = __reduce_max_sync(kFull, scale_class(sigma2, floor2, inv_delta2_p));   // same in all lanes
             __syncwarp();                                                         // readers of this slot are done
             int sym[G];
             float out[G];
@@ -629,14 +712,9 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
             } else {
                 int s, qp;
                 class_params(q, s, qp);
-                const PosCode pc = pos_code(s);
-                const uint16_t* cum = tb.cum[qp - kQMin];
-                const uint32_t* fcs = tb.fc[qp - kQMin];
+                decode_position<G>(sym, s, tb.cum[qp - kQMin], tb.fc[qp - kQMin], x, words, rp, last, lc);
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    sym[g] = decode_step(pc, cum, fcs, x, words, rp, nwords, lane, lt, bad);
-                    out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
-                }
+                for (int g = 0; g < G; ++g) out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
             }
             store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
             kvo += a.kv.sp;
@@ -717,6 +795,19 @@ int sm_count() {
 
 int codec_grid_warps(int) { return sm_count() * kBlocksPerSM * kWarpsPerBlock; }
 
+// Queue layout of a gather launch: as many SMs share a queue as it takes for their resident warps
+// to hold one table's chunks, so that a table is worked on by as few SMs as possible (L1 reuse of
+// shared candidate rows) while the tables in flight stay few when a table has many chunks (L2).
+static void set_queues(CodecArgs& a, int n_tables) {
+    const int sms = sm_count(), warps_per_sm = kBlocksPerSM * kWarpsPerBlock;
+    const long long per_table = (long long)a.S * a.st.max_chunks;
+    long long g = (per_table + warps_per_sm - 1) / warps_per_sm;
+    g = std::max(1LL, std::min<long long>(g, sms));
+    int nq = (sms + (int)g - 1) / (int)g;
+    nq = std::max(1, std::min(nq, std::min(n_tables, kTicketWords)));
+    a.sched_g = (int)g; a.sched_nq = nq;
+}
+
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st) {
     return dispatch_d(d, [&](auto D) {
         long long blocks = (rows + 7) / 8;
@@ -727,8 +818,10 @@ cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, c
     });
 }
 
-cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
+cudaError_t launch_encode(const CodecArgs& a0, cudaStream_t st) {
+    CodecArgs a = a0;
+    set_queues(a, 2 * a.sh.L * a.sh.H);
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int) * kTicketWords, st);
     if (e != cudaSuccess) return e;
     const bool zr = a.sh.zero_q != kZeroOff;
     return dispatch_d(a.sh.d, [&](auto D) {
@@ -762,8 +855,10 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
     });
 }
 
-cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
+cudaError_t launch_decode(const CodecArgs& a0, cudaStream_t st) {
+    CodecArgs a = a0;
+    set_queues(a, 2 * a.sh.L * a.sh.H);
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int) * kTicketWords, st);
     if (e != cudaSuccess) return e;
     const bool zr = a.sh.zero_q != kZeroOff;
     return dispatch_d(a.sh.d, [&](auto D) {

@@ -192,7 +192,8 @@ struct CodecArgs {
     int S, n; const int32_t* pos_begin; const int32_t* pos_end;
     StreamsDev st; DebugDev dbg;
     uint16_t* staging; unsigned long long staging_words_per_warp;   // encoder scratch
-    unsigned int* ticket;                          // work counter (zeroed by the launcher)
+    unsigned int* ticket;                          // kTicketWords work counters (zeroed by the launcher)
+    int sched_nq, sched_g;                         // gather kernels: work queues, SMs that share one (set by the launcher)
     unsigned int* status; Counters* counters;
     // dense variant: prediction read from buffers; one launch covers the 2*H tables of dense_layer
     const float* mu_dense; const float* s1_dense; long long mu_ld, s1_ld; int dense_layer;
@@ -201,6 +202,7 @@ struct CodecArgs {
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
 };
 int codec_grid_warps(int device);
+constexpr int kTicketWords = 1024;               // one counter per work queue (at most one queue per SM)
 
 // Dense (full-vocabulary) prediction, one layer at a time.
 struct DenseShape {

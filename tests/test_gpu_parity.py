@@ -219,6 +219,38 @@ def test_step_and_perplexity_sweep(dev, orc, delta, pp):
     gpu_decode_check(g, kv, delta, 96)
 
 
+@pytest.mark.parametrize("delta,most_planes", [(4.0, 0), (0.1, 2), (0.03, 3), (0.003, 7), (0.0007, 8), (1.0 / 4096, 10)])
+def test_every_plane_count_codes_bit_exactly(dev, orc, delta, most_planes):
+    """The number of raw bit planes per position follows sigma/delta; steps from 4 down to 2^-12 move
+    it from 0 to 11 (the kernels have code of their own for the small counts and a loop for the
+    rest).  With a very fine step the binary32 prediction error is no longer small against the step,
+    so the symbols are not compared with the oracle's here; the coder is: the oracle coder fed with
+    the GPU's symbols and classes must give the GPU's bytes, and the GPU decoder must invert them."""
+    tokens, logits, T, kv = make_workload(int(1000 * delta) + 77, 2, 75, 1, 2, 128, 700, 40, pp=9.0)
+    CP, d = 32, 128
+    g = gpu_encode(dev, T, kv, logits, 40, delta, CP)
+    assert g["rc"] == plc.OK
+    sym_g, q_g = g["sym"].cpu().numpy(), g["q"].cpu().numpy()
+    planes = np.where(q_g < 16, 0, (q_g >> 3) - 1)
+    assert planes.max() >= most_planes                       # the case reaches the plane counts it is meant for
+    off = g["st"].chunk_offset.cpu().numpy(); nby = g["st"].chunk_bytes.cpu().numpy().astype(np.int64)
+    payload = g["st"].payload.cpu().numpy()
+    S, n, W, mc = 2, 75, g["W"], g["mc"]
+    for s_ in range(S):
+        for t_ in range(W):
+            for c in range(mc):
+                slot = (s_ * W + t_) * mc + c
+                p0, P = c * CP, min(CP, n - c * CP)
+                ref, _, _ = orc.rans_encode_chunk(sym_g[s_, p0:p0 + P, t_], q_g[s_, p0:p0 + P, t_])
+                assert np.array_equal(payload[off[slot]:off[slot] + nby[slot]], ref), (s_, t_, c)
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    sym2 = torch.zeros_like(g["sym"])
+    g["ctx"].decode(g["st"], g["logits"], out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None))
+    assert g["ctx"].sync_status() == plc.OK
+    assert torch.equal(sym2, g["sym"])
+    assert float((out.cpu() - kv.float()).abs().max()) <= delta / 2 + 1e-3
+
+
 def test_sigma_floor_and_escapes(dev, orc):
     """A point-mass prediction with noisy KV: tiny scale, large residuals -> escapes must round-trip."""
     tokens, logits, T, kv = make_workload(9, 1, 64, 1, 1, 128, 256, 16, sigma=0.3)
