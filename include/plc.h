@@ -188,6 +188,19 @@ plc_status plc_prefix_dedup(plc_ctx* ctx, const int32_t* tokens_dev, const int32
                             int32_t S, int64_t token_stride, int32_t* lcp_dev, float* dT_dev, int32_t* parent_dev,
                             int32_t* shared_len_dev, void* stream);
 
+/* Semantic prefix clusters (Def. 3 of the paper) on the matrices plc_prefix_dedup wrote.  Reading
+ * taken: with d_T = -log2 P(s ^ s') a longer shared prefix gives a larger d_T, and
+ * d_T(a,c) >= min(d_T(a,b), d_T(b,c)); the relation whose maximal subsets are unique is therefore
+ * "the shared prefix carries at least delta bits", d_T(a,b) >= delta (compared in binary32, the
+ * precision of dT_dev), which makes the clusters the cut of the trie at cost delta.  Every session
+ * belongs to its own cluster.  Outputs, each [S] int32: cluster_dev = smallest member index (the
+ * cluster's label), centroid_dev = the member with the largest P(s) = 2^-dT[s][s] (Def. 3's
+ * argmax; ties: smallest index), begin_dev = lcp(s, centroid), the first position of s that the
+ * centroid's cache does not cover (0 for the centroid itself): the pos_begin from which Cor. 3
+ * charges for the tail.  delta >= 0. */
+plc_status plc_prefix_clusters(plc_ctx* ctx, const int32_t* lcp_dev, const float* dT_dev, int32_t S, float delta,
+                               int32_t* cluster_dev, int32_t* centroid_dev, int32_t* begin_dev, void* stream);
+
 /* Trie-based prefix index of Sec. 7.3 (host side; all pointers are HOST memory): stored session
  * prefixes with insert, best-match lookup and evict, each one walk along a root-to-node path.
  * epsilon > 0 prunes the trie at nodes whose probability P(prefix) = prod_j P(x_j | x_<j) (Def. 1)

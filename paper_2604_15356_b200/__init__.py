@@ -23,7 +23,7 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
-           "plc_trie_stats", "plc_create_linear"]
+           "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters"]
 
 
 def sources():
@@ -224,6 +224,15 @@ class Context:
         _check(lib().plc_prefix_dedup(self._h, _ptr(tokens), _ptr(lens), _ptr(logp2), S, C.c_int64(stride), _ptr(lcp),
                                       _ptr(dT), _ptr(parent), _ptr(shared), _stream()), "plc_prefix_dedup")
         return lcp, dT, parent, shared
+
+    def prefix_clusters(self, lcp, dT, delta):
+        """Def. 3 on the outputs of prefix_dedup -> (cluster, centroid, begin), each [S] int32."""
+        import torch
+        S = lcp.shape[0]
+        out = [torch.empty(S, dtype=torch.int32, device=lcp.device) for _ in range(3)]
+        _check(lib().plc_prefix_clusters(self._h, _ptr(lcp), _ptr(dT), S, C.c_float(delta), _ptr(out[0]), _ptr(out[1]),
+                                         _ptr(out[2]), _stream()), "plc_prefix_clusters")
+        return tuple(out)
 
     def encode(self, kv, logits, streams, pos_begin=None, pos_end=None, debug=None, tokens=None):
         S, n = logits.shape[0], logits.shape[1]

@@ -243,6 +243,14 @@ plc_status plc_prefix_dedup(plc_ctx* c, const int32_t* tokens_dev, const int32_t
                                shared_len_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
+plc_status plc_prefix_clusters(plc_ctx* c, const int32_t* lcp_dev, const float* dT_dev, int32_t S, float delta,
+                               int32_t* cluster_dev, int32_t* centroid_dev, int32_t* begin_dev, void* stream) {
+    if (!c || !lcp_dev || !dT_dev || !cluster_dev || !centroid_dev || !begin_dev) return PLC_E_INVALID;
+    if (S < 0 || !(delta >= 0.0f)) return PLC_E_INVALID;
+    return launch_prefix_clusters(lcp_dev, dT_dev, S, delta, cluster_dev, centroid_dev, begin_dev,
+                                  static_cast<cudaStream_t>(stream)) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
 static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n, const int32_t* pb, const int32_t* pe,
                                cudaStream_t st, const int32_t* tokens = nullptr, int32_t* bits_out = nullptr) {
     plc_status rc = ensure_pairs(c, (long long)S * n);

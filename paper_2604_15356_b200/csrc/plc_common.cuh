@@ -161,6 +161,9 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st);
 cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,
                                 int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st);
 
+cudaError_t launch_prefix_clusters(const int32_t* lcp, const float* dT, int S, float delta, int32_t* cluster,
+                                   int32_t* centroid, int32_t* begin, cudaStream_t st);
+
 constexpr int kZeroOff = -1000000;
 
 struct CodecShape {

@@ -47,7 +47,48 @@ __global__ void parent_kernel(const int32_t* __restrict__ lcp, int S, int32_t* _
     shared_len[a] = bl;
 }
 
+// Semantic prefix clusters (Def. 3) from the matrices above: one warp per session a scans its row.
+// Members of a's cluster: a itself and every b whose shared prefix with a carries at least delta
+// bits, d_T(a,b) >= delta (an equivalence, because d_T(a,c) >= min(d_T(a,b), d_T(b,c))).
+// cluster[a] = smallest member, centroid[a] = member with the smallest -log2 P (the diagonal of dT;
+// ties: smallest index), begin[a] = lcp(a, centroid), 0 for the centroid itself.
+__global__ void __launch_bounds__(256) cluster_kernel(const int32_t* __restrict__ lcp, const float* __restrict__ dT, int S,
+                                                      float delta, int32_t* __restrict__ cluster,
+                                                      int32_t* __restrict__ centroid, int32_t* __restrict__ begin) {
+    const int lane = threadIdx.x & 31;
+    const int a = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (a >= S) return;
+    int first = a, best = a;
+    float pbest = dT[(long long)a * S + a];
+    for (int b = lane; b < S; b += 32) {
+        if (b != a && !(dT[(long long)a * S + b] >= delta)) continue;
+        first = min(first, b);
+        const float pb = dT[(long long)b * S + b];
+        if (pb < pbest || (pb == pbest && b < best)) { pbest = pb; best = b; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        first = min(first, __shfl_xor_sync(kFull, first, o));
+        const float po = __shfl_xor_sync(kFull, pbest, o);
+        const int bo = __shfl_xor_sync(kFull, best, o);
+        if (po < pbest || (po == pbest && bo < best)) { pbest = po; best = bo; }
+    }
+    if (lane == 0) {
+        cluster[a] = first;
+        centroid[a] = best;
+        begin[a] = best == a ? 0 : lcp[(long long)a * S + best];
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_prefix_clusters(const int32_t* lcp, const float* dT, int S, float delta, int32_t* cluster,
+                                   int32_t* centroid, int32_t* begin, cudaStream_t st) {
+    if (S <= 0) return cudaSuccess;
+    cluster_kernel<<<(S + 7) / 8, 256, 0, st>>>(lcp, dT, S, delta, cluster, centroid, begin);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,
                                 int32_t* lcp, float* dT, int32_t* parent, int32_t* shared_len, cudaStream_t st) {

@@ -335,14 +335,37 @@ def test_prefix_dedup_parity_and_tail_coding(dev, orc):
     logp2 = out["logp2"].view(S, n)
     lens = torch.tensor([n, n - 3, n, 250, n, n, 17, n, n, n, n, 0], dtype=torch.int32)
     lcp, dT, parent, shared = ctx.prefix_dedup(tkd, lens.to(dev), logp2)
-    lcp_o, dT_o, par_o, sh_o = orc.prefix_dedup(tokens.numpy(), lens.numpy(), logp2.cpu().numpy())
+    # the oracle works from its own log-probabilities, not from the kernel's
+    _, _, _, _, lp_o = orc.topk_softmax(logits.numpy().reshape(-1, V), tokens.numpy().reshape(-1), K)
+    lp_o = lp_o.reshape(S, n)
+    np.testing.assert_allclose(logp2.cpu().numpy(), lp_o, rtol=1e-4, atol=1e-5)
+    lcp_o, dT_o, par_o, sh_o = orc.prefix_dedup(tokens.numpy(), lens.numpy(), lp_o.astype(np.float32))
     assert np.array_equal(lcp.cpu().numpy(), lcp_o)
     np.testing.assert_allclose(dT.cpu().numpy(), dT_o, rtol=1e-4, atol=1e-6)
     assert np.array_equal(parent.cpu().numpy(), par_o) and np.array_equal(shared.cpu().numpy(), sh_o)
     assert sh_o.max() >= 20                                       # the trie really shares prefixes
+    # semantic prefix clusters (Def. 3) at thresholds that sit in gaps of the d_T values, so that the
+    # 1e-4 agreement of d_T cannot move a session across a threshold
+    vals = np.unique(dT_o[~np.eye(S, dtype=bool)])
+    gaps = [(lo + hi) / 2 for lo, hi in zip(vals[:-1], vals[1:]) if hi - lo > 1e-2 * max(hi, 1.0)]
+    deltas = [0.0] + gaps[:: max(1, len(gaps) // 6)] + [float(vals.max()) * 1.5 + 1.0]
+    sizes = set()
+    diag = np.diag(dT_o)
+    for delta in deltas:
+        cl, ce, be = (t.cpu().numpy() for t in ctx.prefix_clusters(lcp, dT, float(np.float32(delta))))
+        cl_o, ce_o, be_o = orc.prefix_clusters(lcp_o, dT_o.astype(np.float32).astype(np.float64), float(np.float32(delta)))
+        assert np.array_equal(cl, cl_o), delta
+        for a in range(S):
+            members = np.nonzero(cl_o == cl_o[a])[0]
+            order = np.sort(diag[members])
+            if len(order) == 1 or order[1] - order[0] > 1e-3 * max(order[0], 1.0):      # a unique most probable member
+                assert ce[a] == ce_o[a] and be[a] == be_o[a], (delta, a)
+            else:                                                                        # any of the tied members is valid
+                assert ce[a] in members and diag[ce[a]] <= order[0] * (1 + 1e-3) + 1e-6
+                assert be[a] == (0 if ce[a] == a else lcp_o[a, ce[a]])
+        sizes.add(len(set(cl_o.tolist())))
+    assert len(sizes) >= 3 and S in sizes                          # from few clusters to all singletons
     # d_T(s,s) = -log2 P(s)  (Remark after Def. 2)
-    _, _, _, _, lp_o = orc.topk_softmax(logits.numpy().reshape(-1, V), tokens.numpy().reshape(-1), K)
-    lp_o = lp_o.reshape(S, n)
     for s in range(S):
         assert abs(float(dT[s, s]) + lp_o[s, :int(lens[s])].sum()) <= 1e-4 * max(1.0, -lp_o[s, :int(lens[s])].sum())
     # tail coding with pos_begin = shared_len straight from the device
