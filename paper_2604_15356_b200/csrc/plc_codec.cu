@@ -795,13 +795,15 @@ int sm_count() {
 
 int codec_grid_warps(int) { return sm_count() * kBlocksPerSM * kWarpsPerBlock; }
 
-// Queue layout of a gather launch: as many SMs share a queue as it takes for their resident warps
-// to hold one table's chunks, so that a table is worked on by as few SMs as possible (L1 reuse of
-// shared candidate rows) while the tables in flight stay few when a table has many chunks (L2).
+// Queue layout of a gather launch: a queue is served by as many SMs as their resident warps can
+// keep busy with ONE table's chunks (rounded down, so that a queue's warps do not spill over into
+// the next table): a table is then worked on by as few SMs as possible (L1 reuse of candidate rows
+// that positions share), and the tables in flight on the whole GPU stay near
+// resident warps / chunks per table (L2).
 static void set_queues(CodecArgs& a, int n_tables) {
     const int sms = sm_count(), warps_per_sm = kBlocksPerSM * kWarpsPerBlock;
     const long long per_table = (long long)a.S * a.st.max_chunks;
-    long long g = (per_table + warps_per_sm - 1) / warps_per_sm;
+    long long g = per_table / warps_per_sm;
     g = std::max(1LL, std::min<long long>(g, sms));
     int nq = (sms + (int)g - 1) / (int)g;
     nq = std::max(1, std::min(nq, std::min(n_tables, kTicketWords)));

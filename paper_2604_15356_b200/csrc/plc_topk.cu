@@ -1,15 +1,21 @@
 // Top-K softmax over per-position next-token logits (one thread block per row, rows strided over
-// the grid).  Selection is exact: a 4096-bin histogram of the order-preserving 16-bit key of each
-// binary16 logit finds the bin that holds the K-th largest, a 16-way refinement finds the key
-// itself, and equal keys are taken in index order.  Reductions use warp shuffles in a fixed order,
-// so results are bit-reproducible from run to run.
+// the grid).  Selection is exact (logit descending, index ascending, -0 = +0).
+//
+// Fast path (K <= 8 per warp of the block ... K <= 256): pass 0 reads the row from HBM and keeps one
+// maximum per thread; the ceil(K / warps)-th largest thread maximum of every warp, minimised over the
+// warps, is a value with at least K row elements at or above it, i.e. a lower bound of the K-th
+// largest logit that needs no histogram.  Pass 1 (served by L2) sums exp(l - l_max) over the row
+// and collects the few elements at or above that bound (typically 1.2-2 K of them); they are ranked
+// by counting, which yields the K selected in their final order.  Rows whose candidates overflow the
+// list (large tie groups, adversarial layouts) and calls with K > 256 take the radix-select path:
+// a 4096-bin histogram of the order-preserving 16-bit key finds the bin that holds the K-th largest,
+// a 16-way refinement finds the key itself, and equal keys are taken in index order.
+// Reductions use warp shuffles in a fixed order, so results are bit-reproducible from run to run.
 #include "plc_common.cuh"
 
 namespace plc {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
 constexpr int kBins = 4096;
 constexpr int kCandCap = 1024;
 
@@ -18,27 +24,34 @@ __device__ __forceinline__ uint32_t key_of(uint32_t u) {
     if ((u & 0x7fffu) == 0) u = 0;                  // -0 and +0 are the same logit
     return (u & 0x8000u) ? (~u & 0xffffu) : (u | 0x8000u);
 }
-__device__ __forceinline__ float val_of_key(uint32_t key) {
-    uint32_t u = (key & 0x8000u) ? (key & 0x7fffu) : (~key & 0xffffu);
-    return __half2float(__ushort_as_half((unsigned short)u));
+__device__ __forceinline__ uint32_t bits_of_key(uint32_t key) {
+    return (key & 0x8000u) ? (key & 0x7fffu) : (~key & 0xffffu);
 }
+__device__ __forceinline__ float val_of_key(uint32_t key) {
+    return __half2float(__ushort_as_half((unsigned short)bits_of_key(key)));
+}
+constexpr uint32_t kKeyNegInf = 0x03ffu;            // key_of(0xfc00)
 
+template <int THREADS>
 struct Smem {
-    uint32_t hist[kBins];
+    uint32_t hist[kBins];                           // fast path: candidate list (keys, then indices)
     uint32_t sub[16];
     uint32_t sel_key[kCandCap];
     int32_t sel_idx[kCandCap];
     uint32_t cand_key[kCandCap];
     int32_t cand_idx[kCandCap];
     float ek[kCandCap];
-    uint32_t red_k[kWarps];
-    float red_s[kWarps];
-    int scan[kWarps];
-    int nsel, ncand, bstar, count_above, cstar, thr, need, neq, running;
+    uint32_t red_k[THREADS / 32];
+    uint32_t red_t[THREADS / 32];
+    float red_s[THREADS / 32];
+    int scan[THREADS / 32];
+    int nsel, ncand, bstar, count_above, cstar, thr, need, neq, running, nlist;
     float row_max, row_sum, sum_k;
+    uint32_t theta;
 };
 
 // Exclusive scan of one int per thread over the block (thread order); total to all threads.
+template <int THREADS>
 __device__ __forceinline__ int block_excl_scan(int v, int* scratch, int& total) {
     int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     int inc = v;
@@ -52,7 +65,7 @@ __device__ __forceinline__ int block_excl_scan(int v, int* scratch, int& total) 
     __syncthreads();
     int base = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < THREADS / 32; ++w) {
         int x = scratch[w];
         if (w < wid) base += x;
         tot += x;
@@ -62,10 +75,10 @@ __device__ __forceinline__ int block_excl_scan(int v, int* scratch, int& total) 
 }
 
 // Calls f(index, raw binary16 bits) for the elements of the row that this thread owns in tile `t`.
-// A tile is kThreads*8 consecutive elements; a thread owns 8 consecutive ones.
-template <bool VEC, class F>
+// A tile is THREADS*8 consecutive elements; a thread owns 8 consecutive ones.
+template <bool VEC, int THREADS, class F>
 __device__ __forceinline__ void for_tile(const __half* row, int V, int t, F&& f) {
-    int i0 = t * (kThreads * 8) + threadIdx.x * 8;
+    int i0 = t * (THREADS * 8) + threadIdx.x * 8;
     if (VEC) {
         if (i0 < V) {                                // V % 8 == 0: the 8 are all in range
             uint4 r = *reinterpret_cast<const uint4*>(row + i0);
@@ -83,12 +96,147 @@ __device__ __forceinline__ void for_tile(const __half* row, int V, int t, F&& f)
     }
 }
 
-template <bool VEC>
-__global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
-    __shared__ Smem sm;
+__device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b) {
+    __half2 r = __hmax2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// Radix select of the K largest keys of the row into sm.sel_* (unordered); three or more passes
+// over the row.
+template <bool VEC, int THREADS>
+__device__ void select_by_histogram(Smem<THREADS>& sm, const __half* row, int V, int K, int ntiles) {
+    const int tid = threadIdx.x;
+    for (int i = tid; i < kBins; i += THREADS) sm.hist[i] = 0;
+    if (tid < 16) sm.sub[tid] = 0;
+    if (tid == 0) { sm.nsel = 0; sm.ncand = 0; sm.running = 0; }
+    __syncthreads();
+    // Pass A: histogram of the top 12 key bits (keys order like the logits).
+    for (int t = 0; t < ntiles; ++t)
+        for_tile<VEC, THREADS>(row, V, t, [&](int, uint32_t bits) { atomicAdd(&sm.hist[key_of(bits) >> 4], 1u); });
+    __syncthreads();
+    // Bin that holds the K-th largest key: thread t owns BPT bins going down from 4095 - BPT*t.
+    {
+        constexpr int BPT = kBins / THREADS;
+        int local = 0;
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) local += (int)sm.hist[kBins - 1 - (tid * BPT + j)];
+        int total;
+        int excl = block_excl_scan<THREADS>(local, sm.scan, total);
+        if (excl < K && K <= excl + local) {
+            int cum = excl;
+            for (int j = 0; j < BPT; ++j) {
+                int b = kBins - 1 - (tid * BPT + j);
+                int c = (int)sm.hist[b];
+                if (cum + c >= K) { sm.bstar = b; sm.count_above = cum; sm.cstar = c; break; }
+                cum += c;
+            }
+        }
+    }
+    __syncthreads();
+    const int bstar = sm.bstar, cstar = sm.cstar, count_above = sm.count_above;
+    const bool use_cand = cstar <= kCandCap;
+    // Pass B: everything above the bin is selected; inside the bin refine on the low 4 key bits.
+    for (int t = 0; t < ntiles; ++t)
+        for_tile<VEC, THREADS>(row, V, t, [&](int i, uint32_t bits) {
+            uint32_t key = key_of(bits);
+            int bin = (int)(key >> 4);
+            if (bin > bstar) {
+                int slot = atomicAdd(&sm.nsel, 1);
+                sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
+            } else if (bin == bstar) {
+                atomicAdd(&sm.sub[key & 15u], 1u);
+                if (use_cand) {
+                    int slot = atomicAdd(&sm.ncand, 1);
+                    sm.cand_key[slot] = key; sm.cand_idx[slot] = i;
+                }
+            }
+        });
+    __syncthreads();
+    if (tid == 0) {
+        int need1 = K - count_above, cum = 0;
+        for (int j = 15; j >= 0; --j) {
+            int c = (int)sm.sub[j];
+            if (cum + c >= need1) { sm.thr = (bstar << 4) | j; sm.need = need1 - cum; sm.neq = c; break; }
+            cum += c;
+        }
+    }
+    __syncthreads();
+    const uint32_t thr = (uint32_t)sm.thr;
+    const int need = sm.need, neq = sm.neq;
+    if (use_cand) {
+        const int nc = sm.ncand;
+        for (int c = tid; c < nc; c += THREADS) {
+            uint32_t key = sm.cand_key[c];
+            int idx = sm.cand_idx[c];
+            bool take = key > thr;
+            if (key == thr) {
+                if (need == neq) take = true;
+                else {
+                    int rank = 0;
+                    for (int j = 0; j < nc; ++j) rank += (sm.cand_key[j] == thr && sm.cand_idx[j] < idx);
+                    take = rank < need;
+                }
+            }
+            if (take) {
+                int slot = atomicAdd(&sm.nsel, 1);
+                sm.sel_key[slot] = key; sm.sel_idx[slot] = idx;
+            }
+        }
+    } else {
+        // Pass C (large tie groups): re-read the row; equal keys are taken in index order.
+        for (int t = 0; t < ntiles; ++t) {
+            int cnt = 0;
+            for_tile<VEC, THREADS>(row, V, t, [&](int i, uint32_t bits) {
+                uint32_t key = key_of(bits);
+                if ((int)(key >> 4) == bstar && key > thr) {
+                    int slot = atomicAdd(&sm.nsel, 1);
+                    sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
+                }
+                cnt += (key == thr);
+            });
+            int total;
+            int rank = block_excl_scan<THREADS>(cnt, sm.scan, total) + sm.running;
+            for_tile<VEC, THREADS>(row, V, t, [&](int i, uint32_t bits) {
+                uint32_t key = key_of(bits);
+                if (key == thr) {
+                    if (rank < need) {
+                        int slot = atomicAdd(&sm.nsel, 1);
+                        sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
+                    }
+                    ++rank;
+                }
+            });
+            __syncthreads();
+            if (tid == 0) sm.running += total;
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    // Order the K selected by (key descending, index ascending): rank by counting.
+    for (int k = tid; k < K; k += THREADS) {
+        uint32_t key = sm.sel_key[k];
+        int idx = sm.sel_idx[k];
+        int rank = 0;
+        for (int j = 0; j < K; ++j) {
+            uint32_t kj = sm.sel_key[j];
+            rank += (kj > key) || (kj == key && sm.sel_idx[j] < idx);
+        }
+        sm.cand_key[rank] = key; sm.cand_idx[rank] = idx;
+    }
+    __syncthreads();
+}
+
+template <bool VEC, int THREADS>
+__global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
+    constexpr int NW = THREADS / 32;
+    __shared__ Smem<THREADS> sm;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int V = a.V, K = a.K;
-    const int ntiles = (V + kThreads * 8 - 1) / (kThreads * 8);
+    const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
+    const bool fast = K <= 32 * NW && K <= kCandCap;     // a warp can offer at most 32 thread maxima
+    const int per_warp = (K + NW - 1) / NW;
+    uint32_t* list_key = sm.hist;                         // the histogram is idle on the fast path
+    int32_t* list_idx = reinterpret_cast<int32_t*>(sm.hist + kCandCap);
 
     for (long long rowi = blockIdx.x; rowi < a.N; rowi += gridDim.x) {
         if (a.pos_begin || a.pos_end) {
@@ -97,153 +245,122 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
             if (i < b || i >= e) continue;
         }
         const __half* row = a.logits + rowi * (long long)V;
-        for (int i = tid; i < kBins; i += kThreads) sm.hist[i] = 0;
-        if (tid < 16) sm.sub[tid] = 0;
-        if (tid == 0) { sm.nsel = 0; sm.ncand = 0; sm.running = 0; }
-        __syncthreads();
+        if (tid == 0) sm.nlist = 0;
 
-        // Pass A: histogram of the top 12 key bits and the largest key (keys order like the logits).
-        uint32_t kmax = 0;
-        for (int t = 0; t < ntiles; ++t)
-            for_tile<VEC>(row, V, t, [&](int, uint32_t bits) {
-                const uint32_t key = key_of(bits);
-                atomicAdd(&sm.hist[key >> 4], 1u);
-                kmax = max(kmax, key);
-            });
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(kFull, kmax, o));
-        if (lane == 0) sm.red_k[wid] = kmax;
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t km = sm.red_k[0];
-            for (int w = 1; w < kWarps; ++w) km = max(km, sm.red_k[w]);
-            sm.row_max = val_of_key(km);
-        }
-
-        // Bin that holds the K-th largest key: thread t owns bins 4095-16t ... 4095-16t-15.
-        {
-            int local = 0;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) local += (int)sm.hist[kBins - 1 - (tid * 16 + j)];
-            int total;
-            int excl = block_excl_scan(local, sm.scan, total);
-            if (excl < K && K <= excl + local) {
-                int cum = excl;
-                for (int j = 0; j < 16; ++j) {
-                    int b = kBins - 1 - (tid * 16 + j);
-                    int c = (int)sm.hist[b];
-                    if (cum + c >= K) { sm.bstar = b; sm.count_above = cum; sm.cstar = c; break; }
-                    cum += c;
+        // Pass 0 (HBM): one maximum per thread.
+        uint32_t tkey = 0;
+        if (VEC) {
+            uint32_t m2 = 0xfc00fc00u;                                   // (-inf, -inf)
+#pragma unroll 4
+            for (int t = 0; t < ntiles; ++t) {
+                const int i0 = t * (THREADS * 8) + tid * 8;
+                if (i0 < V) {
+                    const uint4 r = *reinterpret_cast<const uint4*>(row + i0);
+                    m2 = hmax2_bits(m2, hmax2_bits(hmax2_bits(r.x, r.y), hmax2_bits(r.z, r.w)));
                 }
             }
+            tkey = max(key_of(m2 & 0xffffu), key_of(m2 >> 16));
+            if (tid * 8 >= V) tkey = 0;                                   // this thread owns nothing
+        } else {
+            for (int t = 0; t < ntiles; ++t)
+                for_tile<VEC, THREADS>(row, V, t, [&](int, uint32_t bits) { tkey = max(tkey, key_of(bits)); });
+        }
+        // per warp: the largest and the per_warp-th largest thread maximum
+        const uint32_t wmax = __reduce_max_sync(kFull, tkey);
+        uint32_t wth = 0;
+        if (fast) {
+            uint32_t v = tkey;
+            for (int r = 0; r < per_warp; ++r) {
+                wth = __reduce_max_sync(kFull, v);
+                const uint32_t eq = __ballot_sync(kFull, v == wth);
+                if (lane == __ffs(eq) - 1) v = 0;
+            }
+        }
+        if (lane == 0) { sm.red_k[wid] = wmax; sm.red_t[wid] = wth; }
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t km = sm.red_k[0], th = sm.red_t[0];
+            for (int w = 1; w < NW; ++w) { km = max(km, sm.red_k[w]); th = min(th, sm.red_t[w]); }
+            sm.row_max = val_of_key(km);
+            sm.theta = max(th, kKeyNegInf);
         }
         __syncthreads();
-        const int bstar = sm.bstar, cstar = sm.cstar, count_above = sm.count_above;
-        const bool use_cand = cstar <= kCandCap;
 
-        // Pass B: everything above the bin is selected; inside the bin refine on the low 4 key bits.
-        // The same pass sums exp(l - l_max) over the row (fast exponential: its relative error of
-        // about 2e-6 at the arguments that matter is inside the tolerance of lse and Z_k).
-        const float lmax_b = sm.row_max;
+        // Pass 1 (L2): sum of exp(l - l_max) over the row (fast exponential: its relative error of
+        // about 2e-6 at the arguments that matter is inside the tolerance of lse and Z_k) and, on
+        // the fast path, the elements at or above the bound.
+        const float lmax = sm.row_max;
+        const uint32_t theta = sm.theta;
         float s = 0.f;
-        for (int t = 0; t < ntiles; ++t)
-            for_tile<VEC>(row, V, t, [&](int i, uint32_t bits) {
-                uint32_t key = key_of(bits);
-                s += __expf(__half2float(__ushort_as_half((unsigned short)bits)) - lmax_b);
-                int bin = (int)(key >> 4);
-                if (bin > bstar) {
-                    int slot = atomicAdd(&sm.nsel, 1);
-                    sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
-                } else if (bin == bstar) {
-                    atomicAdd(&sm.sub[key & 15u], 1u);
-                    if (use_cand) {
-                        int slot = atomicAdd(&sm.ncand, 1);
-                        sm.cand_key[slot] = key; sm.cand_idx[slot] = i;
+        if (VEC) {
+            const uint32_t tb = bits_of_key(theta);
+            const uint32_t th2 = tb | (tb << 16);
+#pragma unroll 2
+            for (int t = 0; t < ntiles; ++t) {
+                const int i0 = t * (THREADS * 8) + tid * 8;
+                if (i0 < V) {
+                    const uint4 r = *reinterpret_cast<const uint4*>(row + i0);
+                    const uint32_t wds[4] = {r.x, r.y, r.z, r.w};
+                    const uint32_t top = hmax2_bits(hmax2_bits(r.x, r.y), hmax2_bits(r.z, r.w));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&wds[j]));
+                        s += __expf(f.x - lmax);
+                        s += __expf(f.y - lmax);
+                    }
+                    // collect unless both halves of the pairwise maximum are below the bound
+                    if (fast && !__hblt2(*reinterpret_cast<const __half2*>(&top), *reinterpret_cast<const __half2*>(&th2))) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const uint32_t bits = (wds[j >> 1] >> (16 * (j & 1))) & 0xffffu;
+                            const uint32_t key = key_of(bits);
+                            if (key >= theta) {
+                                const int slot = atomicAdd(&sm.nlist, 1);
+                                if (slot < kCandCap) { list_key[slot] = key; list_idx[slot] = i0 + j; }
+                            }
+                        }
                     }
                 }
-            });
+            }
+        } else {
+            for (int t = 0; t < ntiles; ++t)
+                for_tile<VEC, THREADS>(row, V, t, [&](int i, uint32_t bits) {
+                    s += __expf(__half2float(__ushort_as_half((unsigned short)bits)) - lmax);
+                    const uint32_t key = key_of(bits);
+                    if (fast && key >= theta) {
+                        const int slot = atomicAdd(&sm.nlist, 1);
+                        if (slot < kCandCap) { list_key[slot] = key; list_idx[slot] = i; }
+                    }
+                });
+        }
         s = warp_sum(s);
         if (lane == 0) sm.red_s[wid] = s;
         __syncthreads();
         if (tid == 0) {
             float ss = 0.f;
-            for (int w = 0; w < kWarps; ++w) ss += sm.red_s[w];
+            for (int w = 0; w < NW; ++w) ss += sm.red_s[w];
             sm.row_sum = ss;
-            int need1 = K - count_above, cum = 0;
-            for (int j = 15; j >= 0; --j) {
-                int c = (int)sm.sub[j];
-                if (cum + c >= need1) { sm.thr = (bstar << 4) | j; sm.need = need1 - cum; sm.neq = c; break; }
-                cum += c;
-            }
         }
-        __syncthreads();
-        const uint32_t thr = (uint32_t)sm.thr;
-        const int need = sm.need, neq = sm.neq;
-
-        if (use_cand) {
-            const int nc = sm.ncand;
-            for (int c = tid; c < nc; c += kThreads) {
-                uint32_t key = sm.cand_key[c];
-                int idx = sm.cand_idx[c];
-                bool take = key > thr;
-                if (key == thr) {
-                    if (need == neq) take = true;
-                    else {
-                        int rank = 0;
-                        for (int j = 0; j < nc; ++j) rank += (sm.cand_key[j] == thr && sm.cand_idx[j] < idx);
-                        take = rank < need;
-                    }
+        const int nlist = sm.nlist;
+        if (fast && nlist >= K && nlist <= kCandCap) {
+            // rank the candidates (at least K of them) by counting; the first K ranks are the result
+            for (int c = tid; c < nlist; c += THREADS) {
+                const uint32_t key = list_key[c];
+                const int idx = list_idx[c];
+                int rank = 0;
+                for (int j = 0; j < nlist; ++j) {
+                    const uint32_t kj = list_key[j];
+                    rank += (kj > key) || (kj == key && list_idx[j] < idx);
                 }
-                if (take) {
-                    int slot = atomicAdd(&sm.nsel, 1);
-                    sm.sel_key[slot] = key; sm.sel_idx[slot] = idx;
-                }
+                if (rank < K) { sm.cand_key[rank] = key; sm.cand_idx[rank] = idx; }
             }
+            __syncthreads();
         } else {
-            // Pass C (large tie groups): re-read the row; equal keys are taken in index order.
-            for (int t = 0; t < ntiles; ++t) {
-                int cnt = 0;
-                for_tile<VEC>(row, V, t, [&](int i, uint32_t bits) {
-                    uint32_t key = key_of(bits);
-                    if ((int)(key >> 4) == bstar && key > thr) {
-                        int slot = atomicAdd(&sm.nsel, 1);
-                        sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
-                    }
-                    cnt += (key == thr);
-                });
-                int total;
-                int rank = block_excl_scan(cnt, sm.scan, total) + sm.running;
-                for_tile<VEC>(row, V, t, [&](int i, uint32_t bits) {
-                    uint32_t key = key_of(bits);
-                    if (key == thr) {
-                        if (rank < need) {
-                            int slot = atomicAdd(&sm.nsel, 1);
-                            sm.sel_key[slot] = key; sm.sel_idx[slot] = i;
-                        }
-                        ++rank;
-                    }
-                });
-                __syncthreads();
-                if (tid == 0) sm.running += total;
-                __syncthreads();
-            }
+            __syncthreads();
+            select_by_histogram<VEC, THREADS>(sm, row, V, K, ntiles);
         }
-        __syncthreads();
 
-        // Order the K selected by (key descending, index ascending): rank by counting.
-        for (int k = tid; k < K; k += kThreads) {
-            uint32_t key = sm.sel_key[k];
-            int idx = sm.sel_idx[k];
-            int rank = 0;
-            for (int j = 0; j < K; ++j) {
-                uint32_t kj = sm.sel_key[j];
-                rank += (kj > key) || (kj == key && sm.sel_idx[j] < idx);
-            }
-            sm.cand_key[rank] = key; sm.cand_idx[rank] = idx;
-        }
-        __syncthreads();
-        const float lmax = sm.row_max;
-        for (int k = tid; k < K; k += kThreads) sm.ek[k] = expf(val_of_key(sm.cand_key[k]) - lmax);
+        for (int k = tid; k < K; k += THREADS) sm.ek[k] = expf(val_of_key(sm.cand_key[k]) - lmax);
         __syncthreads();
         if (wid == 0) {
             float p = 0.f;
@@ -253,7 +370,7 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
         }
         __syncthreads();
         const float sum_k = sm.sum_k, sum_all = sm.row_sum;
-        for (int k = tid; k < K; k += kThreads) {
+        for (int k = tid; k < K; k += THREADS) {
             float w = sm.ek[k] / sum_k;
             int idx = sm.cand_idx[k];
             if (a.pairs) a.pairs[rowi * a.Kp + k] = make_int2(idx, __float_as_int(w));
@@ -261,7 +378,7 @@ __global__ void __launch_bounds__(kThreads) topk_softmax_kernel(TopkArgs a) {
             if (a.w) a.w[rowi * K + k] = w;
         }
         if (a.pairs)
-            for (int k = K + tid; k < a.Kp; k += kThreads) a.pairs[rowi * a.Kp + k] = make_int2(sm.cand_idx[0], 0);
+            for (int k = K + tid; k < a.Kp; k += THREADS) a.pairs[rowi * a.Kp + k] = make_int2(sm.cand_idx[0], 0);
         if (tid == 0) {
             float lse = lmax + logf(sum_all);
             if (a.lse) a.lse[rowi] = lse;
@@ -291,10 +408,19 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    long long blocks = a.N < (long long)sms * 4 ? a.N : (long long)sms * 4;
-    bool vec = (a.V % 8 == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
-    if (vec) topk_softmax_kernel<true><<<(unsigned)blocks, kThreads, 0, st>>>(a);
-    else topk_softmax_kernel<false><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+    const bool vec = (a.V % 8 == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
+    // The second pass over a row should find it in L2: rows of up to 128 KB are read by 256 threads
+    // with four blocks per SM, longer rows by 1024 threads with one block per SM.
+    const bool wide = (long long)a.V * 2 > 128 * 1024;
+    const long long per_sm = wide ? 1 : 4;
+    const long long blocks = a.N < sms * per_sm ? a.N : sms * per_sm;
+    if (wide) {
+        if (vec) topk_softmax_kernel<true, 1024><<<(unsigned)blocks, 1024, 0, st>>>(a);
+        else topk_softmax_kernel<false, 1024><<<(unsigned)blocks, 1024, 0, st>>>(a);
+    } else {
+        if (vec) topk_softmax_kernel<true, 256><<<(unsigned)blocks, 256, 0, st>>>(a);
+        else topk_softmax_kernel<false, 256><<<(unsigned)blocks, 256, 0, st>>>(a);
+    }
     count_launch();
     return cudaGetLastError();
 }

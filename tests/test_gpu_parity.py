@@ -161,11 +161,16 @@ def gpu_decode_check(g, kv, delta, n, pos_begin=None, pos_end=None, out_dtype=pl
 
 def test_topk_softmax_parity(dev, orc):
     rng = np.random.default_rng(0)
-    for V, K, N in [(256, 16, 40), (32000, 64, 24), (1000, 64, 16), (37, 5, 9), (4096, 1, 8), (2048, 1024, 4)]:
+    # the last three shapes have rows longer than 128 KB (the kernel's wide blocks), vectorised and not;
+    # K = 300 and K = 1024 are beyond the per-thread-maximum bound and take the radix-select path
+    for V, K, N in [(256, 16, 40), (32000, 64, 24), (1000, 64, 16), (37, 5, 9), (4096, 1, 8), (2048, 1024, 4),
+                    (32000, 256, 6), (8192, 300, 5), (70008, 64, 7), (65541, 40, 6), (128256, 256, 5)]:
         lg = (rng.standard_normal((N, V)) * 2.5).astype(np.float16)
         lg[1, :] = np.float16(0.25)                              # every logit equal
         lg[2, ::2] = lg[2, 0]                                    # half the row tied at one value
         lg[3, :7] = np.float16(-0.0); lg[3, 7:14] = np.float16(0.0)
+        if N > 4:
+            lg[4] = -np.sort(-lg[4])                             # sorted: the largest all sit in the first threads' slices
         tok = rng.integers(0, V, N).astype(np.int32)
         T = torch.zeros(1, 2, 1, V, 32, dtype=torch.float16, device=dev)
         ctx = plc.Context(T, K, 0.02)
