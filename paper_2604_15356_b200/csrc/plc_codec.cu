@@ -795,15 +795,22 @@ int sm_count() {
 
 int codec_grid_warps(int) { return sm_count() * kBlocksPerSM * kWarpsPerBlock; }
 
-// Queue layout of a gather launch: a queue is served by as many SMs as their resident warps can
-// keep busy with ONE table's chunks (rounded down, so that a queue's warps do not spill over into
-// the next table): a table is then worked on by as few SMs as possible (L1 reuse of candidate rows
-// that positions share), and the tables in flight on the whole GPU stay near
-// resident warps / chunks per table (L2).
+// Queue layout of a gather launch.  With one queue for the whole GPU the resident warps span
+// about (resident warps / chunks per table) + 1 consecutive tables; if those tables fit in L2 that
+// is the layout with the smallest working set and it is kept.  Otherwise L2 cannot hold the tables
+// in flight whatever the order, and the only reuse left is between positions that share candidate
+// rows: then a queue is served by as few SMs as keep busy with ONE table's chunks (rounded down),
+// so that the warps of an SM gather from one or two tables and shared rows stay in that SM's L1.
 static void set_queues(CodecArgs& a, int n_tables) {
     const int sms = sm_count(), warps_per_sm = kBlocksPerSM * kWarpsPerBlock;
-    const long long per_table = (long long)a.S * a.st.max_chunks;
+    const long long per_table = std::max(1LL, (long long)a.S * a.st.max_chunks);
+    const long long spanned = ((long long)sms * warps_per_sm + per_table - 1) / per_table + 1;
+    const double table_bytes = 2.0 * a.sh.V * a.sh.d;
+    int dev = 0, l2 = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev);
     long long g = per_table / warps_per_sm;
+    if ((double)std::min<long long>(spanned, n_tables) * table_bytes <= (double)l2) g = sms;
     g = std::max(1LL, std::min<long long>(g, sms));
     int nq = (sms + (int)g - 1) / (int)g;
     nq = std::max(1, std::min(nq, std::min(n_tables, kTicketWords)));
