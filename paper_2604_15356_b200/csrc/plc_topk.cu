@@ -33,7 +33,7 @@ __device__ __forceinline__ float val_of_key(uint32_t key) {
 constexpr uint32_t kKeyNegInf = 0x03ffu;            // key_of(0xfc00)
 
 template <int THREADS>
-struct Smem {
+struct __align__(16) Smem {
     uint32_t hist[kBins];                           // fast path: candidate list (keys, then indices)
     uint32_t sub[16];
     uint32_t sel_key[kCandCap];
@@ -94,6 +94,15 @@ __device__ __forceinline__ void for_tile(const __half* row, int V, int t, F&& f)
         for (int j = 0; j < 8; ++j)
             if (i0 + j < V) f(i0 + j, (uint32_t)__half_as_ushort(row[i0 + j]));
     }
+}
+
+// exp(x - l_max) as 2^(x log2(e) - l_max log2(e)): one fused multiply-add and one ex2.approx (relative
+// error about 2e-6 at the arguments that matter, inside the tolerance of lse and Z_k; results below
+// 2^-126 flush to zero).  nb = -l_max log2(e).
+__device__ __forceinline__ float exp_rel(float x, float nb) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fmaf_rn(x, 1.44269504088896341f, nb)));
+    return r;
 }
 
 __device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b) {
@@ -235,8 +244,15 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
     const bool fast = K <= 32 * NW && K <= kCandCap;     // a warp can offer at most 32 thread maxima
     const int per_warp = (K + NW - 1) / NW;
-    uint32_t* list_key = sm.hist;                         // the histogram is idle on the fast path
-    int32_t* list_idx = reinterpret_cast<int32_t*>(sm.hist + kCandCap);
+    // Candidate list of the fast path (the histogram is idle there): one order word per candidate,
+    // larger = earlier in (key descending, index ascending); 32-bit words while indices fit 16 bits.
+    const bool narrow = V <= 65536;
+    uint32_t* list32 = sm.hist;
+    unsigned long long* list64 = reinterpret_cast<unsigned long long*>(sm.hist);
+    auto list_put = [&](int slot, uint32_t key, int idx) {
+        if (narrow) list32[slot] = (key << 16) | (0xffffu - (uint32_t)idx);
+        else list64[slot] = ((unsigned long long)key << 32) | (0xffffffffu - (uint32_t)idx);
+    };
 
     for (long long rowi = blockIdx.x; rowi < a.N; rowi += gridDim.x) {
         if (a.pos_begin || a.pos_end) {
@@ -278,19 +294,16 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         }
         if (lane == 0) { sm.red_k[wid] = wmax; sm.red_t[wid] = wth; }
         __syncthreads();
-        if (tid == 0) {
-            uint32_t km = sm.red_k[0], th = sm.red_t[0];
-            for (int w = 1; w < NW; ++w) { km = max(km, sm.red_k[w]); th = min(th, sm.red_t[w]); }
-            sm.row_max = val_of_key(km);
-            sm.theta = max(th, kKeyNegInf);
-        }
-        __syncthreads();
+        uint32_t km = sm.red_k[0], theta = sm.red_t[0];
+#pragma unroll
+        for (int w = 1; w < NW; ++w) { km = max(km, sm.red_k[w]); theta = min(theta, sm.red_t[w]); }
+        theta = max(theta, kKeyNegInf);
+        const float lmax = val_of_key(km);
 
         // Pass 1 (L2): sum of exp(l - l_max) over the row (fast exponential: its relative error of
         // about 2e-6 at the arguments that matter is inside the tolerance of lse and Z_k) and, on
         // the fast path, the elements at or above the bound.
-        const float lmax = sm.row_max;
-        const uint32_t theta = sm.theta;
+        const float nb = -lmax * 1.44269504088896341f;
         float s = 0.f;
         if (VEC) {
             const uint32_t tb = bits_of_key(theta);
@@ -305,8 +318,8 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&wds[j]));
-                        s += __expf(f.x - lmax);
-                        s += __expf(f.y - lmax);
+                        s += exp_rel(f.x, nb);
+                        s += exp_rel(f.y, nb);
                     }
                     // collect unless both halves of the pairwise maximum are below the bound
                     if (fast && !__hblt2(*reinterpret_cast<const __half2*>(&top), *reinterpret_cast<const __half2*>(&th2))) {
@@ -316,7 +329,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
                             const uint32_t key = key_of(bits);
                             if (key >= theta) {
                                 const int slot = atomicAdd(&sm.nlist, 1);
-                                if (slot < kCandCap) { list_key[slot] = key; list_idx[slot] = i0 + j; }
+                                if (slot < kCandCap) list_put(slot, key, i0 + j);
                             }
                         }
                     }
@@ -325,34 +338,43 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         } else {
             for (int t = 0; t < ntiles; ++t)
                 for_tile<VEC, THREADS>(row, V, t, [&](int i, uint32_t bits) {
-                    s += __expf(__half2float(__ushort_as_half((unsigned short)bits)) - lmax);
+                    s += exp_rel(__half2float(__ushort_as_half((unsigned short)bits)), nb);
                     const uint32_t key = key_of(bits);
                     if (fast && key >= theta) {
                         const int slot = atomicAdd(&sm.nlist, 1);
-                        if (slot < kCandCap) { list_key[slot] = key; list_idx[slot] = i; }
+                        if (slot < kCandCap) list_put(slot, key, i);
                     }
                 });
         }
         s = warp_sum(s);
         if (lane == 0) sm.red_s[wid] = s;
         __syncthreads();
-        if (tid == 0) {
-            float ss = 0.f;
-            for (int w = 0; w < NW; ++w) ss += sm.red_s[w];
-            sm.row_sum = ss;
-        }
+        float sum_all = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) sum_all += sm.red_s[w];
         const int nlist = sm.nlist;
         if (fast && nlist >= K && nlist <= kCandCap) {
             // rank the candidates (at least K of them) by counting; the first K ranks are the result
-            for (int c = tid; c < nlist; c += THREADS) {
-                const uint32_t key = list_key[c];
-                const int idx = list_idx[c];
-                int rank = 0;
-                for (int j = 0; j < nlist; ++j) {
-                    const uint32_t kj = list_key[j];
-                    rank += (kj > key) || (kj == key && list_idx[j] < idx);
+            if (narrow) {
+                const int n4 = (nlist + 3) & ~3;
+                for (int c = nlist + tid; c < n4; c += THREADS) list32[c] = 0;       // pad: orders after everything
+                __syncthreads();
+                for (int c = tid; c < nlist; c += THREADS) {
+                    const uint32_t mine = list32[c];
+                    int rank = 0;
+                    for (int j = 0; j < n4; j += 4) {
+                        const uint4 o = *reinterpret_cast<const uint4*>(list32 + j);
+                        rank += (o.x > mine) + (o.y > mine) + (o.z > mine) + (o.w > mine);
+                    }
+                    if (rank < K) { sm.cand_key[rank] = mine >> 16; sm.cand_idx[rank] = (int)(0xffffu - (mine & 0xffffu)); }
                 }
-                if (rank < K) { sm.cand_key[rank] = key; sm.cand_idx[rank] = idx; }
+            } else {
+                for (int c = tid; c < nlist; c += THREADS) {
+                    const unsigned long long mine = list64[c];
+                    int rank = 0;
+                    for (int j = 0; j < nlist; ++j) rank += list64[j] > mine;
+                    if (rank < K) { sm.cand_key[rank] = (uint32_t)(mine >> 32); sm.cand_idx[rank] = (int)(0xffffffffu - (uint32_t)mine); }
+                }
             }
             __syncthreads();
         } else {
@@ -369,7 +391,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
             if (lane == 0) sm.sum_k = p;
         }
         __syncthreads();
-        const float sum_k = sm.sum_k, sum_all = sm.row_sum;
+        const float sum_k = sm.sum_k;
         for (int k = tid; k < K; k += THREADS) {
             float w = sm.ek[k] / sum_k;
             int idx = sm.cand_idx[k];
@@ -410,9 +432,9 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const bool vec = (a.V % 8 == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
     // The second pass over a row should find it in L2: rows of up to 128 KB are read by 256 threads
-    // with four blocks per SM, longer rows by 1024 threads with one block per SM.
+    // with five blocks per SM, longer rows by 1024 threads with one block per SM.
     const bool wide = (long long)a.V * 2 > 128 * 1024;
-    const long long per_sm = wide ? 1 : 4;
+    const long long per_sm = wide ? 1 : 5;
     const long long blocks = a.N < sms * per_sm ? a.N : sms * per_sm;
     if (wide) {
         if (vec) topk_softmax_kernel<true, 1024><<<(unsigned)blocks, 1024, 0, st>>>(a);
