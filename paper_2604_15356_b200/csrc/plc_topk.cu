@@ -235,6 +235,28 @@ __device__ void select_by_histogram(Smem<THREADS>& sm, const __half* row, int V,
     __syncthreads();
 }
 
+// Candidate list of the fast path: one order word per candidate, larger = earlier in (key
+// descending, index ascending); 32-bit words while indices fit 16 bits, 64-bit words otherwise.
+__device__ __forceinline__ void list_put(uint32_t* list, bool narrow, int slot, uint32_t key, int idx) {
+    if (narrow) list[slot] = (key << 16) | (0xffffu - (uint32_t)idx);
+    else reinterpret_cast<unsigned long long*>(list)[slot] = ((unsigned long long)key << 32) | (0xffffffffu - (uint32_t)idx);
+}
+// Appends those of the two logits in `w` (indices i, i + 1) that reach the bound th2 (the bound in
+// both halves).  A warp gets here whenever any of its 256 logits of the moment qualifies, with one
+// or two lanes active, so the test is a packed compare and the key is formed for the hits only.
+__device__ __forceinline__ void collect2(uint32_t w, uint32_t th2, int i, bool narrow, int* nlist, uint32_t* list) {
+    const uint32_t ge = __hge2_mask(*reinterpret_cast<const __half2*>(&w), *reinterpret_cast<const __half2*>(&th2));
+    if (ge == 0) return;
+    if (ge & 0xffffu) {
+        const int slot = atomicAdd(nlist, 1);
+        if (slot < kCandCap) list_put(list, narrow, slot, key_of(w & 0xffffu), i);
+    }
+    if (ge >> 16) {
+        const int slot = atomicAdd(nlist, 1);
+        if (slot < kCandCap) list_put(list, narrow, slot, key_of(w >> 16), i + 1);
+    }
+}
+
 template <bool VEC, int THREADS>
 __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     constexpr int NW = THREADS / 32;
@@ -244,15 +266,10 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
     const bool fast = K <= 32 * NW && K <= kCandCap;     // a warp can offer at most 32 thread maxima
     const int per_warp = (K + NW - 1) / NW;
-    // Candidate list of the fast path (the histogram is idle there): one order word per candidate,
-    // larger = earlier in (key descending, index ascending); 32-bit words while indices fit 16 bits.
+    // The candidate list of the fast path lives in the histogram's memory, which is idle there.
     const bool narrow = V <= 65536;
     uint32_t* list32 = sm.hist;
     unsigned long long* list64 = reinterpret_cast<unsigned long long*>(sm.hist);
-    auto list_put = [&](int slot, uint32_t key, int idx) {
-        if (narrow) list32[slot] = (key << 16) | (0xffffu - (uint32_t)idx);
-        else list64[slot] = ((unsigned long long)key << 32) | (0xffffffffu - (uint32_t)idx);
-    };
 
     for (long long rowi = blockIdx.x; rowi < a.N; rowi += gridDim.x) {
         if (a.pos_begin || a.pos_end) {
@@ -324,14 +341,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
                     // collect unless both halves of the pairwise maximum are below the bound
                     if (fast && !__hblt2(*reinterpret_cast<const __half2*>(&top), *reinterpret_cast<const __half2*>(&th2))) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const uint32_t bits = (wds[j >> 1] >> (16 * (j & 1))) & 0xffffu;
-                            const uint32_t key = key_of(bits);
-                            if (key >= theta) {
-                                const int slot = atomicAdd(&sm.nlist, 1);
-                                if (slot < kCandCap) list_put(slot, key, i0 + j);
-                            }
-                        }
+                        for (int j = 0; j < 4; ++j) collect2(wds[j], th2, i0 + 2 * j, narrow, &sm.nlist, sm.hist);
                     }
                 }
             }
@@ -342,7 +352,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
                     const uint32_t key = key_of(bits);
                     if (fast && key >= theta) {
                         const int slot = atomicAdd(&sm.nlist, 1);
-                        if (slot < kCandCap) list_put(slot, key, i);
+                        if (slot < kCandCap) list_put(sm.hist, narrow, slot, key, i);
                     }
                 });
         }
