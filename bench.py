@@ -102,9 +102,10 @@ def oracle_sample_rate(w, positions, layers):
     Tn = w["T"][:layers].cpu().numpy()
     kvn = w["kv"][:layers, :, :1, :, :positions].cpu().numpy()
     lgn = w["logits"][:1, :positions].cpu().numpy()
+    tkn = w["tokens"][:1, :positions].cpu().numpy()
     ocfg = oracle.Config(layers, H, d, V, K, cfg["delta"], 0.0, cfg["chunk_pos"], 0)
     t0 = time.perf_counter()
-    enc = oracle.encode(ocfg, Tn, kvn, lgn, None)
+    enc = oracle.encode(ocfg, Tn, kvn, lgn, tkn)
     t1 = time.perf_counter()
     rc, out, _ = oracle.decode(ocfg, Tn, lgn, enc, kvn.shape)
     t2 = time.perf_counter()
@@ -112,7 +113,10 @@ def oracle_sample_rate(w, positions, layers):
     W_full = 2 * cfg["L"] * H
     vecs = positions * 2 * layers * H
     return dict(value=vecs / W_full / (t2 - t0), encode=vecs / W_full / (t1 - t0), decode=vecs / W_full / (t2 - t1),
-                seconds=t2 - t0, bytes=int(enc["stats"].payload_bytes), vectors=vecs)
+                seconds=t2 - t0, bytes=int(enc["stats"].payload_bytes), vectors=vecs,
+                bits_per_component=8.0 * enc["stats"].payload_bytes / (vecs * d),
+                ideal_bits_per_component=enc["stats"].ideal_bits / (vecs * d),        # sum of -log2(f/M) + raw bits
+                token_bits_per_position=enc["stats"].token_bits / positions)          # sum of -log2 P(x_i | x_<i)
 
 
 def main():
@@ -321,7 +325,10 @@ def main():
         cpu = {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"session 0, first {pos} positions, {layers} of {L} layers, all heads ({r['vectors']} vectors, "
                          f"{r['seconds']:.1f} s encode+decode); rate scaled by W={W} vectors per KV token",
-               "encode": r["encode"], "decode": r["decode"]}
+               "encode": r["encode"], "decode": r["decode"],
+               "sample_bits_per_component": r["bits_per_component"],
+               "sample_ideal_bits_per_component": r["ideal_bits_per_component"],
+               "sample_token_bits_per_position": r["token_bits_per_position"]}
 
     if rank == 0:
         line = {

@@ -262,14 +262,17 @@ __device__ __forceinline__ int encode_step(int sym, int s_dyn, const EncEntry* t
 
 // All G components of one position, last component first, dispatched on the number of planes.
 template <int G>
-__device__ __forceinline__ int encode_position(const int (&sym)[G], int s, const EncEntry* tbl, uint32_t& x,
+__device__ __forceinline__ int encode_position(const int (&sym)[G], int s, bool mixed, const EncEntry* tbl, uint32_t& x,
                                                uint16_t* __restrict__ stage, int wp, const LaneCode& lc, unsigned& n_escapes) {
 #define PLC_ENC_CASE(S_, LABEL)                                                                            \
     LABEL:                                                                                                 \
         _Pragma("unroll") for (int g = G - 1; g >= 0; --g)                                                 \
             wp = encode_step<S_>(sym[g], s, tbl, x, stage, wp, lc, n_escapes);                             \
         break;
-    switch (s) {       // the plane counts that occur in practice get code of their own
+    // The plane counts that occur in practice get code of their own.  With a per-position step
+    // (`mixed`) neighbouring positions differ in plane count, and jumping between a dozen
+    // specialised bodies costs more in instruction fetch than they save: those take the loop.
+    switch (mixed ? -1 : s) {
         PLC_ENC_CASE(0, case 0) PLC_ENC_CASE(1, case 1) PLC_ENC_CASE(2, case 2) PLC_ENC_CASE(3, case 3)
         PLC_ENC_CASE(4, case 4) PLC_ENC_CASE(5, case 5) PLC_ENC_CASE(6, case 6) PLC_ENC_CASE(7, case 7)
         PLC_ENC_CASE(-1, default)
@@ -324,14 +327,14 @@ __device__ __forceinline__ int decode_step(int s_dyn, const uint16_t* cum, const
 }
 
 template <int G>
-__device__ __forceinline__ void decode_position(int (&sym)[G], int s, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
+__device__ __forceinline__ void decode_position(int (&sym)[G], int s, bool mixed, const uint16_t* cum, const uint32_t* fcs, uint32_t& x,
                                                 const uint16_t* __restrict__ words, int& rp, int last, const LaneCode& lc) {
 #define PLC_DEC_CASE(S_, LABEL)                                                                            \
     LABEL:                                                                                                 \
         _Pragma("unroll") for (int g = 0; g < G; ++g)                                                      \
             sym[g] = decode_step<S_>(s, cum, fcs, x, words, rp, last, lc);                                 \
         break;
-    switch (s) {
+    switch (mixed ? -1 : s) {
         PLC_DEC_CASE(0, case 0) PLC_DEC_CASE(1, case 1) PLC_DEC_CASE(2, case 2) PLC_DEC_CASE(3, case 3)
         PLC_DEC_CASE(4, case 4) PLC_DEC_CASE(5, case 5) PLC_DEC_CASE(6, case 6) PLC_DEC_CASE(7, case 7)
         PLC_DEC_CASE(-1, default)
@@ -629,7 +632,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             if (ZR && skip) { ++n_skipped; continue; }                             // nothing is coded
             int s, qp;
             class_params(q, s, qp);
-            wp = encode_position<G>(sym, s, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
+            wp = encode_position<G>(sym, s, a.step_exp != nullptr, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
         }
         commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes, n_skipped);
         __syncwarp();
@@ -712,7 +715,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
             } else {
                 int s, qp;
                 class_params(q, s, qp);
-                decode_position<G>(sym, s, tb.cum[qp - kQMin], tb.fc[qp - kQMin], x, words, rp, last, lc);
+                decode_position<G>(sym, s, a.step_exp != nullptr, tb.cum[qp - kQMin], tb.fc[qp - kQMin], x, words, rp, last, lc);
 #pragma unroll
                 for (int g = 0; g < G; ++g) out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
             }
