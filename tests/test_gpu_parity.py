@@ -205,6 +205,18 @@ def test_multi_stream_ragged_parity(dev, orc, d, K, V, n, CP):
     gpu_decode_check(g, kv, 0.02, n)
 
 
+def test_tables_beyond_l2_take_the_per_sm_queues(dev, orc):
+    """Four candidate tables of 64 MB each: the tables one global work queue would span no longer fit
+    in L2, so the fused kernels deal the tables to per-SM queues (and steal at the tail: two chunks
+    per table against 148 SMs).  Also the widest top-K case: rows of 512 KB, indices beyond 16 bits."""
+    V, K, n, CP = 262144, 24, 50, 32
+    tokens, logits, T, kv = make_workload(4242, 1, n, 1, 2, 128, V, K, pp=20.0, max_states=16)
+    g = gpu_encode(dev, T, kv, logits, K, 0.02, CP)
+    assert g["rc"] == plc.OK
+    check_against_oracle(orc, g, T, kv, logits, K, 0.02, CP)
+    gpu_decode_check(g, kv, 0.02, n)
+
+
 def test_position_ranges_and_empty_sessions(dev, orc):
     tokens, logits, T, kv = make_workload(7, 3, 100, 1, 2, 128, 512, 32)
     pb, pe = [0, 37, 100], [100, 91, 100]
