@@ -262,6 +262,68 @@ def prefix_clusters(lcp, dT, delta):
     return cl, ce, be
 
 
+def rotq_rotate(r, neg):
+    """Sign flips and orthonormal Hadamard transform of one vector (Prop. 3 step 3, rotated quantiser)."""
+    r = np.ascontiguousarray(r, dtype=np.float64)
+    neg = np.ascontiguousarray(neg, dtype=np.uint8)
+    y = np.zeros_like(r)
+    lib().plo_rotq_rotate(_p(r), _p(neg), len(r), _p(y))
+    return y
+
+
+def rotq_unrotate(y, neg):
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    neg = np.ascontiguousarray(neg, dtype=np.uint8)
+    r = np.zeros_like(y)
+    lib().plo_rotq_unrotate(_p(y), _p(neg), len(y), _p(r))
+    return r
+
+
+def rotq_quantise(kv_vec, mu, neg, bits):
+    """kv_vec [d] float16, mu [d] f64 -> (scale float32, codes [d] int32)."""
+    kvv = _h(kv_vec)
+    mu = np.ascontiguousarray(mu, dtype=np.float64)
+    neg = np.ascontiguousarray(neg, dtype=np.uint8)
+    d = len(mu)
+    code = np.zeros(d, np.int32)
+    sc = C.c_float()
+    rc = lib().plo_rotq_quantise(_p(kvv), _p(mu), _p(neg), d, int(bits), C.byref(sc), _p(code))
+    if rc:
+        raise ValueError("rotq_quantise: bad arguments")
+    return np.float32(sc.value), code
+
+
+def rotq_reconstruct(mu, neg, bits, scale, code):
+    mu = np.ascontiguousarray(mu, dtype=np.float64)
+    neg = np.ascontiguousarray(neg, dtype=np.uint8)
+    code = np.ascontiguousarray(code, dtype=np.int32)
+    out = np.zeros(len(mu), np.float32)
+    rc = lib().plo_rotq_reconstruct(_p(mu), _p(neg), len(mu), int(bits), C.c_float(float(scale)), _p(code), _p(out))
+    if rc:
+        raise ValueError("rotq_reconstruct: bad arguments")
+    return out
+
+
+def rotq_pack(code, scale, bits):
+    code = np.ascontiguousarray(code, dtype=np.int32)
+    d = len(code)
+    rec = np.zeros(4 + d * bits // 8, np.uint8)
+    rc = lib().plo_rotq_pack(_p(code), C.c_float(float(scale)), d, int(bits), _p(rec))
+    if rc:
+        raise ValueError("rotq_pack: bad arguments")
+    return rec
+
+
+def rotq_unpack(rec, d, bits):
+    rec = np.ascontiguousarray(rec, dtype=np.uint8)
+    code = np.zeros(d, np.int32)
+    sc = C.c_float()
+    rc = lib().plo_rotq_unpack(_p(rec), d, int(bits), C.byref(sc), _p(code))
+    if rc:
+        raise ValueError("rotq_unpack: bad arguments")
+    return np.float32(sc.value), code
+
+
 def _strides(kv):
     """kv laid out [L,2,S,H,n,d] (any permutation of a contiguous array works): element strides."""
     es = kv.itemsize

@@ -7,7 +7,9 @@
  * leg may call it.  Nothing here is tuned for speed.
  *
  * Pinned parts (see tests/test_oracle_*.py): top-K softmax, mixture, mixture variance, scale class,
- * quantise / reconstruct, frequency tables, rANS chunk coder, LCP / trie metric, dedup parents.
+ * quantise / reconstruct, frequency tables, rANS chunk coder, LCP / trie metric, dedup parents,
+ * prefix clusters, adaptive step, zero-rate rule, linear-embedding predictor, rotated fixed-rate
+ * quantiser.
  * Parity unpinned: the end-to-end bit rate against the paper's 3.3-4.3 bits per token position
  * (Cor. 1) -- the paper states no achieved rate for any coder; the rate is only reported.
  *
@@ -22,6 +24,7 @@
  *   longest common prefix, d_T = -log2 P(s ^ s') ...... Def. 2 (trie metric)
  *   prefix costs zero bits, tail is delta coded ....... Prop. 2, proof, "Description of KV(s)"
  *   best-match lookup = deepest stored ancestor ....... Sec. 7.3 (trie-based prefix index)
+ *   per-vector quantiser on the residual .............. Prop. 3, step 3 (rotated fixed-rate quantiser)
  * The paper names no entropy coder beyond "standard source coding" (Prop. 2, proof); the coder
  * below (uniform step, discretised-Laplace model, 32-lane interleaved rANS) is this build's
  * stated reading and is defined in full in the comments of each function.
@@ -287,6 +290,108 @@ void plo_quantise(const uint16_t* kv, const double* mu, int d, float delta, int3
 /* Prop. 3, "Correctness": KV = R + KV^, with R at its quantised value; one fused binary32 step. */
 void plo_reconstruct(const double* mu, const int32_t* sym, int d, float delta, float* out) {
     for (int j = 0; j < d; ++j) out[j] = fmaf((float)sym[j], delta, (float)mu[j]);
+}
+
+/* ---------------------------------------------------------------- rotated fixed-rate quantiser */
+
+/* Prop. 3, step 3: "any per-vector quantizer" applied to R_i.  Besides the entropy-coded uniform
+ * quantiser above, this build offers the generic member of the family the paper points to (a
+ * random rotation followed by a b-bit scalar quantiser; the paper gives no details of TurboQuant,
+ * so nothing of it is reproduced here).  For one residual vector r of d = 2^m components:
+ *   x_j = eps_j r_j                          eps_j = -1 where neg[j] != 0, else +1   (input to the method)
+ *   y_k = d^(-1/2) sum_j (-1)^popcount(j & k) x_j      (Sylvester-Hadamard matrix, orthonormal, symmetric)
+ *   s   = max_k |y_k|                                   (per-vector scale, stored as binary32)
+ *   c_k = clamp(floor((y_k / s + 1) 2^b / 2), 0, 2^b - 1)          (mid-rise, 2^b levels on [-s, s])
+ * and back:  y^_k = s ((c_k + 1/2) 2 / 2^b - 1),  x^ = H y^ (the same matrix),  r^_j = eps_j x^_j,
+ * so |y^_k - y_k| <= s / 2^b and ||r^ - r||_2 = ||y^ - y||_2 <= sqrt(d) s / 2^b.
+ * The transform is written out from its definition, O(d^2), in double. */
+static int parity(unsigned v) { int p = 0; while (v) { p ^= 1; v &= v - 1; } return p; }
+
+void plo_rotq_rotate(const double* r, const uint8_t* neg, int d, double* y) {
+    const double norm = 1.0 / sqrt((double)d);
+    for (int k = 0; k < d; ++k) {
+        double acc = 0.0;
+        for (int j = 0; j < d; ++j) {
+            double x = neg[j] ? -r[j] : r[j];
+            acc += parity((unsigned)(j & k)) ? -x : x;
+        }
+        y[k] = acc * norm;
+    }
+}
+
+void plo_rotq_unrotate(const double* y, const uint8_t* neg, int d, double* r) {
+    const double norm = 1.0 / sqrt((double)d);
+    for (int j = 0; j < d; ++j) {
+        double acc = 0.0;
+        for (int k = 0; k < d; ++k) acc += parity((unsigned)(j & k)) ? -y[k] : y[k];
+        acc *= norm;
+        r[j] = neg[j] ? -acc : acc;
+    }
+}
+
+/* Residual (Def. 6) of one vector, rotation, scale and codes.  The decisions (scale, codes) are taken
+ * in binary32, the precision of the kernels: y is rounded to float, s = max |y| as a float,
+ * c = floor(fma(y * (1/s), 2^b / 2, 2^b / 2)) with the reciprocal rounded once; s = 0 gives the middle
+ * level everywhere and reconstructs to zero. */
+int plo_rotq_quantise(const uint16_t* kv, const double* mu, const uint8_t* neg, int d, int b, float* scale, int32_t* code) {
+    if (d < 1 || d > 4096 || (d & (d - 1)) || b < 1 || b > 8) return PLO_E_INVALID;
+    double r[4096], y[4096];
+    for (int j = 0; j < d; ++j) r[j] = (double)((float)half_to_double(kv[j]) - (float)mu[j]);
+    plo_rotq_rotate(r, neg, d, y);
+    float s = 0.0f;
+    for (int k = 0; k < d; ++k) { float a = fabsf((float)y[k]); if (a > s) s = a; }
+    const float inv = s > 0.0f ? 1.0f / s : 0.0f, half_levels = (float)(1 << b) * 0.5f;
+    for (int k = 0; k < d; ++k) {
+        float u = fmaf((float)y[k] * inv, half_levels, half_levels);
+        int c = (int)floorf(u);
+        if (c < 0) c = 0;
+        if (c > (1 << b) - 1) c = (1 << b) - 1;
+        code[k] = c;
+    }
+    *scale = s;
+    return PLO_OK;
+}
+
+/* Prop. 3, "Correctness": KV' = KV^ + r^ with r^ rebuilt from the codes. */
+int plo_rotq_reconstruct(const double* mu, const uint8_t* neg, int d, int b, float scale, const int32_t* code, float* out) {
+    if (d < 1 || d > 4096 || (d & (d - 1)) || b < 1 || b > 8) return PLO_E_INVALID;
+    double yq[4096], r[4096];
+    for (int k = 0; k < d; ++k)
+        yq[k] = (double)(scale * fmaf((float)code[k] + 0.5f, 2.0f / (float)(1 << b), -1.0f));
+    plo_rotq_unrotate(yq, neg, d, r);
+    for (int j = 0; j < d; ++j) out[j] = (float)mu[j] + (float)r[j];
+    return PLO_OK;
+}
+
+/* Record of one vector: the scale (binary32, little endian) followed by (d/32) * b words of 32 bits.
+ * Word g*b + p holds bit p of the codes of 32 components, one per lane: lane l's g-th component is
+ * the one the rANS format gives to that lane (comp_index).  4 + d*b/8 bytes. */
+static int comp_index(int l, int g, int d);
+int plo_rotq_pack(const int32_t* code, float scale, int d, int b, uint8_t* rec) {
+    if (!(d == 32 || d == 64 || d == 128 || d == 256) || b < 1 || b > 8) return PLO_E_INVALID;
+    memcpy(rec, &scale, 4);
+    const int G = d / NLANES;
+    for (int g = 0; g < G; ++g)
+        for (int p = 0; p < b; ++p) {
+            uint32_t w = 0;
+            for (int l = 0; l < NLANES; ++l) w |= (uint32_t)((code[comp_index(l, g, d)] >> p) & 1) << l;
+            memcpy(rec + 4 + 4 * (g * b + p), &w, 4);
+        }
+    return PLO_OK;
+}
+
+int plo_rotq_unpack(const uint8_t* rec, int d, int b, float* scale, int32_t* code) {
+    if (!(d == 32 || d == 64 || d == 128 || d == 256) || b < 1 || b > 8) return PLO_E_INVALID;
+    memcpy(scale, rec, 4);
+    const int G = d / NLANES;
+    for (int j = 0; j < d; ++j) code[j] = 0;
+    for (int g = 0; g < G; ++g)
+        for (int p = 0; p < b; ++p) {
+            uint32_t w;
+            memcpy(&w, rec + 4 + 4 * (g * b + p), 4);
+            for (int l = 0; l < NLANES; ++l) code[comp_index(l, g, d)] |= (int32_t)((w >> l) & 1u) << p;
+        }
+    return PLO_OK;
 }
 
 /* ---------------------------------------------------------------- frequency tables */
