@@ -138,6 +138,8 @@ def main():
                     help="prediction: top-K gather (default), full-vocabulary bf16 tensor-core contraction, or the "
                          "linear-embedding model of Sec. 7.1 (two chained contractions; see --d-model)")
     ap.add_argument("--d-model", type=int, default=4096, help="embedding width of --variant linear")
+    ap.add_argument("--rotq", type=int, default=0,
+                    help="bits > 0: rotated fixed-rate quantiser on the residual (Prop. 3 step 3) instead of the entropy coder")
     ap.add_argument("--sigma-floor", type=float, default=0.0,
                     help="standard deviation added in quadrature to the mixture's before the scale class is taken")
     ap.add_argument("--zero-rate", type=float, default=0.0,
@@ -164,6 +166,8 @@ def main():
         return append_arm(args, torch, plc, workloads, dev)
     if args.workload == "dedup":
         return dedup_arm(args, torch, plc, workloads, dev)
+    if args.rotq > 0:
+        return rotq_arm(args, torch, plc, workloads, dev)
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -515,6 +519,64 @@ def dedup_arm(args, torch, plc, workloads, dev):
                          "accounting": "logits read once (2*S*n*V bytes) over the summed log2 P launches; the encode and "
                                        "decode calls scan the logits of the coded positions once more each"},
             "gpu_launches": launches}
+    print(json.dumps(line))
+    return 0
+
+
+def rotq_arm(args, torch, plc, workloads, dev):
+    """Predict, rotate and quantise the residual to `--rotq` bits per component (fixed-size records),
+    then decode; same workloads, same prediction kernels, no entropy coder."""
+    over = {}
+    for kvs in args.set:
+        k, v = kvs.split("=")
+        over[k] = float(v) if "." in v else int(v)
+    w = workloads.build(args.workload, dev, seed=20260415, **over)
+    cfg = w["cfg"]
+    S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
+    W = 2 * L * H
+    ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16)
+    ctx.reserve(S * n)
+    g = torch.Generator().manual_seed(7)
+    params = ctx.rotq_params(args.rotq, torch.randint(0, 2, (d,), generator=g).tolist())
+    rb = ctx.rotq_record_bytes(args.rotq)
+    records = torch.empty(S * W * n * rb, dtype=torch.uint8, device=dev)
+    out = torch.empty_like(w["kv"])
+    for _ in range(max(args.warmup, 1)):
+        ctx.encode_rotq(w["kv"], w["logits"], params, records)
+        ctx.decode_rotq(records, w["logits"], params, out)
+    torch.cuda.synchronize()
+    assert ctx.sync_status() == plc.OK
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+    launches0 = plc.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    ev[0].record()
+    for i in range(args.steps):
+        ctx.encode_rotq(w["kv"], w["logits"], params, records)
+        ev[2 * i + 1].record()
+        ctx.decode_rotq(records, w["logits"], params, out)
+        ev[2 * i + 2].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = plc.launch_count() - launches0
+    enc = statistics.mean(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps))
+    dec = statistics.mean(ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(args.steps))
+    ms = ev[0].elapsed_time(ev[-1]) / args.steps
+    diff = out.float() - w["kv"].float()
+    rms = float(diff.pow(2).mean().sqrt())
+    peak, kind = measured_peaks()
+    vecs = S * n * W
+    bytes_ns = vecs * d * 2 + vecs * K * d * 2 + vecs * rb
+    line = {"metric": METRIC, "value": S * n / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K, "quantiser": "rotated, %d bits" % args.rotq,
+                       "chunk_pos": cfg["chunk_pos"], "l2": "inputs larger than L2"},
+            "encode_ms": enc, "decode_ms": dec, "bits_per_component": 8.0 * rb / d, "bits_per_token": 8.0 * rb * W,
+            "rms_error": rms, "max_error": float(diff.abs().max()),
+            "roofline": {"kernel": "rotq_kernel", "bound": "hbm", "achieved": bytes_ns / (max(enc, dec) / 1e3) / 1e9, "peak": peak,
+                         "unit": "GB/s", "frac": bytes_ns / (max(enc, dec) / 1e3) / 1e9 / peak, "traffic": None, "peak_kind": kind,
+                         "accounting": "KV + gathered T rows (K*d*2 B per vector, served by L1 / L2) + records, per call (top-K included)"},
+            "gpu_launches": launches, "clocks": clocks}
     print(json.dumps(line))
     return 0
 

@@ -253,6 +253,35 @@ plc_status plc_decode_adaptive(plc_ctx* ctx, const plc_streams* in, const void* 
                                int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
                                const plc_kv_view* kv_out, const plc_debug_buffers* dbg, void* stream);
 
+/* Prop. 3 of the paper, step 3, with a rotated fixed-rate quantiser in place of the entropy-coded one
+ * ("any per-vector quantizer" may follow the residual; the paper names TurboQuant and gives no details
+ * of it, so this is the generic member of that family): for every coded (stream, position)
+ *     x = eps * (KV - KV^),   y = H x  (Sylvester-Hadamard matrix of order d, scaled by d^(-1/2)),
+ *     s = max |y|,   c_k = clamp(floor((y_k / s + 1) 2^bits / 2), 0, 2^bits - 1),
+ * and back  y^_k = s ((c_k + 1/2) 2 / 2^bits - 1),  KV' = KV^ + eps * H y^,  so that
+ * ||KV' - KV||_2 <= sqrt(d) s / 2^bits  (Prop. 3, "Correctness": the error on KV is the error on R).
+ * eps_j = -1 where bit j of sign_bits is set, else +1: the caller draws these d random signs once and
+ * passes the same ones to both directions.  KV^ is the top-k prediction of the context (PLC_PRED_TOPK,
+ * adaptive_b0 = 0; PLC_E_STATE otherwise).
+ * Records: fixed size, plc_rotq_record_bytes = 4 + d*bits/8 bytes (1 <= bits <= 8 and at most 256
+ * bytes: PLC_E_SHAPE otherwise); the record of (session s, table t, position i) starts at byte
+ * ((s*W + t)*n + i) * record_bytes of records_dev (4-byte aligned): the scale s as binary32, then for
+ * g < d/32 and p < bits one 32-bit word whose bit l is bit p of the code of component
+ * 8 (l mod d/8) + (d/32) (l div d/8) + g.  Positions outside [pos_begin, pos_end) are not touched.
+ * Errors: PLC_E_CAPACITY if records_capacity < S*W*n*record_bytes (nothing is launched), and as for
+ * plc_encode / plc_decode. */
+typedef struct {
+    int32_t bits;
+    uint32_t sign_bits[8];
+} plc_rotq_params;
+plc_status plc_rotq_record_bytes(const plc_ctx* ctx, int32_t bits, uint64_t* bytes);
+plc_status plc_encode_rotq(plc_ctx* ctx, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
+                           const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_rotq_params* params,
+                           void* records_dev, uint64_t records_capacity, void* stream);
+plc_status plc_decode_rotq(plc_ctx* ctx, const void* records_dev, uint64_t records_capacity, const void* logits_dev,
+                           int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                           const plc_rotq_params* params, const plc_kv_view* kv_out, void* stream);
+
 /* Decode-time append (integration point 1 for one new token per session).  kv_step_dev
  * [L][2][B][H][d] f16, logits_step_dev [B][V] f16.  The new position's symbols and class go to the
  * open chunk; when it holds chunk_pos positions it is coded into sb->streams (a LIFO coder cannot

@@ -23,7 +23,8 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_get_stats", "plc_table_constants", "plc_build_table", "plc_set_profiling", "plc_last_kernel_ms",
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
-           "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters"]
+           "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters", "plc_rotq_record_bytes", "plc_encode_rotq",
+           "plc_decode_rotq"]
 
 
 def sources():
@@ -68,6 +69,10 @@ class DebugBuffers(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("payload_bytes", C.c_uint64), ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64),
                 ("coded_vectors", C.c_uint64), ("skipped_vectors", C.c_uint64)]
+
+
+class RotqParams(C.Structure):
+    _fields_ = [("bits", C.c_int32), ("sign_bits", C.c_uint32 * 8)]
 
 
 class LinearModel(C.Structure):
@@ -224,6 +229,35 @@ class Context:
         _check(lib().plc_prefix_dedup(self._h, _ptr(tokens), _ptr(lens), _ptr(logp2), S, C.c_int64(stride), _ptr(lcp),
                                       _ptr(dT), _ptr(parent), _ptr(shared), _stream()), "plc_prefix_dedup")
         return lcp, dT, parent, shared
+
+    def rotq_params(self, bits, neg):
+        """neg: d booleans (component j negated before the transform)."""
+        p = RotqParams()
+        p.bits = int(bits)
+        for j, v in enumerate(neg):
+            if v:
+                p.sign_bits[j >> 5] |= 1 << (j & 31)
+        return p
+
+    def rotq_record_bytes(self, bits):
+        b = C.c_uint64()
+        _check(lib().plc_rotq_record_bytes(self._h, int(bits), C.byref(b)), "plc_rotq_record_bytes")
+        return b.value
+
+    def encode_rotq(self, kv, logits, params, records, pos_begin=None, pos_end=None):
+        """Rotated fixed-rate quantiser (Prop. 3 step 3): records uint8 [S*W*n*record_bytes] on the device."""
+        S, n = logits.shape[0], logits.shape[1]
+        view = kv if isinstance(kv, KVView) else kv_view(kv)
+        _check(lib().plc_encode_rotq(self._h, C.byref(view), _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end),
+                                     C.byref(params), _ptr(records), C.c_uint64(records.numel() * records.element_size()),
+                                     _stream()), "plc_encode_rotq")
+
+    def decode_rotq(self, records, logits, params, kv_out, pos_begin=None, pos_end=None):
+        S, n = logits.shape[0], logits.shape[1]
+        view = kv_out if isinstance(kv_out, KVView) else kv_view(kv_out)
+        _check(lib().plc_decode_rotq(self._h, _ptr(records), C.c_uint64(records.numel() * records.element_size()),
+                                     _ptr(logits), S, n, _ptr(pos_begin), _ptr(pos_end), C.byref(params), C.byref(view),
+                                     _stream()), "plc_decode_rotq")
 
     def prefix_clusters(self, lcp, dT, delta):
         """Def. 3 on the outputs of prefix_dedup -> (cluster, centroid, begin), each [S] int32."""

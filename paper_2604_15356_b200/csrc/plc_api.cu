@@ -404,6 +404,55 @@ plc_status plc_decode_adaptive(plc_ctx* c, const plc_streams* in, const void* lo
     return decode_impl(c, in, logits_dev, tokens_dev, S, n, pos_begin_dev, pos_end_dev, kv_out, dbg, stream);
 }
 
+static int rotq_words(const plc_ctx* c, int bits) { return 1 + c->cfg.head_dim / 32 * bits; }
+
+plc_status plc_rotq_record_bytes(const plc_ctx* c, int32_t bits, uint64_t* bytes) {
+    if (!c || !bytes) return PLC_E_INVALID;
+    if (bits < 1 || bits > 8 || rotq_words(c, bits) > 64) return PLC_E_SHAPE;
+    *bytes = 4ull * rotq_words(c, bits);
+    return PLC_OK;
+}
+
+static plc_status rotq_impl(plc_ctx* c, const plc_kv_view* kv, int elem_bytes, const void* logits_dev, int32_t S, int32_t n,
+                            const int32_t* pb, const int32_t* pe, const plc_rotq_params* p, const void* records_dev,
+                            uint64_t capacity, bool encode, void* stream) {
+    if (!c || !logits_dev || !p || !records_dev || S < 0 || n < 0) return PLC_E_INVALID;
+    if (c->cfg.variant != PLC_PRED_TOPK || c->cfg.adaptive_b0 > 0) return PLC_E_STATE;
+    if (p->bits < 1 || p->bits > 8 || rotq_words(c, p->bits) > 64) return PLC_E_SHAPE;
+    if (reinterpret_cast<uintptr_t>(records_dev) & 3) return PLC_E_ALIGN;
+    plc_status rc = check_view(kv, c->cfg.head_dim, elem_bytes);
+    if (rc) return rc;
+    const unsigned long long W = 2ull * c->cfg.n_layers * c->cfg.n_kv_heads;
+    if (4ull * rotq_words(c, p->bits) * W * (unsigned long long)S * (unsigned long long)n > capacity) return PLC_E_CAPACITY;
+    if (S == 0 || n == 0) return PLC_OK;
+    const int mc = (n + c->cfg.chunk_pos - 1) / c->cfg.chunk_pos;
+    if ((long long)W * S * mc >= (1ll << 32)) return PLC_E_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = run_topk_for(c, logits_dev, S, n, pb, pe, st);
+    if (rc) return rc;
+    CodecArgs a = base_args(c);
+    a.kv = to_dev(kv); a.S = S; a.n = n; a.pos_begin = pb; a.pos_end = pe; a.pairs = c->pairs;
+    a.st.max_chunks = mc;
+    RotqArgs r{};
+    r.bits = p->bits; r.rec_words = rotq_words(c, p->bits);
+    for (int i = 0; i < 8; ++i) r.sign_bits[i] = p->sign_bits[i];
+    r.records = static_cast<uint32_t*>(const_cast<void*>(records_dev));
+    return launch_rotq(a, r, encode, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_encode_rotq(plc_ctx* c, const plc_kv_view* kv, const void* logits_dev, int32_t S, int32_t n,
+                           const int32_t* pos_begin_dev, const int32_t* pos_end_dev, const plc_rotq_params* p,
+                           void* records_dev, uint64_t records_capacity, void* stream) {
+    return rotq_impl(c, kv, 2, logits_dev, S, n, pos_begin_dev, pos_end_dev, p, records_dev, records_capacity, true, stream);
+}
+
+plc_status plc_decode_rotq(plc_ctx* c, const void* records_dev, uint64_t records_capacity, const void* logits_dev,
+                           int32_t S, int32_t n, const int32_t* pos_begin_dev, const int32_t* pos_end_dev,
+                           const plc_rotq_params* p, const plc_kv_view* kv_out, void* stream) {
+    return rotq_impl(c, kv_out, c && c->cfg.out_dtype == PLC_OUT_F16 ? 2 : 4, logits_dev, S, n, pos_begin_dev, pos_end_dev, p,
+                     records_dev, records_capacity, false, stream);
+}
+
 plc_status plc_append_sizes(const plc_ctx* c, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes) {
     if (!c || B < 0 || !open_sym_bytes || !open_q_bytes) return PLC_E_INVALID;
     const uint64_t W = 2ull * c->cfg.n_layers * c->cfg.n_kv_heads;

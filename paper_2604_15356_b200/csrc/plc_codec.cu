@@ -736,6 +736,124 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
     }
 }
 
+// In-place orthonormal Walsh-Hadamard transform of a d-vector spread over the warp in the coder's
+// ownership (lane l, register g  <->  component 8 (l mod R) + G (l div R) + g): every bit of the
+// component index is either a bit of g (butterflies between registers) or a bit of the lane number
+// (butterflies by shuffle), so log2(G) + 5 = log2(d) stages visit every bit once; the element whose
+// bit is set receives partner - self.  Output index = input index (natural Hadamard order).
+template <int D>
+__device__ __forceinline__ void hadamard(float (&v)[Geo<D>::G], int lane) {
+    constexpr int G = Geo<D>::G;
+#pragma unroll
+    for (int m = 1; m < G; m <<= 1) {
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+            if (!(g & m)) { const float a = v[g], b = v[g | m]; v[g] = a + b; v[g | m] = a - b; }
+    }
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const bool up = (lane & m) != 0;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float p = __shfl_xor_sync(kFull, v[g], m);
+            v[g] = up ? p - v[g] : v[g] + p;
+        }
+    }
+    constexpr float norm = D == 32 ? 0.17677669529663687f : D == 64 ? 0.125f : D == 128 ? 0.08838834764831845f : 0.0625f;   // d^(-1/2)
+#pragma unroll
+    for (int g = 0; g < G; ++g) v[g] *= norm;
+}
+
+// Rotated fixed-rate quantiser (Prop. 3 step 3: a per-vector quantiser on the residual R = KV - KV^):
+// x = eps * R, y = H x (orthonormal Hadamard), s = max |y|, b-bit mid-rise codes on [-s, s]; the
+// record is s followed by one ballot word per (register, code bit).  ENC: KV -> records;
+// otherwise records -> KV' = KV^ + eps * H y^.  One warp per (stream, chunk of positions).
+template <int D, bool ENC>
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM) rotq_kernel(const CodecArgs a, const RotqArgs rq) {
+    constexpr int G = Geo<D>::G;
+    const int lane = threadIdx.x & 31;
+    const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp, B = rq.bits;
+    int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
+    const unsigned total = (unsigned)Wt * a.S * a.st.max_chunks;
+    const float inv_d = 1.0f / D, half_levels = 0.5f * (float)(1 << B), cell = 2.0f / (float)(1 << B);
+    const int c0 = first_comp<D>(lane);
+    float sgn[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) sgn[g] = (rq.sign_bits[(c0 + g) >> 5] >> ((c0 + g) & 31)) & 1u ? -1.0f : 1.0f;
+    QueueCursor qc = queue_of_this_sm(a);
+    const unsigned per_table = (unsigned)a.S * (unsigned)a.st.max_chunks;
+    for (unsigned item = next_queued(a, qc, per_table, Wt, lane); item < total; item = next_queued(a, qc, per_table, Wt, lane)) {
+        const Item it = bulk_item(a, item);
+        if (it.P <= 0) continue;
+        const char* col = reinterpret_cast<const char*>(a.T + (size_t)it.t * a.sh.V * D + 8 * (lane % Geo<D>::R));
+        const float* n2 = a.rownorm2 + (size_t)it.t * a.sh.V;
+        const int2* gp = a.pairs + ((long long)it.s * a.n + it.p0) * Kp;
+        __syncwarp();
+        prefetch_pairs(sp0, gp, Kp, lane);
+        int buf = 0;
+        long long kvo = kv_elem(a.kv, it.t, H, it.s, it.p0) + c0;
+        uint32_t* rec = rq.records + (((long long)it.s * Wt + it.t) * a.n + it.p0) * rq.rec_words;
+        for (int p = 0; p < it.P; ++p, rec += rq.rec_words, kvo += a.kv.sp) {
+            const int2* sp = sp0 + buf * Kp;
+            if (p + 1 < it.P) {
+                gp += Kp;
+                prefetch_pairs(sp0 + (buf ^ 1) * Kp, gp, Kp, lane);
+                pairs_ready<1>();
+            } else {
+                pairs_ready<0>();
+            }
+            buf ^= 1;
+            float mu[G], sigma2;
+            predict<D>(col, n2, sp, Kp, lane, inv_d, mu, sigma2);
+            __syncwarp();                                                         // readers of this slot are done
+            float y[G];
+            if (ENC) {
+                load_half_vec<G>(reinterpret_cast<const __half*>(a.kv.base) + kvo, y);
+#pragma unroll
+                for (int g = 0; g < G; ++g) y[g] = __fsub_rn(y[g], mu[g]) * sgn[g];
+                hadamard<D>(y, lane);
+                float amax = 0.f;
+#pragma unroll
+                for (int g = 0; g < G; ++g) amax = fmaxf(amax, fabsf(y[g]));
+                const float scale = __uint_as_float(__reduce_max_sync(kFull, __float_as_uint(amax)));   // non-negative floats order like their bits
+                const float inv = scale > 0.f ? __fdiv_rn(1.0f, scale) : 0.f;
+                uint32_t mine0 = __float_as_uint(scale), mine1 = 0u;               // word 0 of the record is the scale
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    int c = (int)floorf(__fmaf_rn(__fmul_rn(y[g], inv), half_levels, half_levels));
+                    c = min(max(c, 0), (1 << B) - 1);
+                    for (int b = 0; b < B; ++b) {
+                        const uint32_t plane = __ballot_sync(kFull, (c >> b) & 1);
+                        const int w = 1 + g * B + b;
+                        if ((w & 31) == lane) { if (w < 32) mine0 = plane; else mine1 = plane; }
+                    }
+                }
+                if (lane < rq.rec_words) rec[lane] = mine0;                         // rec_words <= 64
+                if (lane + 32 < rq.rec_words) rec[lane + 32] = mine1;
+            } else {
+                const uint32_t w0 = lane < rq.rec_words ? __ldg(rec + lane) : 0u;
+                const uint32_t w1 = lane + 32 < rq.rec_words ? __ldg(rec + lane + 32) : 0u;
+                const float scale = __uint_as_float(__shfl_sync(kFull, w0, 0));
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    int c = 0;
+                    for (int b = 0; b < B; ++b) {
+                        const int w = 1 + g * B + b;
+                        const uint32_t plane = __shfl_sync(kFull, w < 32 ? w0 : w1, w & 31);
+                        c |= (int)((plane >> lane) & 1u) << b;
+                    }
+                    y[g] = scale * __fmaf_rn((float)c + 0.5f, cell, -1.0f);
+                }
+                hadamard<D>(y, lane);
+                float out[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) out[g] = __fadd_rn(mu[g], y[g] * sgn[g]);
+                store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
+            }
+        }
+    }
+}
+
 // Decode-time append: one warp per (session, table) predicts the new position and stores its
 // symbols and class in slot a.open_slot of the stream's open chunk.
 template <int D>
@@ -885,6 +1003,22 @@ cudaError_t launch_decode(const CodecArgs& a0, cudaStream_t st) {
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
         kern<<<sm_count() * kBlocksPerSM, kThreads, sm, st>>>(a);
+        count_launch();
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_rotq(const CodecArgs& a0, const RotqArgs& r, bool encode, cudaStream_t st) {
+    CodecArgs a = a0;
+    set_queues(a, 2 * a.sh.L * a.sh.H);
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int) * kTicketWords, st);
+    if (e != cudaSuccess) return e;
+    return dispatch_d(a.sh.d, [&](auto D) {
+        auto kern = encode ? rotq_kernel<decltype(D)::value, true> : rotq_kernel<decltype(D)::value, false>;
+        size_t sm = 0;
+        cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
+        if (e2 != cudaSuccess) return e2;
+        kern<<<sm_count() * kBlocksPerSM, kThreads, sm, st>>>(a, r);
         count_launch();
         return cudaGetLastError();
     });

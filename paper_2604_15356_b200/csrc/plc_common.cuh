@@ -205,6 +205,16 @@ struct CodecArgs {
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
 };
 int codec_grid_warps(int device);
+
+// Rotated fixed-rate quantiser (Prop. 3 step 3): records of 1 + (d/32)*bits words per (stream, position),
+// record of (session s, table t, position i) at word ((s*W + t)*n + i) * rec_words.
+struct RotqArgs {
+    int bits;
+    uint32_t sign_bits[8];      // bit j set: component j is negated before and after the transform
+    uint32_t* records;
+    int rec_words;
+};
+cudaError_t launch_rotq(const CodecArgs& a, const RotqArgs& r, bool encode, cudaStream_t st);
 constexpr int kTicketWords = 1024;               // one counter per work queue (at most one queue per SM)
 
 // Dense (full-vocabulary) prediction, one layer at a time.

@@ -268,6 +268,77 @@ def test_every_plane_count_codes_bit_exactly(dev, orc, delta, most_planes):
     assert float((out.cpu() - kv.float()).abs().max()) <= delta / 2 + 1e-3
 
 
+@pytest.mark.parametrize("d,bits,ranges", [(128, 4, False), (128, 3, True), (64, 8, False), (32, 1, False), (256, 7, False)])
+def test_rotated_quantiser_parity(dev, orc, d, bits, ranges):
+    """Prop. 3 step 3 with the rotated fixed-rate quantiser: records against the oracle's.
+    Tolerances: the kernel rotates in binary32 (log2 d butterfly stages) and predicts in binary32, the
+    oracle in double, so the scale agrees to 1e-5 relative, fewer than 2e-3 of the codes differ and
+    only by one level; where scale and codes agree the record bytes are identical; the decoded vector
+    is the oracle's reconstruction from the same record within 1e-5 of the scale; and
+    ||KV' - KV||_2 <= sqrt(d) s / 2^bits."""
+    S, n, L, H, V, K, CP = 2, 70, 1, 2, 600, 24, 32
+    tokens, logits, T, kv = make_workload(900 + d + bits, S, n, L, H, d, V, K, pp=8.0, sigma=0.2)
+    rng = np.random.default_rng(d * 10 + bits)
+    neg = rng.integers(0, 2, d).astype(np.uint8)
+    pb, pe = ([3, 40], [70, 41]) if ranges else (None, None)
+    ctx = plc.Context(T.to(dev), K, 0.02, chunk_pos=CP)
+    W = ctx.W
+    rb = ctx.rotq_record_bytes(bits)
+    assert rb == 4 + d * bits // 8
+    params = ctx.rotq_params(bits, neg)
+    records = torch.zeros(S * W * n * rb, dtype=torch.uint8, device=dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    pbd = None if pb is None else torch.tensor(pb, dtype=torch.int32, device=dev)
+    ped = None if pe is None else torch.tensor(pe, dtype=torch.int32, device=dev)
+    ctx.encode_rotq(kvd, lgd, params, records, pbd, ped)
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    ctx.decode_rotq(records, lgd, params, out, pbd, ped)
+    assert ctx.sync_status() == plc.OK
+    rec = records.cpu().numpy().reshape(S, W, n, rb)
+    o = out.cpu().numpy()                                           # [L][2][S][H][n][d]
+    kvn = kv.numpy()
+    idx_o, w_o, *_ = orc.topk_softmax(logits.numpy().reshape(S * n, V), None, K)
+    Tn = T.numpy().reshape(W, V, d)
+    n_codes = n_diff = 0
+    for s_ in range(S):
+        b, e = (0, n) if pb is None else (pb[s_], pe[s_])
+        for t_ in range(W):
+            l_, a_, h_ = t_ // (2 * H), (t_ // H) % 2, t_ % H
+            for i in range(n):
+                if not (b <= i < e):
+                    assert not rec[s_, t_, i].any() and not o[l_, a_, s_, h_, i].any()     # untouched
+                    continue
+                mu, _ = orc.mixture(Tn[t_], idx_o[s_ * n + i], w_o[s_ * n + i])
+                x = kvn[l_, a_, s_, h_, i]
+                sc_o, code_o = orc.rotq_quantise(x, mu, neg, bits)
+                sc_g, code_g = orc.rotq_unpack(rec[s_, t_, i], d, bits)
+                assert abs(float(sc_g) - float(sc_o)) <= 1e-5 * float(sc_o) + 1e-9
+                diff = code_g != code_o
+                n_codes += d; n_diff += int(diff.sum())
+                assert np.abs(code_g - code_o).max() <= 1
+                if sc_g == sc_o and not diff.any():
+                    assert np.array_equal(rec[s_, t_, i], orc.rotq_pack(code_o, sc_o, bits))
+                back = orc.rotq_reconstruct(mu, neg, bits, sc_g, code_g)
+                got = o[l_, a_, s_, h_, i]
+                assert np.abs(got - back).max() <= 1e-5 * max(float(sc_g), 1.0) + 2e-6 * np.abs(mu).max()
+                err = got.astype(np.float64) - x.astype(np.float64)
+                assert np.linalg.norm(err) <= np.sqrt(d) * float(sc_g) / (1 << bits) * (1 + 1e-3) + 1e-4
+    assert n_codes > 0 and n_diff <= 2e-3 * n_codes
+
+
+def test_rotated_quantiser_argument_checks(dev):
+    tokens, logits, T, kv = make_workload(5, 1, 8, 1, 1, 256, 64, 4)
+    ctx = plc.Context(T.to(dev), 4, 0.02, chunk_pos=8)
+    with pytest.raises(plc.PlcError) as e:
+        ctx.rotq_record_bytes(8)                                    # 4 + 256 bytes: beyond the record limit
+    assert e.value.code == plc.E_SHAPE
+    params = ctx.rotq_params(4, np.zeros(256, np.uint8))
+    small = torch.zeros(16, dtype=torch.uint8, device=dev)
+    with pytest.raises(plc.PlcError) as e:
+        ctx.encode_rotq(kv.to(dev), logits.to(dev), params, small)
+    assert e.value.code == plc.E_CAPACITY
+
+
 def test_sigma_floor_and_escapes(dev, orc):
     """A point-mass prediction with noisy KV: tiny scale, large residuals -> escapes must round-trip."""
     tokens, logits, T, kv = make_workload(9, 1, 64, 1, 1, 128, 256, 16, sigma=0.3)
