@@ -76,7 +76,7 @@ class ClockSampler:
 # DRAM bytes per vector of the fused kernels, from the ncu capture summarised in
 # profiles/fused_kernels_mid_L4.md (dram__bytes_read.sum + dram__bytes_write.sum over 4.19 M vectors;
 # traffic grows in proportion to the vectors).  Valid for the default workload and chunk size only.
-NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.5, "decode_kernel": 434.2}
+NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.3, "decode_kernel": 431.9}
 
 
 def max_over_ranks(ms, dist, device):
