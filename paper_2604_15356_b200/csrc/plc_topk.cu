@@ -1,13 +1,13 @@
 // Top-K softmax over per-position next-token logits (one thread block per row, rows strided over
 // the grid).  Selection is exact (logit descending, index ascending, -0 = +0).
 //
-// Fast path (K <= 8 per warp of the block ... K <= 256): pass 0 reads the row from HBM and keeps one
+// Fast path (K <= 16 per warp of the block: K <= 128 with 256 threads): pass 0 reads the row from HBM and keeps one
 // maximum per thread; the ceil(K / warps)-th largest thread maximum of every warp, minimised over the
 // warps, is a value with at least K row elements at or above it, i.e. a lower bound of the K-th
 // largest logit that needs no histogram.  Pass 1 (served by L2) sums exp(l - l_max) over the row
 // and collects the few elements at or above that bound (typically 1.2-2 K of them); they are ranked
-// by counting, which yields the K selected in their final order.  Rows whose candidates overflow the
-// list (large tie groups, adversarial layouts) and calls with K > 256 take the radix-select path:
+// by counting (long lists: sorted), which yields the K selected in their final order.  Rows whose
+// candidates overflow the list (large tie groups, adversarial layouts) and larger K take the radix-select path:
 // a 4096-bin histogram of the order-preserving 16-bit key finds the bin that holds the K-th largest,
 // a 16-way refinement finds the key itself, and equal keys are taken in index order.
 // Reductions use warp shuffles in a fixed order, so results are bit-reproducible from run to run.
@@ -108,6 +108,21 @@ __device__ __forceinline__ float exp_rel(float x, float nb) {
 __device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b) {
     __half2 r = __hmax2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
     return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// Sorts n_pad (a power of two) order words in shared memory, largest first, with the block.
+template <int THREADS, class W>
+__device__ __forceinline__ void bitonic_desc(W* v, int n_pad) {
+    for (int k = 2; k <= n_pad; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < (n_pad >> 1); t += THREADS) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));       // lower index of the pair
+                const W a = v[i], b = v[i | j];
+                const bool desc = (i & k) == 0;
+                if ((a < b) == desc) { v[i] = b; v[i | j] = a; }
+            }
+            __syncthreads();
+        }
 }
 
 // Radix select of the K largest keys of the row into sm.sel_* (unordered); three or more passes
@@ -221,7 +236,22 @@ __device__ void select_by_histogram(Smem<THREADS>& sm, const __half* row, int V,
         }
     }
     __syncthreads();
-    // Order the K selected by (key descending, index ascending): rank by counting.
+    // Order the K selected by (key descending, index ascending): a sort of packed order words in the
+    // histogram's memory for large K, rank by counting otherwise.
+    if (K > 128) {
+        unsigned long long* w = reinterpret_cast<unsigned long long*>(sm.hist);
+        int n_pad = 256;
+        while (n_pad < K) n_pad <<= 1;
+        for (int k = tid; k < n_pad; k += THREADS)
+            w[k] = k < K ? ((unsigned long long)sm.sel_key[k] << 32) | (0xffffffffu - (uint32_t)sm.sel_idx[k]) : 0ull;
+        __syncthreads();
+        bitonic_desc<THREADS>(w, n_pad);
+        for (int k = tid; k < K; k += THREADS) {
+            sm.cand_key[k] = (uint32_t)(w[k] >> 32); sm.cand_idx[k] = (int)(0xffffffffu - (uint32_t)w[k]);
+        }
+        __syncthreads();
+        return;
+    }
     for (int k = tid; k < K; k += THREADS) {
         uint32_t key = sm.sel_key[k];
         int idx = sm.sel_idx[k];
@@ -264,8 +294,10 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int V = a.V, K = a.K;
     const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
-    const bool fast = K <= 32 * NW && K <= kCandCap;     // a warp can offer at most 32 thread maxima
     const int per_warp = (K + NW - 1) / NW;
+    // A warp can offer at most 32 thread maxima, and the bound is only tight while it asks for the
+    // upper half of them: beyond 16 per warp the candidates overflow the list on ordinary rows.
+    const bool fast = per_warp <= 16 && K <= kCandCap;
     // The candidate list of the fast path lives in the histogram's memory, which is idle there.
     const bool narrow = V <= 65536;
     uint32_t* list32 = sm.hist;
@@ -364,10 +396,32 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         for (int w = 0; w < NW; ++w) sum_all += sm.red_s[w];
         const int nlist = sm.nlist;
         if (fast && nlist >= K && nlist <= kCandCap) {
-            // rank the candidates (at least K of them) by counting; the first K ranks are the result
-            if (narrow) {
+            // Order the candidates (at least K of them); the first K are the result.  Short lists are
+            // ranked by counting (n^2 / THREADS compares per thread, no barriers), long ones sorted.
+            constexpr int kRankMax = 192;
+            if (nlist > kRankMax) {
+                int n_pad = 256;
+                while (n_pad < nlist) n_pad <<= 1;
+                if (narrow) {
+                    for (int c = nlist + tid; c < n_pad; c += THREADS) list32[c] = 0;    // pad: orders after everything
+                    __syncthreads();
+                    bitonic_desc<THREADS>(list32, n_pad);
+                    for (int k = tid; k < K; k += THREADS) {
+                        const uint32_t v = list32[k];
+                        sm.cand_key[k] = v >> 16; sm.cand_idx[k] = (int)(0xffffu - (v & 0xffffu));
+                    }
+                } else {
+                    for (int c = nlist + tid; c < n_pad; c += THREADS) list64[c] = 0;
+                    __syncthreads();
+                    bitonic_desc<THREADS>(list64, n_pad);
+                    for (int k = tid; k < K; k += THREADS) {
+                        const unsigned long long v = list64[k];
+                        sm.cand_key[k] = (uint32_t)(v >> 32); sm.cand_idx[k] = (int)(0xffffffffu - (uint32_t)v);
+                    }
+                }
+            } else if (narrow) {
                 const int n4 = (nlist + 3) & ~3;
-                for (int c = nlist + tid; c < n4; c += THREADS) list32[c] = 0;       // pad: orders after everything
+                for (int c = nlist + tid; c < n4; c += THREADS) list32[c] = 0;           // pad: orders after everything
                 __syncthreads();
                 for (int c = tid; c < nlist; c += THREADS) {
                     const uint32_t mine = list32[c];
