@@ -410,6 +410,34 @@ __device__ __forceinline__ void load_half_vec(const __half* p, float (&v)[G]) {
     }
 }
 
+// The same load without the conversion (the bits wait in (G+1)/2 registers), and the conversion.
+template <int G>
+__device__ __forceinline__ void load_half_raw(const __half* p, uint32_t (&raw)[(G + 1) / 2]) {
+    if constexpr (G == 8) {
+        const uint4 r = *reinterpret_cast<const uint4*>(p);
+        raw[0] = r.x; raw[1] = r.y; raw[2] = r.z; raw[3] = r.w;
+    } else if constexpr (G == 4) {
+        const uint2 r = *reinterpret_cast<const uint2*>(p);
+        raw[0] = r.x; raw[1] = r.y;
+    } else if constexpr (G == 2) {
+        raw[0] = *reinterpret_cast<const uint32_t*>(p);
+    } else {
+        raw[0] = (uint32_t)__half_as_ushort(*p);
+    }
+}
+template <int G>
+__device__ __forceinline__ void half_raw_to_float(const uint32_t (&raw)[(G + 1) / 2], float (&v)[G]) {
+    if constexpr (G == 1) {
+        v[0] = __half2float(__ushort_as_half((unsigned short)raw[0]));
+    } else {
+#pragma unroll
+        for (int j = 0; j < G / 2; ++j) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[j]));
+            v[2 * j] = f.x; v[2 * j + 1] = f.y;
+        }
+    }
+}
+
 template <int G>
 __device__ __forceinline__ void store_vec(void* base, long long elem, const float (&v)[G], int out_f16) {
     if (out_f16) {
@@ -504,17 +532,24 @@ extern __shared__ int2 g_pair_smem[];   // per warp: two slots of Kp entries
 // Prediction read from the dense variant's buffers: mu [row][tables_in_layer*D] and the variance
 // term s1 [row][tables_in_layer] (sum_v p_v ||T_v||^2 / d); sigma2 = max(0, s1 - ||mu||^2 / d).
 template <int D>
-__device__ __forceinline__ void predict_dense(const CodecArgs& a, long long row, int t_local, int c0, float inv_d,
-                                              float (&mu)[Geo<D>::G], float& sigma2) {
+__device__ __forceinline__ void dense_fetch(const CodecArgs& a, long long row, int t_local, int c0,
+                                            float (&m)[Geo<D>::G], float& s1) {
     constexpr int G = Geo<D>::G;
     const float* mp = a.mu_dense + row * a.mu_ld + (long long)t_local * D + c0;
 #pragma unroll
-    for (int g = 0; g < G; ++g) mu[g] = __ldg(mp + g);
+    for (int g = 0; g < G; ++g) m[g] = __ldg(mp + g);
+    s1 = __ldg(a.s1_dense + row * a.s1_ld + t_local);
+}
+template <int D>
+__device__ __forceinline__ void dense_finish(const CodecArgs& a, int t_local, int c0, float inv_d, const float (&m)[Geo<D>::G],
+                                             float s1, float (&mu)[Geo<D>::G], float& sigma2) {
+    constexpr int G = Geo<D>::G;
+#pragma unroll
+    for (int g = 0; g < G; ++g) mu[g] = m[g];
     if (a.mu_bias) {
 #pragma unroll
         for (int g = 0; g < G; ++g) mu[g] = __fadd_rn(mu[g], __half2float(a.mu_bias[t_local * D + c0 + g]));
     }
-    const float s1 = __ldg(a.s1_dense + row * a.s1_ld + t_local);
     const float s2 = warp_norm2<G>(mu);
     sigma2 = fmaxf(0.f, s1 - s2 * inv_d);
 }
@@ -577,6 +612,10 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             }
             kvp = reinterpret_cast<const __half*>(a.kv.base) + kv_elem(a.kv, it.t, H, it.s, it.p0 + it.P - 1) + c0;
         }
+        // dense source: the prediction of the next position is fetched while this one is coded
+        float m_next[G] = {};
+        float s1_next = 0.f;
+        if (DENSE) dense_fetch<D>(a, (long long)it.s * a.n + it.p0 + it.P - 1, it.t - a.dense_layer * Wl, c0, m_next, s1_next);
         for (int p = it.P - 1; p >= 0; --p) {
             int sym[G];
             int q;
@@ -589,8 +628,16 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                 for (int g = 0; g < G; ++g) sym[g] = a.open_sym[o * D + c0 + g];
             } else {
                 float mu[G], sigma2;
+                uint32_t kv_raw[(G + 1) / 2];
+                load_half_raw<G>(kvp, kv_raw);                                     // in flight during the prediction
+                kvp -= a.kv.sp;
                 if (DENSE) {
-                    predict_dense<D>(a, (long long)it.s * a.n + it.p0 + p, it.t - a.dense_layer * Wl, c0, inv_d, mu, sigma2);
+                    float m_cur[G];
+#pragma unroll
+                    for (int g = 0; g < G; ++g) m_cur[g] = m_next[g];
+                    const float s1_cur = s1_next;
+                    if (p > 0) dense_fetch<D>(a, (long long)it.s * a.n + it.p0 + p - 1, it.t - a.dense_layer * Wl, c0, m_next, s1_next);
+                    dense_finish<D>(a, it.t - a.dense_layer * Wl, c0, inv_d, m_cur, s1_cur, mu, sigma2);
                 } else {
                     const int2* sp = sp0 + buf * Kp;
                     if (p > 0) {                                                  // one position ahead
@@ -614,8 +661,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                 q = __reduce_max_sync(kFull, scale_class(sigma2, floor2, inv_delta2_p));   // same in all lanes
                 skip = ZR && q <= zero_q;
                 float kvv[G];
-                load_half_vec<G>(kvp, kvv);
-                kvp -= a.kv.sp;
+                half_raw_to_float<G>(kv_raw, kvv);
 #pragma unroll
                 for (int g = 0; g < G; ++g) sym[g] = quantise(kvv[g], mu[g], inv_delta_p);
                 __syncwarp();                                                     // readers of this slot are done
@@ -681,10 +727,18 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
         if (!DENSE) prefetch_pairs(sp0, gp, Kp, lane);
         int buf = 0;
         long long kvo = kv_elem(a.kv, it.t, H, it.s, it.p0) + c0;
+        float m_next[G] = {};
+        float s1_next = 0.f;
+        if (DENSE) dense_fetch<D>(a, (long long)it.s * a.n + it.p0, it.t - a.dense_layer * Wl, c0, m_next, s1_next);
         for (int p = 0; p < it.P; ++p) {
             float mu[G], sigma2;
             if (DENSE) {
-                predict_dense<D>(a, (long long)it.s * a.n + it.p0 + p, it.t - a.dense_layer * Wl, c0, inv_d, mu, sigma2);
+                float m_cur[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) m_cur[g] = m_next[g];
+                const float s1_cur = s1_next;
+                if (p + 1 < it.P) dense_fetch<D>(a, (long long)it.s * a.n + it.p0 + p + 1, it.t - a.dense_layer * Wl, c0, m_next, s1_next);
+                dense_finish<D>(a, it.t - a.dense_layer * Wl, c0, inv_d, m_cur, s1_cur, mu, sigma2);
             } else {
                 const int2* sp = sp0 + buf * Kp;
                 if (p + 1 < it.P) {
