@@ -297,7 +297,9 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     const int per_warp = (K + NW - 1) / NW;
     // A warp can offer at most 32 thread maxima, and the bound is only tight while it asks for the
     // upper half of them: beyond 16 per warp the candidates overflow the list on ordinary rows.
-    const bool fast = per_warp <= 16 && K <= kCandCap;
+    // Calls that want no selected set (only lse / log2 P of the tokens / step exponents) skip the selection.
+    const bool select = a.pairs || a.idx || a.w || a.zk;
+    const bool fast = select && per_warp <= 16 && K <= kCandCap;
     // The candidate list of the fast path lives in the histogram's memory, which is idle there.
     const bool narrow = V <= 65536;
     uint32_t* list32 = sm.hist;
@@ -441,30 +443,33 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
                 }
             }
             __syncthreads();
-        } else {
+        } else if (select) {
             __syncthreads();
             select_by_histogram<VEC, THREADS>(sm, row, V, K, ntiles);
         }
 
-        for (int k = tid; k < K; k += THREADS) sm.ek[k] = expf(val_of_key(sm.cand_key[k]) - lmax);
-        __syncthreads();
-        if (wid == 0) {
-            float p = 0.f;
-            for (int k = lane; k < K; k += 32) p += sm.ek[k];
-            p = warp_sum(p);
-            if (lane == 0) sm.sum_k = p;
+        float sum_k = 0.f;
+        if (select) {
+            for (int k = tid; k < K; k += THREADS) sm.ek[k] = expf(val_of_key(sm.cand_key[k]) - lmax);
+            __syncthreads();
+            if (wid == 0) {
+                float p = 0.f;
+                for (int k = lane; k < K; k += 32) p += sm.ek[k];
+                p = warp_sum(p);
+                if (lane == 0) sm.sum_k = p;
+            }
+            __syncthreads();
+            sum_k = sm.sum_k;
+            for (int k = tid; k < K; k += THREADS) {
+                float w = sm.ek[k] / sum_k;
+                int idx = sm.cand_idx[k];
+                if (a.pairs) a.pairs[rowi * a.Kp + k] = make_int2(idx, __float_as_int(w));
+                if (a.idx) a.idx[rowi * K + k] = idx;
+                if (a.w) a.w[rowi * K + k] = w;
+            }
+            if (a.pairs)
+                for (int k = K + tid; k < a.Kp; k += THREADS) a.pairs[rowi * a.Kp + k] = make_int2(sm.cand_idx[0], 0);
         }
-        __syncthreads();
-        const float sum_k = sm.sum_k;
-        for (int k = tid; k < K; k += THREADS) {
-            float w = sm.ek[k] / sum_k;
-            int idx = sm.cand_idx[k];
-            if (a.pairs) a.pairs[rowi * a.Kp + k] = make_int2(idx, __float_as_int(w));
-            if (a.idx) a.idx[rowi * K + k] = idx;
-            if (a.w) a.w[rowi * K + k] = w;
-        }
-        if (a.pairs)
-            for (int k = K + tid; k < a.Kp; k += THREADS) a.pairs[rowi * a.Kp + k] = make_int2(sm.cand_idx[0], 0);
         if (tid == 0) {
             float lse = lmax + logf(sum_all);
             if (a.lse) a.lse[rowi] = lse;
@@ -496,16 +501,22 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const bool vec = (a.V % 8 == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
     // The second pass over a row should find it in L2: rows of up to 128 KB are read by 256 threads
-    // with five blocks per SM, longer rows by 1024 threads with one block per SM.
+    // with five blocks per SM, longer rows by 512 threads with two blocks per SM (two, so that one
+    // block streams while the other sits at the barrier between its passes).
     const bool wide = (long long)a.V * 2 > 128 * 1024;
-    const long long per_sm = wide ? 1 : 5;
-    const long long blocks = a.N < sms * per_sm ? a.N : sms * per_sm;
+    auto launch = [&](auto kern, int threads, int cap) {
+        int occ = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, 0) != cudaSuccess || occ < 1) occ = 1;
+        const long long per_sm = occ < cap ? occ : cap;       // the rows in flight stay within L2
+        const long long blocks = a.N < sms * per_sm ? a.N : sms * per_sm;
+        kern<<<(unsigned)blocks, threads, 0, st>>>(a);
+    };
     if (wide) {
-        if (vec) topk_softmax_kernel<true, 1024><<<(unsigned)blocks, 1024, 0, st>>>(a);
-        else topk_softmax_kernel<false, 1024><<<(unsigned)blocks, 1024, 0, st>>>(a);
+        if (vec) launch(topk_softmax_kernel<true, 512>, 512, 2);
+        else launch(topk_softmax_kernel<false, 512>, 512, 2);
     } else {
-        if (vec) topk_softmax_kernel<true, 256><<<(unsigned)blocks, 256, 0, st>>>(a);
-        else topk_softmax_kernel<false, 256><<<(unsigned)blocks, 256, 0, st>>>(a);
+        if (vec) launch(topk_softmax_kernel<true, 256>, 256, 5);
+        else launch(topk_softmax_kernel<false, 256>, 256, 5);
     }
     count_launch();
     return cudaGetLastError();

@@ -184,6 +184,9 @@ def test_topk_softmax_parity(dev, orc):
         again = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev))
         for k in out:
             assert torch.equal(out[k], again[k])                  # run-to-run identical
+        only = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev), want=("lse", "logp2"))
+        assert set(only) == {"lse", "logp2"}                      # no selected set asked for: the selection is skipped
+        assert torch.equal(only["lse"], out["lse"]) and torch.equal(only["logp2"], out["logp2"])
 
 
 def test_tiny_config_full_parity(dev, orc):
