@@ -172,7 +172,9 @@ plc_status plc_reserve(plc_ctx* ctx, int64_t max_positions);
  * Outputs, each optional (NULL = skip): idx_dev [N][K] int32 ordered by (logit descending, index
  * ascending); w_dev [N][K] float, exp(l_k - l_max) / sum over the K; lse_dev [N] natural
  * log-sum-exp over V; zk_dev [N] sum of the K probabilities; logp2_dev [N] log2 P(tokens[i])
- * (needs tokens_dev; the edge weight of the probabilistic language trie, Def. 1). */
+ * (needs tokens_dev; the edge weight of the probabilistic language trie, Def. 1).  A call with idx_dev,
+ * w_dev and zk_dev all NULL does not determine the K largest at all (one pass for the maximum, one for
+ * the sum): the cheap way to get the trie's edge weights for plc_prefix_dedup. */
 plc_status plc_topk_softmax(plc_ctx* ctx, const void* logits_dev, const int32_t* tokens_dev, int64_t N,
                             int32_t* idx_dev, float* w_dev, float* lse_dev, float* zk_dev, float* logp2_dev,
                             void* stream);
