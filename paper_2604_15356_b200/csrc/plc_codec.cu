@@ -369,7 +369,7 @@ __device__ __forceinline__ unsigned smid() {
 struct QueueCursor { int q, tried; };
 __device__ __forceinline__ QueueCursor queue_of_this_sm(const CodecArgs& a) {
     QueueCursor qc;
-    qc.q = min((int)(smid() / (unsigned)a.sched_g), a.sched_nq - 1);
+    qc.q = (int)((smid() / (unsigned)a.sched_g) % (unsigned)a.sched_nq);   // fewer tables than SM groups: spread the groups evenly
     qc.tried = 0;
     return qc;
 }
