@@ -90,7 +90,9 @@ typedef struct {
  * chunk_bytes_dev[slot]  = its exact size (0 = no such chunk).  Chunks are placed in the order in
  * which they are finished, so offsets differ from run to run; the bytes of each chunk do not.
  * *total_bytes_dev = bytes of payload_dev in use (with padding); the caller zeroes it before the
- * first plc_encode into a buffer and may keep it to append more chunks behind the ones present. */
+ * first plc_encode into a buffer and may keep it to append more chunks behind the ones present.
+ * It must be a multiple of 16 whenever an encoder runs (the library only ever adds multiples of 16);
+ * otherwise the chunks of that call are not written and the status word reports PLC_E_ALIGN. */
 typedef struct {
     uint8_t* payload_dev;
     uint64_t payload_capacity;
@@ -108,6 +110,8 @@ typedef struct {
     int32_t* q_dev;
     float* mu_dev;
     int32_t* bits_dev;   /* [S][n] int32: b_i of the adaptive quantiser (adaptive calls only) */
+    int32_t count_ideal_bits;   /* non-zero (plc_encode and variants): add the code length the coder's model
+                                 * assigns to everything coded to plc_stats.ideal_bits */
 } plc_debug_buffers;
 
 typedef struct {
@@ -116,6 +120,11 @@ typedef struct {
     uint64_t n_escapes;       /* components whose magnitude left the 63-symbol alphabet */
     uint64_t coded_vectors;   /* (stream, position) pairs covered by the chunks written */
     uint64_t skipped_vectors; /* of those, pairs the zero-rate rule left out of the stream */
+    double ideal_bits;        /* sum over the coded components of log2(2^15 / f) + raw bit-plane bits + 32 per
+                               * escape: the ideal -log2 P code length under the coder's own model (Prop. 2's
+                               * "standard source coding" rate); only encodes that asked for it contribute
+                               * (plc_debug_buffers.count_ideal_bits).  8 * payload_bytes exceeds it by the
+                               * coder's state flush (128 bytes per chunk) and rounding only. */
 } plc_stats;
 
 /* State of a batch of B sessions that grow by one position per plc_append_step (lock step).
@@ -308,7 +317,8 @@ plc_status plc_append_sizes(const plc_ctx* ctx, int32_t B, uint64_t* open_sym_by
  *   chunk, with n_streams = B*W); classes outside [-24, 135] are clamped and reported.
  *   Chunk `chunk_index` of stream i goes to index slot i*out->max_chunks + chunk_index.
  *   status_dev: one device word, an OUTPUT: 0, or a bit-or of 1 (payload capacity exceeded; nothing
- *   is written past it and *total_bytes_dev holds the size needed) and 4 (a class was out of range).
+ *   is written past it and *total_bytes_dev holds the size needed), 4 (a class was out of range) and
+ *   16 (*total_bytes_dev was not a multiple of 16: the chunk is not written).
  * Limits: n_pos * head_dim <= 4096 components per chunk (PLC_E_SHAPE beyond that); head_dim in
  * {32, 64, 128, 256}.  All working memory is one static device array of about 8 MiB that every GPU
  * using the library holds until the process exits.  Every call on a device shares that array, so
@@ -319,8 +329,15 @@ plc_status plc_rans_encode_static(const int32_t* sym_dev, const int32_t* q_dev, 
                                   int32_t head_dim, int32_t chunk_capacity, int32_t chunk_index,
                                   const plc_streams* out, uint32_t* status_dev, void* stream);
 
-/* Waits for the stream and returns the device status word's most severe code; clears it. */
+/* Waits for the stream and returns the device status word's most severe code; clears it.
+ * PLC_E_ALIGN here means that *total_bytes_dev was not a multiple of 16 when an encoder reserved a
+ * chunk's place (the chunk is then not written). */
 plc_status plc_sync_status(plc_ctx* ctx, void* stream);
+/* The same word read without waiting for any enqueued work (a 4-byte copy on a stream of the
+ * context's own) and without clearing it: *bits receives the raw word (1 capacity, 2 corrupt,
+ * 8 a bounded wait inside a kernel ran out, 16 unaligned byte cursor), the return value its most
+ * severe code.  Work still running may set further bits afterwards. */
+plc_status plc_poll_status(plc_ctx* ctx, uint32_t* bits);
 /* Waits for the stream, copies the counters, optionally clears them. */
 plc_status plc_get_stats(plc_ctx* ctx, plc_stats* out, int32_t reset, void* stream);
 
@@ -334,6 +351,11 @@ plc_status plc_build_table(int32_t qp, uint32_t* f, uint32_t* c);
  * variant's tensor-core contraction of the last layer) and returns its duration.  PLC_E_STATE if
  * no such launch was recorded. */
 plc_status plc_set_profiling(plc_ctx* ctx, int32_t on);
+/* Work-queue layout the most recent top-K plc_encode / plc_decode of this context used: *n_queues
+ * queues of (table, session, chunk) items, each served by *sms_per_queue SMs (one queue for the whole
+ * GPU when the tables in flight fit in L2, else about one table's worth of chunks per queue).  For
+ * tests and benchmarks that must state which path they ran.  PLC_E_STATE before the first such call. */
+plc_status plc_last_schedule(const plc_ctx* ctx, int32_t* n_queues, int32_t* sms_per_queue);
 plc_status plc_last_kernel_ms(plc_ctx* ctx, int32_t which, float* ms);
 /* Number of kernels this library has launched in this process (for benchmarks). */
 uint64_t plc_launch_count(void);

@@ -24,7 +24,7 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
            "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters", "plc_rotq_record_bytes", "plc_encode_rotq",
-           "plc_decode_rotq"]
+           "plc_decode_rotq", "plc_poll_status", "plc_last_schedule"]
 
 
 def sources():
@@ -63,12 +63,13 @@ class Streams(C.Structure):
 
 
 class DebugBuffers(C.Structure):
-    _fields_ = [("sym_dev", C.c_void_p), ("q_dev", C.c_void_p), ("mu_dev", C.c_void_p), ("bits_dev", C.c_void_p)]
+    _fields_ = [("sym_dev", C.c_void_p), ("q_dev", C.c_void_p), ("mu_dev", C.c_void_p), ("bits_dev", C.c_void_p),
+                ("count_ideal_bits", C.c_int32)]
 
 
 class Stats(C.Structure):
     _fields_ = [("payload_bytes", C.c_uint64), ("n_chunks", C.c_uint64), ("n_escapes", C.c_uint64),
-                ("coded_vectors", C.c_uint64), ("skipped_vectors", C.c_uint64)]
+                ("coded_vectors", C.c_uint64), ("skipped_vectors", C.c_uint64), ("ideal_bits", C.c_double)]
 
 
 class RotqParams(C.Structure):
@@ -128,9 +129,14 @@ def kv_view(kv):
 class StreamSet:
     """Device buffers of a coded output: payload, per-chunk index, byte cursor."""
 
-    def __init__(self, n_streams, max_chunks, capacity, device="cuda"):
+    def __init__(self, n_streams, max_chunks, capacity, device="cuda", guard=0):
+        """guard > 0 allocates that many extra bytes behind the stated capacity, filled with 0xA5, so
+        that a test can show nothing was written past the capacity (``guard_intact``)."""
         import torch
-        self.payload = torch.empty(int(capacity), dtype=torch.uint8, device=device)
+        self.capacity = int(capacity)
+        self.payload = torch.empty(self.capacity + int(guard), dtype=torch.uint8, device=device)
+        if guard:
+            self.payload[self.capacity:] = 0xA5
         self.chunk_offset = torch.zeros(n_streams * max_chunks, dtype=torch.int64, device=device)
         self.chunk_bytes = torch.zeros(n_streams * max_chunks, dtype=torch.int32, device=device)
         self.total_bytes = torch.zeros(1, dtype=torch.int64, device=device)
@@ -138,8 +144,11 @@ class StreamSet:
         self.n_streams = n_streams
 
     def c(self):
-        return Streams(self.payload.data_ptr(), self.payload.numel(), self.chunk_offset.data_ptr(),
+        return Streams(self.payload.data_ptr(), self.capacity, self.chunk_offset.data_ptr(),
                        self.chunk_bytes.data_ptr(), self.total_bytes.data_ptr(), self.max_chunks)
+
+    def guard_intact(self):
+        return bool((self.payload[self.capacity:] == 0xA5).all())
 
     def chunk(self, slot):
         """Bytes of one chunk as a CPU numpy array."""
@@ -294,6 +303,18 @@ class Context:
 
     def sync_status(self):
         return lib().plc_sync_status(self._h, _stream())
+
+    def poll_status(self):
+        """(status code, raw bits) of the device status word, without waiting for enqueued work."""
+        bits = C.c_uint32()
+        rc = lib().plc_poll_status(self._h, C.byref(bits))
+        return rc, bits.value
+
+    def last_schedule(self):
+        """(queues, SMs per queue) of the most recent top-K encode / decode launch."""
+        nq, g = C.c_int32(), C.c_int32()
+        _check(lib().plc_last_schedule(self._h, C.byref(nq), C.byref(g)), "plc_last_schedule")
+        return nq.value, g.value
 
     def set_profiling(self, on=True):
         _check(lib().plc_set_profiling(self._h, int(on)), "plc_set_profiling")

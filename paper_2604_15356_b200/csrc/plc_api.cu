@@ -23,6 +23,8 @@ struct plc_ctx {
     unsigned long long staging_words_per_warp;
     unsigned int* ticket;
     unsigned int* status;
+    unsigned int* status_host;      // pinned word plc_poll_status copies into
+    cudaStream_t poll_stream;       // non-blocking stream of plc_poll_status
     Counters* counters;
     uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1; linear variant: P, Ebar, s1, A_layer, mu
     size_t dense_bytes;
@@ -32,12 +34,21 @@ struct plc_ctx {
     int lin_dm;
     uint8_t* lin_model;             // E transposed (bf16) and the candidate-norm table of every (layer, table)
     size_t lin_off[2];
+    int last_nq, last_g;            // work-queue layout of the most recent top-K encode / decode launch
     int profiling;                  // record events around the codec kernels
     cudaEvent_t ev[6];              // encode start/stop, decode start/stop, dense contraction start/stop
     int ev_valid[3];
 };
 
 namespace {
+
+plc_status status_code(unsigned int w) {
+    if (w & kStTimeout) return PLC_E_CUDA;
+    if (w & kStCorrupt) return PLC_E_CORRUPT;
+    if (w & kStCursor) return PLC_E_ALIGN;
+    if (w & kStCapacity) return PLC_E_CAPACITY;
+    return PLC_OK;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 bool valid_d(int d) { return d == 32 || d == 64 || d == 128 || d == 256; }
@@ -188,6 +199,8 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
               cudaMalloc(&c->staging, sizeof(uint16_t) * c->staging_words_per_warp * warps) == cudaSuccess &&
               cudaMalloc(&c->ticket, sizeof(unsigned int) * kTicketWords) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(unsigned int)) == cudaSuccess &&
+              cudaMallocHost(&c->status_host, sizeof(unsigned int)) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->poll_stream, cudaStreamNonBlocking) == cudaSuccess &&
               cudaMalloc(&c->counters, sizeof(Counters)) == cudaSuccess;
     if (ok) ok = cudaMemset(c->status, 0, sizeof(unsigned int)) == cudaSuccess &&
                  cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
@@ -212,6 +225,8 @@ plc_status plc_destroy(plc_ctx* c) {
     cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->step_exp); cudaFree(c->staging);
     cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch); cudaFree(c->lin_model);
     for (int i = 0; i < 6; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    if (c->status_host) cudaFreeHost(c->status_host);
+    if (c->poll_stream) cudaStreamDestroy(c->poll_stream);
     delete c;
     return PLC_OK;
 }
@@ -335,13 +350,14 @@ static plc_status encode_impl(plc_ctx* c, const plc_kv_view* kv, const void* log
     CodecArgs a = base_args(c);
     a.kv = to_dev(kv); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
     a.st = to_dev(out);
-    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev, dbg->count_ideal_bits};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, true, st);
     if (c->cfg.variant == PLC_PRED_LINEAR) return run_linear(c, a, logits_dev, true, st);
     rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;
     a.step_exp = tokens_dev ? c->step_exp : nullptr;
+    codec_schedule(a, 2 * a.sh.L * a.sh.H, &c->last_nq, &c->last_g);
     if (c->profiling) cudaEventRecord(c->ev[0], st);
     cudaError_t e = launch_encode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[1], st); c->ev_valid[0] = 1; }
@@ -378,13 +394,14 @@ static plc_status decode_impl(plc_ctx* c, const plc_streams* in, const void* log
     CodecArgs a = base_args(c);
     a.kv = to_dev(kv_out); a.S = S; a.n = n; a.pos_begin = pos_begin_dev; a.pos_end = pos_end_dev;
     a.st = to_dev(in);
-    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev};
+    if (dbg) a.dbg = DebugDev{dbg->sym_dev, dbg->q_dev, dbg->mu_dev, dbg->count_ideal_bits};
     if (c->cfg.variant == PLC_PRED_DENSE) return run_dense(c, a, logits_dev, false, st);
     if (c->cfg.variant == PLC_PRED_LINEAR) return run_linear(c, a, logits_dev, false, st);
     rc = run_topk_for(c, logits_dev, S, n, pos_begin_dev, pos_end_dev, st, tokens_dev, dbg ? dbg->bits_dev : nullptr);
     if (rc) return rc;
     a.pairs = c->pairs;
     a.step_exp = tokens_dev ? c->step_exp : nullptr;
+    codec_schedule(a, 2 * a.sh.L * a.sh.H, &c->last_nq, &c->last_g);
     if (c->profiling) cudaEventRecord(c->ev[2], st);
     cudaError_t e = launch_decode(a, st);
     if (c->profiling) { cudaEventRecord(c->ev[3], st); c->ev_valid[1] = 1; }
@@ -508,10 +525,18 @@ plc_status plc_sync_status(plc_ctx* c, void* stream) {
     if (cudaMemcpyAsync(&w, c->status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PLC_E_CUDA;
     if (cudaMemsetAsync(c->status, 0, sizeof(w), st) != cudaSuccess) return PLC_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
-    if (w & kStTimeout) return PLC_E_CUDA;
-    if (w & kStCorrupt) return PLC_E_CORRUPT;
-    if (w & kStCapacity) return PLC_E_CAPACITY;
-    return PLC_OK;
+    return status_code(w);
+}
+
+plc_status plc_poll_status(plc_ctx* c, uint32_t* bits) {
+    if (!c || !bits) return PLC_E_INVALID;
+    // a copy on the context's own non-blocking stream: it does not wait for the work enqueued on the
+    // caller's streams and reads the word as it stands now
+    if (cudaMemcpyAsync(c->status_host, c->status, sizeof(unsigned int), cudaMemcpyDeviceToHost, c->poll_stream) != cudaSuccess)
+        return PLC_E_CUDA;
+    if (cudaStreamSynchronize(c->poll_stream) != cudaSuccess) return PLC_E_CUDA;
+    *bits = *c->status_host;
+    return status_code(*c->status_host);
 }
 
 plc_status plc_get_stats(plc_ctx* c, plc_stats* out, int32_t reset, void* stream) {
@@ -523,6 +548,7 @@ plc_status plc_get_stats(plc_ctx* c, plc_stats* out, int32_t reset, void* stream
     if (cudaStreamSynchronize(st) != cudaSuccess) return PLC_E_CUDA;
     out->payload_bytes = h.payload_bytes; out->n_chunks = h.n_chunks; out->n_escapes = h.n_escapes;
     out->coded_vectors = h.coded_vectors; out->skipped_vectors = h.skipped_vectors;
+    out->ideal_bits = h.ideal_bits;
     return PLC_OK;
 }
 
@@ -537,6 +563,13 @@ plc_status plc_build_table(int32_t qp, uint32_t* f, uint32_t* cdf) {
     build_freqs(qp, f);
     cdf[0] = 0;
     for (int i = 0; i < kNumSym; ++i) cdf[i + 1] = cdf[i] + f[i];
+    return PLC_OK;
+}
+
+plc_status plc_last_schedule(const plc_ctx* c, int32_t* n_queues, int32_t* sms_per_queue) {
+    if (!c || !n_queues || !sms_per_queue) return PLC_E_INVALID;
+    if (c->last_nq < 1) return PLC_E_STATE;
+    *n_queues = c->last_nq; *sms_per_queue = c->last_g;
     return PLC_OK;
 }
 

@@ -508,12 +508,14 @@ __device__ __forceinline__ void commit_chunk(const CodecArgs& a, long long slot,
     off = __shfl_sync(kFull, off, 0);
     if (lane == 0 && n_escapes) atomicAdd(&a.counters->n_escapes, (unsigned long long)n_escapes);
     const bool fits = off + nbytes <= a.st.capacity;
+    const bool aligned = (off & 15ull) == 0;             // the caller's byte cursor must be a multiple of 16
     if (lane == 0) {
         a.st.chunk_offset[slot] = off;
         a.st.chunk_bytes[slot] = nbytes;
         if (!fits) atomicOr(a.status, kStCapacity);
+        if (!aligned) atomicOr(a.status, kStCursor);
     }
-    if (!fits) return;
+    if (!fits || !aligned) return;
     uint8_t* dst = a.st.payload + off;
     reinterpret_cast<uint32_t*>(dst)[lane] = x;
     uint16_t* dw = reinterpret_cast<uint16_t*>(dst + 128);
@@ -601,6 +603,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
         int wp = cap_words;
         unsigned n_escapes = 0;
         int n_skipped = 0;
+        float ideal = 0.f;                                                         // this lane's share, if asked for
         const int2* gp = nullptr;
         const __half* kvp = nullptr;
         int buf = 0;
@@ -678,7 +681,20 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             if (ZR && skip) { ++n_skipped; continue; }                             // nothing is coded
             int s, qp;
             class_params(q, s, qp);
+            if (a.dbg.ideal) {                      // statistics only: log2(2^15 / f) + s raw bits (+ 32 per escape)
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const int nh = -((sym[g] + (s ? (1 << (s - 1)) : 0)) >> s);
+                    const uint32_t zz0 = (uint32_t)((nh << 1) ^ (nh >> 31));
+                    const uint32_t f = tb.enc[qp - kQMin][min(zz0, (uint32_t)kEsc)].fc & 0xffffu;
+                    ideal += (float)(kProbBits + s) - log2f((float)f) + (zz0 > 2u * kHiMax ? 32.f : 0.f);
+                }
+            }
             wp = encode_position<G>(sym, s, a.step_exp != nullptr, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
+        }
+        if (a.dbg.ideal) {
+            ideal = warp_sum(ideal);
+            if (lane == 0) atomicAdd(&a.counters->ideal_bits, (double)ideal);
         }
         commit_chunk(a, it.slot, x, stage, wp, cap_words, lane, it.P, n_escapes, n_skipped);
         __syncwarp();
@@ -970,12 +986,20 @@ int sm_count() {
 
 int codec_grid_warps(int) { return sm_count() * kBlocksPerSM * kWarpsPerBlock; }
 
+static void set_queues(CodecArgs& a, int n_tables);
+
 // Queue layout of a gather launch.  With one queue for the whole GPU the resident warps span
 // about (resident warps / chunks per table) + 1 consecutive tables; if those tables fit in L2 that
 // is the layout with the smallest working set and it is kept.  Otherwise L2 cannot hold the tables
 // in flight whatever the order, and the only reuse left is between positions that share candidate
 // rows: then a queue is served by as few SMs as keep busy with ONE table's chunks (rounded down),
 // so that the warps of an SM gather from one or two tables and shared rows stay in that SM's L1.
+void codec_schedule(const CodecArgs& a0, int n_tables, int* nq, int* g) {
+    CodecArgs a = a0;
+    set_queues(a, n_tables);
+    *nq = a.sched_nq; *g = a.sched_g;
+}
+
 static void set_queues(CodecArgs& a, int n_tables) {
     const int sms = sm_count(), warps_per_sm = kBlocksPerSM * kWarpsPerBlock;
     const long long per_table = std::max(1LL, (long long)a.S * a.st.max_chunks);

@@ -21,11 +21,12 @@ constexpr int kSymLimit = 1 << 30;
 constexpr uint32_t kFull = 0xffffffffu;
 
 // Bits of the device status word.
-constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u, kStTimeout = 8u;
+constexpr uint32_t kStCapacity = 1u, kStCorrupt = 2u, kStBadClass = 4u, kStTimeout = 8u, kStCursor = 16u;
 
 // Device counters (plc_stats).
 struct Counters {
     unsigned long long payload_bytes, n_chunks, n_escapes, coded_vectors, skipped_vectors;
+    double ideal_bits;     // code length under the coder's model (only counted on request)
 };
 
 // Frequency-table entry used by the encoder: rcp = floor(2^32 / f) (2^32-1 for f = 1),
@@ -184,6 +185,7 @@ struct StreamsDev {
 
 struct DebugDev {
     int32_t* sym; int32_t* q; float* mu;
+    int ideal;             // non-zero: add every coded component's model code length to Counters::ideal_bits
 };
 
 struct CodecArgs {
@@ -205,6 +207,8 @@ struct CodecArgs {
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
 };
 int codec_grid_warps(int device);
+// Work-queue layout a gather launch over n_tables tables would use: nq queues, g SMs per queue.
+void codec_schedule(const CodecArgs& a, int n_tables, int* nq, int* g);
 
 // Rotated fixed-rate quantiser (Prop. 3 step 3): records of 1 + (d/32)*bits words per (stream, position),
 // record of (session s, table t, position i) at word ((s*W + t)*n + i) * rec_words.

@@ -5,9 +5,11 @@
 // K-major (V contiguous).  One CTA computes a 128 x 256 tile: a TMA producer thread fills a
 // 4-stage shared-memory ring (128B-swizzled boxes of 64 K-elements), one thread issues
 // tcgen05.mma (128x256x16) into 256 TMEM columns and releases ring slots with tcgen05.commit,
-// four warps read the accumulators back with tcgen05.ld and store the tile.  No cluster, no
-// multicast.  Every mbarrier wait is bounded; a wait that runs out sets an error bit, the CTA
-// drains its own copies, frees its TMEM and returns.
+// four warps read the accumulators back with tcgen05.ld and store the tile.  Single-CTA launch:
+// every TMA load lands in this CTA's own shared memory and the tensor maps cover this GPU's memory
+// only.  Every mbarrier wait is bounded; a wait that runs out sets an error bit and a CTA-wide
+// `failed` word: the producer stops and waits (bounded) for the copies it has in flight, the
+// epilogue stores nothing, and the CTA frees its TMEM and returns.
 // The variance term s1[row][table] = sum_v P[row][v] * bf16(||Tb_v||^2 / d) is a second launch of
 // the same kernel with a narrow N tile (one column per table).
 #include <cuda.h>
@@ -17,6 +19,13 @@
 
 namespace plc {
 namespace {
+
+int dense_sm_count() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        sms = 1;
+    return sms;
+}
 
 constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4, kUmmaK = 16;
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
@@ -80,6 +89,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);   // full[4], empty[4], tmem_full
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+    volatile uint32_t* failed = tmem_slot + 1;        // set by any role whose wait ran out
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * bn;
     const uint32_t stage_tx = (uint32_t)(kABytes + bn * kBK * 2), idesc = make_idesc(bn);
@@ -88,6 +98,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(tfull, 1);
+        *failed = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -106,7 +117,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % kStages;
             const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
-            ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, status);
+            ok = !*failed && mbar_wait(empty0 + 8 * s, ph ^ 1u, status);
             if (!ok) break;
             mbar_expect_tx(full0 + 8 * s, stage_tx);
             const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
@@ -116,6 +127,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         if (!ok) {
             // drain: the copies already issued still land in this CTA's shared memory
+            *failed = 1u;
             for (int kb = issued > kStages ? issued - kStages : 0; kb < issued; ++kb)
                 mbar_wait(full0 + 8 * (kb % kStages), (uint32_t)(kb / kStages) & 1u, status);
         }
@@ -126,7 +138,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int s = kb % kStages;
             const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
             ok = mbar_wait(full0 + 8 * s, ph, status);
-            if (!ok) break;
+            if (!ok) { *failed = 1u; __threadfence_block(); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
             const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kABytes);
@@ -135,10 +147,12 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
             umma_commit(empty0 + 8 * s);              // frees the ring slot when these MMAs have read it
         }
-        umma_commit(tfull);                           // accumulators complete (or nothing pending)
+        umma_commit(tfull);                           // arrives when the MMAs issued so far are done (all of them, or none pending)
     } else if (warp >= 2) {
         // epilogue: warp w reads TMEM lanes 32*(w%4) ... +31
-        const bool ok = mbar_wait(tfull, 0, status);
+        bool ok = mbar_wait(tfull, 0, status);
+        if (!ok) *failed = 1u;
+        ok = ok && !*failed;                          // partial accumulators are never stored
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int q = warp & 3;
         const int row = m0 + q * 32 + lane;
@@ -300,6 +314,12 @@ __global__ void __launch_bounds__(256) rownorm_bf16_kernel(const __half* __restr
     }
 }
 
+// Blocks of 256 threads for n work items, at most 16 per SM (grid-stride kernels).
+unsigned blocks_for(long long n) {
+    const long long b = (n + 255) / 256, cap = (long long)dense_sm_count() * 16;
+    return (unsigned)(b < cap ? (b > 0 ? b : 1) : cap);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -387,7 +407,8 @@ size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
 }
 
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st) {
-    long long blocks = sh.rows < 148 * 8 ? sh.rows : 148 * 8;
+    const long long cap_blocks = (long long)dense_sm_count() * 8;
+    long long blocks = sh.rows < cap_blocks ? sh.rows : cap_blocks;
     __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(scratch + off[0]);
     if (sh.V % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0)
         softmax_bf16_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(logits, sh.rows, sh.V, sh.ldv, P);
@@ -415,7 +436,7 @@ cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* sc
     const long long nrows = (long long)sh.tables * sh.V;
     e = cudaMemsetAsync(Nb, 0, (size_t)((sh.tables + 15) / 16 * 16) * sh.ldv * 2, st);     // padding rows / columns read as zero
     if (e != cudaSuccess) return e;
-    rownorm_bf16_kernel<<<(unsigned)((nrows + 7) / 8 < 148 * 16 ? (nrows + 7) / 8 : 148 * 16), 256, 0, st>>>(T_layer, nrows, sh.V, sh.d, sh.ldv, Nb);
+    rownorm_bf16_kernel<<<blocks_for(nrows * 32), 256, 0, st>>>(T_layer, nrows, sh.V, sh.d, sh.ldv, Nb);
     CUtensorMap ma, mb;
     const int nb_rows = (sh.tables + 15) / 16 * 16;                     // norm matrix rows, <= 256
     CUtensorMap mn;
@@ -464,7 +485,7 @@ size_t linear_scratch_bytes(const LinearShape& sh, size_t* off /*[6]: P, Ef, Eb1
 }
 
 static int tile_for(int n) { return n % 256 == 0 ? 256 : (n % 128 == 0 ? 128 : 64); }
-static unsigned blocks_for(long long n) { long long b = (n + 255) / 256; return (unsigned)(b < 148 * 16 ? (b > 0 ? b : 1) : 148 * 16); }
+
 
 // Creation: E transposed to bf16 and the norm table of every (layer, table).  Allocates (and
 // frees) its temporaries; synchronises the stream.
@@ -490,7 +511,7 @@ cudaError_t linear_prepare(const __half* E, const __half* A, const __half* c, co
             e = launch_gemm(Eb, sh.V, Ab, sh.ncols_pad, sh.dm, 256, tlin, sh.ncols, sh.ncols, status, st);
             if (e != cudaSuccess) break;
             const long long pairs = (long long)sh.V * sh.tables;
-            tlin_norm_kernel<<<(unsigned)((pairs + 7) / 8 < 148 * 16 ? (pairs + 7) / 8 : 148 * 16), 256, 0, st>>>(
+            tlin_norm_kernel<<<blocks_for(pairs * 32), 256, 0, st>>>(
                 tlin, sh.ncols, c + (size_t)l * sh.ncols, sh.V, sh.tables, sh.d, sh.ldv, NbAll + (size_t)l * sh.tables * sh.ldv);
             count_launch(2);
             e = cudaGetLastError();

@@ -95,7 +95,10 @@ cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, cons
     if (S <= 0) return cudaSuccess;
     long long pairs = (long long)S * S;
     long long blocks = (pairs + 7) / 8;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        sms = 1;
+    if (blocks > (long long)sms * 8) blocks = (long long)sms * 8;
     lcp_dt_kernel<<<(unsigned)blocks, 256, 0, st>>>(tokens, lens, logp2, S, (long long)stride, lcp, dT);
     parent_kernel<<<(S + 127) / 128, 128, 0, st>>>(lcp, S, parent, shared_len);
     count_launch(2);

@@ -22,7 +22,6 @@ constexpr size_t kStBytes = kStHeader + (size_t)kStWarps * kStWordsPerWarp * siz
 // once per device with cudaGetSymbolAddress (static_scratch() below).
 static __device__ __align__(256) unsigned char g_static_scratch[kStBytes];
 
-constexpr uint32_t kStBadClass = 4u;
 
 struct EncTablesSt { EncEntry enc[kNumTables][kNumSym]; };
 
@@ -111,11 +110,13 @@ rans_encode_static_kernel(const int32_t* __restrict__ sym, const int32_t* __rest
         unsigned long long off = 0;
         if (lane == 0) off = atomicAdd(out.total_bytes, (unsigned long long)((nbytes + 15u) & ~15u));
         off = __shfl_sync(kFull, off, 0);
-        const bool fits = off + nbytes <= out.capacity;
+        const bool aligned = (off & 15ull) == 0;        // the caller's byte cursor must be a multiple of 16
+        const bool fits = off + nbytes <= out.capacity && aligned;
         if (lane == 0) {
             out.chunk_offset[slot] = off;
             out.chunk_bytes[slot] = nbytes;
-            if (!fits) atomicOr(status, kStCapacity);
+            if (off + nbytes > out.capacity) atomicOr(status, kStCapacity);
+            if (!aligned) atomicOr(status, kStCursor);
         }
         if (__any_sync(kFull, bad_class) && lane == 0) atomicOr(status, kStBadClass);
         if (fits) {

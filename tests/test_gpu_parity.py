@@ -43,18 +43,18 @@ def make_workload(seed, S, n, L, H, d, V, K, pp=12.0, sigma=0.05, alpha=0.0, max
     return tokens, logits, T, kv
 
 
-def gpu_encode(dev, T, kv, logits, K, delta, CP, pos_begin=None, pos_end=None, capacity=None, sigma_floor=0.0):
+def gpu_encode(dev, T, kv, logits, K, delta, CP, pos_begin=None, pos_end=None, capacity=None, sigma_floor=0.0, guard=0):
     L, _, H, V, d = T.shape
     S, n = logits.shape[:2]
     ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, sigma_floor=sigma_floor)
     W = ctx.W
     mc = ctx.max_chunks(n)
     cap = capacity if capacity is not None else S * W * mc * 160 + 3 * S * n * W * d + 4096
-    st = plc.StreamSet(S * W, mc, cap, dev)
+    st = plc.StreamSet(S * W, mc, cap, dev, guard=guard)
     sym = torch.zeros(S, n, W, d, dtype=torch.int32, device=dev)
     q = torch.full((S, n, W), -99, dtype=torch.int32, device=dev)
     mu = torch.zeros(S, n, W, d, dtype=torch.float32, device=dev)
-    dbg = plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr())
+    dbg = plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr(), None, 1)
     kvd, lgd = kv.to(dev), logits.to(dev)
     pb = None if pos_begin is None else torch.tensor(pos_begin, dtype=torch.int32, device=dev)
     pe = None if pos_end is None else torch.tensor(pos_end, dtype=torch.int32, device=dev)
@@ -134,6 +134,11 @@ def check_against_oracle(orc, g, T, kv, logits, K, delta, CP, pos_begin=None, po
     stats = g["ctx"].stats()
     assert stats.payload_bytes == total_g
     assert abs(total_g / enc["stats"].payload_bytes - 1) < 1e-3
+    # the ideal code length under the coder's model, counted on the GPU over everything coded, is the
+    # oracle's (symbols differ in fewer than 1e-4 places); the bytes exceed it by the state flush only
+    ideal_o = enc["stats"].ideal_bits
+    assert abs(stats.ideal_bits - ideal_o) <= 1e-3 * ideal_o + 64
+    assert stats.ideal_bits <= 8 * total_g <= stats.ideal_bits + (1024 + 16) * stats.n_chunks + 1e-3 * ideal_o
     return enc
 
 
@@ -363,14 +368,36 @@ def test_capacity_overflow_is_reported_not_written(dev):
     tokens, logits, T, kv = make_workload(11, 1, 128, 1, 2, 128, 512, 32)
     big = gpu_encode(dev, T, kv, logits, 32, 0.02, 32)
     need = int(big["st"].total_bytes)
-    cap = need // 2
-    g = gpu_encode(dev, T, kv, logits, 32, 0.02, 32, capacity=cap + 64)
+    cap = need // 2 + 8                                            # not a multiple of 16: chunks end before it or do not fit
+    g = gpu_encode(dev, T, kv, logits, 32, 0.02, 32, capacity=cap, guard=1 << 16)
     assert g["rc"] == plc.E_CAPACITY
     assert int(g["st"].total_bytes) == need                       # the size that would have been needed
-    guard = g["st"].payload[cap:]                                  # nothing past the stated capacity ...
-    assert g["st"].payload.numel() == cap + 64
-    g["ctx"].cfg                                                   # (context stays usable)
+    assert g["st"].payload.numel() == cap + (1 << 16) and g["st"].guard_intact()   # nothing past the stated capacity
+    off = g["st"].chunk_offset.cpu().numpy().astype(np.int64); nby = g["st"].chunk_bytes.cpu().numpy().astype(np.int64)
+    fits = off + nby <= cap
+    assert fits.any() and not fits.all()
+    ref = {slot: big["st"].chunk(slot) for slot in np.nonzero(fits)[0][:50]}
+    for slot, r in ref.items():                                    # the chunks that fit are complete and correct
+        assert np.array_equal(g["st"].chunk(int(slot)), r)
     assert g["ctx"].sync_status() == plc.OK                        # status word was cleared by the read
+    assert g["ctx"].poll_status() == (plc.OK, 0)
+
+
+def test_unaligned_byte_cursor_is_reported_not_used(dev):
+    """*total_bytes_dev must be a multiple of 16 when an encoder runs: with a cursor that is not, no
+    chunk is written (a 32-bit store at such an offset would be misaligned) and the status says so."""
+    tokens, logits, T, kv = make_workload(13, 1, 64, 1, 2, 128, 512, 32)
+    L, _, H, V, d = T.shape
+    ctx = plc.Context(T.to(dev), 32, 0.02, chunk_pos=32)
+    st = plc.StreamSet(ctx.W, 2, 3 * 64 * ctx.W * d + 4096, dev)
+    st.payload.fill_(0x5A)
+    st.total_bytes.fill_(6)
+    ctx.encode(kv.to(dev), logits.to(dev), st)
+    torch.cuda.synchronize()
+    rc, bits = ctx.poll_status()
+    assert rc == plc.E_ALIGN and bits & 16
+    assert ctx.sync_status() == plc.E_ALIGN
+    assert bool((st.payload == 0x5A).all())
 
 
 def test_damaged_streams_are_reported(dev):

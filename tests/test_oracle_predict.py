@@ -180,8 +180,11 @@ def test_quantise_reconstruct_error_bound_and_idempotence(orc):
         kv = (rng.standard_normal(d) * 1.5).astype(np.float16)
         mu = rng.standard_normal(d) * 0.7
         sym = orc.quantise(kv, mu, delta)
-        ref = np.rint((kv.astype(np.float64) - mu) / delta)
-        assert (sym != ref).mean() < 0.02 and np.abs(sym - ref).max() <= 1     # only boundary cases may move
+        t = (kv.astype(np.float64) - mu) / float(np.float32(delta))
+        ref = np.rint(t)                                                       # Def. 6 + uniform quantiser, in double
+        moved = sym != ref                                                     # only exact-boundary cases may move
+        assert moved.sum() <= 1 and np.abs(sym - ref).max() <= 1
+        assert not moved.any() or np.abs(t - np.floor(t) - 0.5)[moved].max() < 1e-3
         out = orc.reconstruct(mu, sym, delta)
         assert np.abs(out.astype(np.float64) - kv.astype(np.float64)).max() <= delta / 2 + 1e-6
         # re-quantising the reconstruction (kept in float64 here) returns the same symbols

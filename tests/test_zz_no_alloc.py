@@ -51,10 +51,18 @@ def test_static_coder_matches_append_sealing_twice():
                 assert np.array_equal(out.chunk(s), ref[s]), (steps, call, s)
             assert int(out.total_bytes) == int(sb.streams.total_bytes)
         # a payload buffer that is too small is reported through the status word, nothing is overrun
-        small = plc.StreamSet(B * W, 1, 1024, dev)
+        small = plc.StreamSet(B * W, 1, 1024, dev, guard=1 << 16)
         assert plc.rans_encode_static(sym, q, steps, 0, small, status) == plc.OK
         torch.cuda.synchronize()
         assert int(status) == 1 and int(small.total_bytes) == int(sb.streams.total_bytes)
+        assert small.guard_intact()
+        # a byte cursor that is not a multiple of 16 is reported (bit 16) and nothing is written
+        odd = plc.StreamSet(B * W, 1, cap, dev)
+        odd.payload.fill_(0x5A)
+        odd.total_bytes.fill_(4)
+        assert plc.rans_encode_static(sym, q, steps, 0, odd, status) == plc.OK
+        torch.cuda.synchronize()
+        assert int(status) == 16 and bool((odd.payload == 0x5A).all())
     # sizes beyond the static working memory are refused on the host
     big_sym = torch.zeros(2, 64, 128, dtype=torch.int32, device=dev)
     big_q = torch.zeros(2, 64, dtype=torch.int32, device=dev)
