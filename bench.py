@@ -7,7 +7,13 @@ A step = one pass of the whole path over one batch: top-K softmax, fused predict
 encode of every (stream, position), then the decode of the same batch.  The metric is KV tokens per
 second (a KV token = one token position of one session across all 2*L*H streams) that were both
 encoded and decoded.  With N > 1 (torchrun) every rank runs its own batch (streams shard with no
-exchange): weak scaling, value = tokens of all ranks / slowest rank's time.
+exchange): weak scaling, value = tokens of all ranks / slowest rank's time; `--shard layers` instead
+gives rank r the layers [r L/N, (r+1) L/N) of ONE batch (strong scaling: each rank holds only its
+slice of T and of the KV tensor, the union of the ranks' chunks is the single-GPU result).
+
+The default run (no --workload, one GPU) prints the headline line for `llama2-7b` and, in its
+`configs` object, one compact record per benchmark configuration (tiny, llama2-7b, 70b-longctx top-K
+and dense, the dedup pipeline, the append path with its perplexity x step sweep).
 """
 import argparse
 import json
@@ -31,6 +37,62 @@ def measured_peaks():
     if os.path.exists(p):
         return float(json.load(open(p))["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def tensor_peak():
+    """Sustained dense bf16 TFLOP/s (the contraction is timed inside a long step)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p)).get("bf16_tflops_sustained", 1400.0)), "measured sustained bf16"
+    return 1400.0, "fallback"
+
+
+def parse_over(pairs):
+    over = {}
+    for kvs in pairs:
+        k, v = kvs.split("=")
+        over[k] = float(v) if "." in v else int(v)
+    return over
+
+
+# Issue-slot use of the fused kernels (sm__throughput) from the ncu capture summarised in
+# profiles/fused_kernels_mid_L4.md; quoted beside the roofline fraction, not part of it.
+NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.636, "decode_kernel": 0.658}
+
+
+def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None):
+    """Roofline record of the fused predict + quantise + code kernels (the slower of the two).
+    Two ceilings apply to a launch: HBM on the COMPULSORY bytes (KV once, bitstream once, every
+    table once) and the plain fp32 ALUs on the mixture's K*d fused multiply-adds per vector; the
+    fraction reported is the larger of the two (the ceiling the kernel is closer to), `bound` says
+    which.  The gathered-row accounting of the benchmark definition (K*d*2 bytes per vector) is
+    kept apart: those rows come from L1 / L2, so it is not an HBM utilisation."""
+    dom_enc = ek >= dk
+    ms = ek if dom_enc else dk
+    name = "encode_kernel" if dom_enc else "decode_kernel"
+    sec = ms / 1e3
+    bytes_c = kv_bytes + t_bytes + payload
+    hbm_frac = bytes_c / sec / 1e9 / peak
+    fma = vecs * K * d
+    flop_peak = 2.0 * sms * 128 * sm_mhz * 1e6 / 1e12            # TFLOP/s of the fp32 FMA pipes at the sampled clock
+    flop_ach = 2.0 * fma / sec / 1e12
+    alu_frac = flop_ach / flop_peak
+    bytes_ns = kv_bytes + vecs * K * d * 2 + payload
+    r = {"kernel": name, "ms_per_launch": ms, "encode_kernel_ms": ek, "decode_kernel_ms": dk,
+         "hbm_compulsory": {"bytes_per_launch": bytes_c, "achieved": bytes_c / sec / 1e9, "peak": peak, "unit": "GB/s",
+                            "frac": hbm_frac, "peak_kind": peak_kind},
+         "fp32_fma": {"achieved": flop_ach, "peak": flop_peak, "unit": "TFLOP/s", "frac": alu_frac,
+                      "peak_kind": "SMs x 128 lanes x 2 flop x sampled SM clock (%d x %.0f MHz)" % (sms, sm_mhz)},
+         "issue_slot_use_ncu": NCU_ISSUE_SLOT_USE.get(name),
+         "northstar_bytes_frac": bytes_ns / sec / 1e9 / peak,
+         "northstar_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
+                           "L1 / L2 hits, so this is an on-chip gather rate, not an HBM utilisation",
+         "traffic": None if traffic_per_vector is None else traffic_per_vector[name] * vecs}
+    if alu_frac >= hbm_frac:
+        r.update(bound="alu", achieved=flop_ach, peak=flop_peak, unit="TFLOP/s", frac=alu_frac)
+    else:
+        r.update(bound="hbm", achieved=bytes_c / sec / 1e9, peak=peak, unit="GB/s", frac=hbm_frac)
+    return r
 
 
 class ClockSampler:
@@ -77,6 +139,8 @@ class ClockSampler:
 # profiles/fused_kernels_mid_L4.md (dram__bytes_read.sum + dram__bytes_write.sum over 4.19 M vectors;
 # traffic grows in proportion to the vectors).  Valid for the default workload and chunk size only.
 NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.3, "decode_kernel": 431.9}
+NCU_TRAFFIC_NOTE = ("dram__bytes_read + dram__bytes_write of a 4-layer ncu capture (profiles/fused_kernels_mid_L4.md) "
+                    "scaled by the vectors of a launch")
 
 
 def max_over_ranks(ms, dist, device):
@@ -93,9 +157,10 @@ def job_value(world, tokens_per_rank_step, ms_per_step):
     return world * tokens_per_rank_step / (ms_per_step / 1e3)
 
 
-def oracle_sample_rate(w, positions, layers):
+def oracle_sample_rate(w, positions, layers, workers=1):
     """Times the CPU oracle (encode + decode) on a slice of the workload: `positions` positions of
-    session 0, `layers` layers, all heads.  Returns KV tokens/s (vectors / W / seconds)."""
+    session 0, `layers` layers, all heads, cut along the head axis over `workers` processes (1 = the
+    single-threaded oracle in this process).  Returns KV tokens/s (vectors / W / seconds)."""
     import oracle
     cfg = w["cfg"]
     H, d, V, K = cfg["H"], cfg["d"], cfg["V"], cfg["K"]
@@ -104,19 +169,242 @@ def oracle_sample_rate(w, positions, layers):
     lgn = w["logits"][:1, :positions].cpu().numpy()
     tkn = w["tokens"][:1, :positions].cpu().numpy()
     ocfg = oracle.Config(layers, H, d, V, K, cfg["delta"], 0.0, cfg["chunk_pos"], 0)
-    t0 = time.perf_counter()
-    enc = oracle.encode(ocfg, Tn, kvn, lgn, tkn)
-    t1 = time.perf_counter()
-    rc, out, _ = oracle.decode(ocfg, Tn, lgn, enc, kvn.shape)
-    t2 = time.perf_counter()
-    assert rc == 0
+    r = oracle.roundtrip_parallel(ocfg, Tn, kvn, lgn, tkn, workers=workers)
+    assert r["rc"] == 0 and r["max_err"] <= cfg["delta"] / 2 + 1e-3
     W_full = 2 * cfg["L"] * H
     vecs = positions * 2 * layers * H
-    return dict(value=vecs / W_full / (t2 - t0), encode=vecs / W_full / (t1 - t0), decode=vecs / W_full / (t2 - t1),
-                seconds=t2 - t0, bytes=int(enc["stats"].payload_bytes), vectors=vecs,
-                bits_per_component=8.0 * enc["stats"].payload_bytes / (vecs * d),
-                ideal_bits_per_component=enc["stats"].ideal_bits / (vecs * d),        # sum of -log2(f/M) + raw bits
-                token_bits_per_position=enc["stats"].token_bits / positions)          # sum of -log2 P(x_i | x_<i)
+    return dict(value=vecs / W_full / r["seconds"], encode=vecs / W_full / r["encode_s"], decode=vecs / W_full / r["decode_s"],
+                seconds=r["seconds"], bytes=r["payload_bytes"], vectors=vecs, workers=r["workers"],
+                bits_per_component=8.0 * r["payload_bytes"] / (vecs * d),
+                ideal_bits_per_component=r["ideal_bits"] / (vecs * d),                # sum of -log2(f/M) + raw bits
+                token_bits_per_position=r["token_bits"] / positions)                  # sum of -log2 P(x_i | x_<i)
+
+
+def cpu_baseline(w):
+    """The oracle as it stands on the host's cores: single-threaded, then one process per slice of
+    heads on every core this process may use.  Bounded samples of the same workload."""
+    import oracle
+    cfg = w["cfg"]
+    L, n, H, W = cfg["L"], cfg["n"], cfg["H"], 2 * cfg["L"] * cfg["H"]
+    layers, pos = min(L, 2), min(n, 256)
+    one = oracle_sample_rate(w, pos, layers, workers=1)
+    cores = oracle.host_cores()
+    many = oracle_sample_rate(w, pos, layers, workers=cores) if cores > 1 and H > 1 else one
+    return {"value": many["value"], "unit": UNIT, "cores": many["workers"], "kind": "oracle",
+            "host_cores": cores, "cpu_count": os.cpu_count(),
+            "sample": f"session 0, first {pos} positions, {layers} of {L} layers, all heads ({one['vectors']} vectors; "
+                      f"{many['seconds']:.1f} s encode+decode with one process per slice of heads on {many['workers']} cores, "
+                      f"{one['seconds']:.1f} s single-threaded); rate scaled by W={W} vectors per KV token",
+            "single_core": {"value": one["value"], "encode": one["encode"], "decode": one["decode"], "seconds": one["seconds"]},
+            "encode": many["encode"], "decode": many["decode"],
+            "sample_bits_per_component": one["bits_per_component"],
+            "sample_ideal_bits_per_component": one["ideal_bits_per_component"],
+            "sample_token_bits_per_position": one["token_bits_per_position"]}
+
+
+def shard_layers(L, world, rank):
+    """Layers [lo, hi) that rank codes under --shard layers (contiguous, sizes differ by at most one)."""
+    return L * rank // world, L * (rank + 1) // world
+
+
+def shard_slots(S, L, H, mc, world, rank):
+    """(session, table, chunk) index slots of the single-GPU run that this rank produces under
+    --shard layers: table = (layer*2 + kv)*H + head for the rank's own layers."""
+    lo, hi = shard_layers(L, world, rank)
+    return {(s, t, c) for s in range(S) for t in range(lo * 2 * H, hi * 2 * H) for c in range(mc)}
+
+
+def run_codec(args, torch, plc, workloads, dev, name, over, steps, warmup, dist=None, world=1, rank=0,
+              variant="topk", d_model=4096, adaptive_b0=0, zero_rate=0.0, sigma_floor=0.0, shard=None,
+              want_e2e=False, want_cpu=False, e2e_steps=2, e2e_groups=4, w=None, layers=None):
+    """Times `steps` passes (encode then decode) of workload `name` after `warmup` untimed ones and
+    returns (line, workload).  `w` reuses a workload already built; `layers` = (lo, hi) restricts the
+    run to a slice of its layers (views, nothing is copied)."""
+    import math
+    linear = variant == "linear"
+    dense = variant == "dense"
+    if w is None:
+        o = dict(over)
+        if linear:
+            o["dm"] = d_model
+        seed = 20260415 + (0 if shard else 1000 * rank)           # a sharded job codes ONE batch: same inputs on every rank
+        w = workloads.build(name, dev, seed=seed, **o)
+    cfg = dict(w["cfg"])
+    T, kv = w["T"], w["kv"]
+    if shard == "layers":
+        layers = shard_layers(cfg["L"], world, rank)
+    if layers is not None:
+        lo, hi = layers
+        T, kv = T[lo:hi], kv[lo:hi]
+        cfg["L"] = hi - lo
+    S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
+    W = 2 * L * H
+    adaptive = (adaptive_b0, 4, math.log2(cfg["pp"])) if adaptive_b0 > 0 else None
+    tok = w["tokens"] if adaptive else None
+    if linear:
+        ctx = plc.Context.linear(w["E"], w["A"], w["c"], cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                                 zero_rate_D=zero_rate, sigma_floor=sigma_floor)
+    else:
+        ctx = plc.Context(T, K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                          variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive, zero_rate_D=zero_rate,
+                          sigma_floor=sigma_floor)
+        ctx.reserve(S * n)
+    ctx.set_profiling(True)
+    mc = ctx.max_chunks(n)
+    kv_bytes = kv.numel() * 2
+    st = plc.StreamSet(S * W, mc, int(0.70 * kv_bytes) + S * W * mc * 160 + (1 << 20), dev)
+    out = torch.empty_like(kv)
+    tokens_per_step = S * n
+    count = plc.DebugBuffers(None, None, None, None, 1)               # statistics only: ideal code length of what is coded
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(warmup, 1)):
+        st.total_bytes.zero_()
+        if i == 0:
+            ctx.stats(reset=True)
+        ctx.encode(kv, w["logits"], st, tokens=tok, debug=count if i == 0 else None)
+        if i == 0:
+            first = ctx.stats(reset=True)                             # one pass with the ideal-length counter on
+        ctx.decode(st, w["logits"], out, tokens=tok)
+    barrier()
+    assert ctx.sync_status() == plc.OK, "device status after warm-up"
+    ctx.stats(reset=True)
+
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+    launches0 = plc.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * steps)]
+    for which in range(3):
+        ctx.kernel_ms(which, reset=True)                              # the log of profiled launches starts empty
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    gemm_k = []
+    for i in range(steps):
+        st.total_bytes.zero_()
+        ev[3 * i].record()
+        ctx.encode(kv, w["logits"], st, tokens=tok)
+        ev[3 * i + 1].record()
+        ctx.decode(st, w["logits"], out, tokens=tok)
+        ev[3 * i + 2].record()
+    t_end.record()
+    barrier()
+    # the library's own events around every fused-kernel launch of the region, read after it
+    ek, n_ek = ctx.kernel_ms(0)
+    dk, n_dk = ctx.kernel_ms(1)
+    if dense or linear:
+        gemm_k.append(ctx.kernel_ms(2)[0])
+    launches = plc.launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    enc_ms = [ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(steps)]
+    dec_ms = [ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(steps)]
+    assert ctx.sync_status() == plc.OK, "device status after the timed region"
+    stats = ctx.stats()
+    payload_per_step = stats.payload_bytes / steps
+    chunks_per_step = stats.n_chunks / steps
+    sched = ctx.last_schedule() if variant == "topk" else None
+
+    ms_per_step = max_over_ranks(total_ms, dist, dev) / steps
+    if shard:
+        value = tokens_per_step / (ms_per_step / 1e3)               # one batch, cut across the ranks (strong scaling)
+    else:
+        value = job_value(world, tokens_per_step, ms_per_step)
+
+    # spot check of the decoded batch (outside the timed region)
+    sel = torch.randint(0, n, (64,), device=dev)
+    err = float((out[:, :, :, :, sel].float() - kv[:, :, :, :, sel].float()).abs().max())
+    if not zero_rate:      # skipped positions are bounded in expectation only
+        assert err <= cfg["delta"] * (2.0 ** (adaptive_b0 - 1) if adaptive else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
+
+    peak, peak_kind = measured_peaks()
+    vecs = S * n * W
+    ek_last, dk_last = ek, dk
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    default_kernels = name == "llama2-7b" and not over and variant == "topk" and not adaptive and not zero_rate and \
+        not sigma_floor and layers is None
+    roofline = fused_roofline(vecs, K, d, 0 if linear else T.numel() * 2, kv_bytes, payload_per_step, ek, dk, sm_mhz, sms, peak,
+                              peak_kind, NCU_DRAM_BYTES_PER_VECTOR if default_kernels else None)
+    if roofline["traffic"] is not None:
+        roofline["traffic_note"] = NCU_TRAFFIC_NOTE
+    if dense or linear:
+        gm = statistics.mean(gemm_k)
+        tpeak, tkind = tensor_peak()
+        if dense:      # 2 * rows * V * (2H*d) flop per layer and direction
+            flop = 2.0 * S * n * V * (2 * H * d)
+        else:          # per layer: rows x (2H*d) x d_model
+            flop = 2.0 * S * n * d_model * (2 * H * d)
+        roofline = {"kernel": "dense_gemm_kernel", "bound": "tensor", "achieved": flop / (gm / 1e3) / 1e12, "peak": tpeak,
+                    "unit": "TFLOP/s", "frac": flop / (gm / 1e3) / 1e12 / tpeak, "traffic": None, "peak_kind": tkind,
+                    "ms_per_launch": gm, "flop_per_launch": flop, "launches_per_step": 2 * L,
+                    "coder_kernels_ms_last_layer": {"encode": ek_last, "decode": dk_last}}
+        if linear:
+            roofline["flop_per_step_all_contractions"] = 2 * (L * flop + 2.0 * S * n * V * d_model +
+                                                              2.0 * S * n * V * 256 * ((W + 255) // 256))
+    e2e = None
+    if want_e2e and not linear:
+        del out, st
+        torch.cuda.empty_cache()
+
+        def make_ctx(Tslice):
+            return plc.Context(Tslice, K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
+                               variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive,
+                               zero_rate_D=zero_rate, sigma_floor=sigma_floor)
+        e2e = run_e2e(torch, plc, make_ctx, dict(cfg=cfg, T=T, kv=kv, logits=w["logits"]), dev, world, dist, tokens_per_step,
+                      tok, e2e_groups if variant == "topk" else 1, e2e_steps, adaptive_b0, bool(shard))
+
+    cpu = None
+    if want_cpu and rank == 0 and not linear:
+        cpu = cpu_baseline(dict(cfg=cfg, T=T, kv=kv, logits=w["logits"], tokens=w["tokens"]))
+
+    coded_bits = 8.0 * first.payload_bytes
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if shard else "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": name, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
+                   "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
+                   "kv_dtype": "f16", "decode_out": "f16", "variant": variant, "adaptive_b0": adaptive_b0,
+                   "zero_rate_D": zero_rate, "sigma_floor": sigma_floor,
+                   "shard": ("layers %d..%d of %d on rank 0, the other ranks alike" % (*shard_layers(w["cfg"]["L"], world, 0), w["cfg"]["L"])) if shard else None,
+                   "layer_subset": list(layers) if layers is not None and not shard else None,
+                   "work_queues": None if sched is None else {"queues": sched[0], "sms_per_queue": sched[1]},
+                   "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
+        "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
+        "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),
+        "encode_ms": statistics.mean(enc_ms), "decode_ms": statistics.mean(dec_ms),
+        "bits_per_token": 8 * (payload_per_step + 12 * chunks_per_step) / tokens_per_step,
+        "bits_per_component": 8 * payload_per_step / (vecs * d),
+        "ideal_bits_per_component": first.ideal_bits / (vecs * d),
+        "ideal_note": "sum of -log2(f / 2^15) + raw bit-plane bits over every component coded in one pass (counted by "
+                      "the encode kernel): the -log2 P code length under the coder's model; coded / ideal = %.5f" %
+                      (coded_bits / max(first.ideal_bits, 1.0)),
+        "paper_bound_bits_per_token": "3.3-4.3 at perplexity 10-20 (Cor. 1: theory for the token stream, not this synthetic KV)",
+        "escapes_per_step": stats.n_escapes / steps,
+        "skipped_vector_fraction": stats.skipped_vectors / max(stats.coded_vectors, 1),
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+    }
+    return line, w
+
+
+def compact(line, keep=("value", "unit", "ms_per_step", "steps", "warmup", "encode_ms", "decode_ms", "bits_per_token",
+                        "bits_per_component", "ideal_bits_per_component", "clocks", "gpu_launches", "latency_ms", "stage_ms",
+                        "sweep", "shared_fraction", "relative_storage_vs_no_dedup", "covered_tokens_s", "extrapolated_full")):
+    """One configuration's record inside the headline line: the figures, its own roofline and clocks."""
+    r = {k: line[k] for k in keep if k in line}
+    r["config"] = {k: v for k, v in line["config"].items() if v is not None}
+    rf = line["roofline"]
+    r["roofline"] = {k: rf[k] for k in ("kernel", "bound", "achieved", "peak", "unit", "frac", "ms_per_launch", "accounting",
+                                        "encode_kernel_ms", "decode_kernel_ms") if k in rf}
+    for sub in ("hbm_compulsory", "fp32_fma"):
+        if sub in rf:
+            r["roofline"][sub + "_frac"] = rf[sub]["frac"]
+    return r
 
 
 def main():
@@ -125,7 +413,10 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
-    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--workload", default=None,
+                    help="tiny | llama2-7b | 70b-longctx | dedup | append; default: llama2-7b as the headline plus, on one "
+                         "GPU, a compact record of every benchmark configuration (see --no-configs)")
+    ap.add_argument("--no-configs", action="store_true", help="default run: headline only")
     ap.add_argument("--chunk-pos", type=int, default=None)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--e2e-groups", type=int, default=4, help="layer groups (streams) of the host-buffer step")
@@ -144,11 +435,17 @@ def main():
                     help="standard deviation added in quadrature to the mixture's before the scale class is taken")
     ap.add_argument("--zero-rate", type=float, default=0.0,
                     help="D > 0: zero-rate rule (Thm. 3), positions with mixture variance <= D carry no symbols")
+    ap.add_argument("--shard", default=None, choices=["layers"],
+                    help="with --gpus N: cut ONE batch across the ranks by layer (strong scaling) instead of one batch per rank")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    all_configs = args.workload is None and not args.no_configs and world == 1 and args.variant == "topk" and \
+        not (args.set or args.adaptive or args.rotq or args.zero_rate or args.sigma_floor or args.chunk_pos or args.shard)
+    if args.workload is None:
+        args.workload = "llama2-7b"
 
     import torch
     from paper_2604_15356_b200 import workloads
@@ -163,9 +460,11 @@ def main():
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     if args.workload == "append":
-        return append_arm(args, torch, plc, workloads, dev)
+        print(json.dumps(append_arm(args, torch, plc, workloads, dev)))
+        return 0
     if args.workload == "dedup":
-        return dedup_arm(args, torch, plc, workloads, dev)
+        print(json.dumps(dedup_arm(args, torch, plc, workloads, dev)))
+        return 0
     if args.rotq > 0:
         return rotq_arm(args, torch, plc, workloads, dev)
     dist = None
@@ -173,213 +472,74 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    over = {}
-    for kvs in args.set:
-        k, v = kvs.split("=")
-        over[k] = float(v) if "." in v else int(v)
+    over = parse_over(args.set)
     if args.chunk_pos:
         over["chunk_pos"] = args.chunk_pos
-    linear = args.variant == "linear"
-    if linear:
-        over["dm"] = args.d_model
-    w = workloads.build(args.workload, dev, seed=20260415 + 1000 * rank, **over)
-    cfg = w["cfg"]
-    S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
-    W = 2 * L * H
-    dense = args.variant == "dense"
-    import math
-    adaptive = (args.adaptive, 4, math.log2(cfg["pp"])) if args.adaptive > 0 else None
-    tok = w["tokens"] if adaptive else None
-    if linear:
-        ctx = plc.Context.linear(w["E"], w["A"], w["c"], cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                                 zero_rate_D=args.zero_rate, sigma_floor=args.sigma_floor)
-    else:
-        ctx = plc.Context(w["T"], K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                          variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive, zero_rate_D=args.zero_rate,
-                          sigma_floor=args.sigma_floor)
-        ctx.reserve(S * n)
-    ctx.set_profiling(True)
-    mc = ctx.max_chunks(n)
-    kv_bytes = w["kv"].numel() * 2
-    st = plc.StreamSet(S * W, mc, int(0.70 * kv_bytes) + (1 << 20), dev)
-    out = torch.empty_like(w["kv"])
-    tokens_per_step = S * n
-
-    def step():
-        st.total_bytes.zero_()
-        ctx.encode(w["kv"], w["logits"], st, tokens=tok)
-        ctx.decode(st, w["logits"], out, tokens=tok)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(max(args.warmup, 1)):
-        step()
-    barrier()
-    assert ctx.sync_status() == plc.OK, "device status after warm-up"
-    ctx.stats(reset=True)
-
-    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
-    sampler = ClockSampler(uuid)
-    launches0 = plc.launch_count()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * args.steps)]
-    enc_k, dec_k, gemm_k = [], [], []
-    barrier()
-    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(args.steps):
-        st.total_bytes.zero_()
-        ev[3 * i].record()
-        ctx.encode(w["kv"], w["logits"], st, tokens=tok)
-        ev[3 * i + 1].record()
-        ctx.decode(st, w["logits"], out, tokens=tok)
-        ev[3 * i + 2].record()
-        enc_k.append(ctx.last_kernel_ms(0)); dec_k.append(ctx.last_kernel_ms(1))
-        if dense or linear:
-            gemm_k.append(ctx.last_kernel_ms(2))
-    t_end.record()
-    barrier()
-    launches = plc.launch_count() - launches0
-    clocks = sampler.stop()
-    total_ms = t_start.elapsed_time(t_end)
-    enc_ms = [ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(args.steps)]
-    dec_ms = [ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(args.steps)]
-    assert ctx.sync_status() == plc.OK, "device status after the timed region"
-    stats = ctx.stats()
-    payload_per_step = stats.payload_bytes / args.steps
-    chunks_per_step = stats.n_chunks / args.steps
-
-    ms_per_step = max_over_ranks(total_ms, dist, dev) / args.steps
-    value = job_value(world, tokens_per_step, ms_per_step)
-
-    # spot check of the decoded batch (outside the timed region)
-    sel = torch.randint(0, n, (64,), device=dev)
-    err = float((out[:, :, :, :, sel].float() - w["kv"][:, :, :, :, sel].float()).abs().max())
-    if not args.zero_rate:      # skipped positions are bounded in expectation only
-        assert err <= cfg["delta"] * (2.0 ** (args.adaptive - 1) if adaptive else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
-
-    peak, peak_kind = measured_peaks()
-    vecs = S * n * W
-    ek, dk = statistics.mean(enc_k), statistics.mean(dec_k)
-    gathered = vecs * K * d * 2
-    bytes_ns = vecs * d * 2 + gathered + payload_per_step    # KV + T rows read + bitstream (either direction)
-    bytes_c = vecs * d * 2 + (0 if linear else w["T"].numel() * 2) + payload_per_step
-    dom_enc = ek >= dk
-    dom_ms = ek if dom_enc else dk
-    sm_mhz = clocks.get("sm_mhz") or 1965.0
-    sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    fma_peak = sms * 128 * sm_mhz * 1e6                      # fp32 FMA/s at the sampled clock
-    fma_ach = vecs * K * d / (dom_ms / 1e3)
-    dom_name = "encode_kernel" if dom_enc else "decode_kernel"
-    default_cfg = args.workload == "llama2-7b" and not over and not dense and not adaptive and not linear and not args.zero_rate and not args.sigma_floor
-    traffic = NCU_DRAM_BYTES_PER_VECTOR[dom_name] * vecs if default_cfg else None
-    roofline = {"kernel": dom_name, "bound": "hbm",
-                "achieved": bytes_ns / (dom_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
-                "frac": bytes_ns / (dom_ms / 1e3) / 1e9 / peak, "traffic": traffic, "peak_kind": peak_kind,
-                "traffic_note": "ncu dram bytes of a 4-layer capture scaled by vectors; far below the algorithmic bytes "
-                                "because gathered T rows are L1 / L2 hits, not HBM reads",
-                "accounting": "KV + gathered T rows (K*d*2 B per vector, mostly served by L2) + bitstream, per launch",
-                "bytes_per_launch": bytes_ns, "ms_per_launch": dom_ms,
-                "compulsory": {"bytes_per_launch": bytes_c, "achieved": bytes_c / (dom_ms / 1e3) / 1e9,
-                               "frac": bytes_c / (dom_ms / 1e3) / 1e9 / peak},
-                "fp32_fma": {"achieved_gfma_s": fma_ach / 1e9, "peak_gfma_s": fma_peak / 1e9, "frac": fma_ach / fma_peak},
-                "encode_kernel_ms": ek, "decode_kernel_ms": dk}
-
-    if dense:
-        # the contraction dominates: 2 * rows * V * (2H*d) flop per layer and direction
-        gm = statistics.mean(gemm_k)
-        flop = 2.0 * S * n * V * (2 * H * d)
-        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
-        tpeak = float(pk.get("bf16_tflops_sustained", 1400.0))
-        roofline = {"kernel": "dense_gemm_kernel", "bound": "tensor", "achieved": flop / (gm / 1e3) / 1e12, "peak": tpeak,
-                    "unit": "TFLOP/s", "frac": flop / (gm / 1e3) / 1e12 / tpeak, "traffic": None,
-                    "peak_kind": "measured sustained bf16" if pk else "fallback", "ms_per_launch": gm,
-                    "flop_per_launch": flop, "launches_per_step": 2 * L,
-                    "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
-    if linear:
-        # per layer: rows x (2H*d) x d_model; once per call: rows x d_model x V (Ebar) and rows x (L*2H) x V (variance)
-        gm = statistics.mean(gemm_k)
-        dm = args.d_model
-        flop = 2.0 * S * n * dm * (2 * H * d)
-        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
-        tpeak = float(pk.get("bf16_tflops_sustained", 1400.0))
-        roofline = {"kernel": "dense_gemm_kernel", "bound": "tensor", "achieved": flop / (gm / 1e3) / 1e12, "peak": tpeak,
-                    "unit": "TFLOP/s", "frac": flop / (gm / 1e3) / 1e12 / tpeak, "traffic": None,
-                    "peak_kind": "measured sustained bf16" if pk else "fallback", "ms_per_launch": gm,
-                    "flop_per_launch": flop, "launches_per_step": 2 * L,
-                    "flop_per_step_all_contractions": 2 * (L * flop + 2.0 * S * n * V * dm + 2.0 * S * n * V * 256 * ((W + 255) // 256)),
-                    "coder_kernels_ms_last_layer": {"encode": ek, "decode": dk}}
-    e2e = None
-    if not args.no_e2e and not linear:
-        del out, st
+    line, w = run_codec(args, torch, plc, workloads, dev, args.workload, over, args.steps, args.warmup, dist, world, rank,
+                        variant=args.variant, d_model=args.d_model, adaptive_b0=args.adaptive, zero_rate=args.zero_rate,
+                        sigma_floor=args.sigma_floor, shard=args.shard, want_e2e=not args.no_e2e,
+                        want_cpu=world == 1 and not args.no_cpu_baseline, e2e_steps=args.e2e_steps, e2e_groups=args.e2e_groups)
+    if all_configs:
+        del w
         torch.cuda.empty_cache()
-
-        def make_ctx(Tslice):
-            return plc.Context(Tslice, K, cfg["delta"], chunk_pos=cfg["chunk_pos"], out_dtype=plc.OUT_F16,
-                               variant=plc.PRED_DENSE if dense else plc.PRED_TOPK, adaptive=adaptive,
-                               zero_rate_D=args.zero_rate, sigma_floor=args.sigma_floor)
-        e2e = run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok, args.e2e_groups)
-
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not linear:
-        layers, pos = min(L, 2), min(n, 256)
-        r = oracle_sample_rate(w, pos, layers)
-        cpu = {"value": r["value"], "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"session 0, first {pos} positions, {layers} of {L} layers, all heads ({r['vectors']} vectors, "
-                         f"{r['seconds']:.1f} s encode+decode); rate scaled by W={W} vectors per KV token",
-               "encode": r["encode"], "decode": r["decode"],
-               "sample_bits_per_component": r["bits_per_component"],
-               "sample_ideal_bits_per_component": r["ideal_bits_per_component"],
-               "sample_token_bits_per_position": r["token_bits_per_position"]}
-
+        line["configs"] = every_config(args, torch, plc, workloads, dev, line)
     if rank == 0:
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
-                       "delta": cfg["delta"], "chunk_pos": cfg["chunk_pos"], "perplexity": cfg["pp"],
-                       "kv_dtype": "f16", "decode_out": "f16", "variant": args.variant, "adaptive_b0": args.adaptive, "zero_rate_D": args.zero_rate, "sigma_floor": args.sigma_floor,
-                       "l2": "inputs larger than L2 (KV+logits %.1f GB per step)" % ((kv_bytes + w["logits"].numel() * 2) / 1e9)},
-            "encode_tokens_s": tokens_per_step / (statistics.mean(enc_ms) / 1e3),
-            "decode_tokens_s": tokens_per_step / (statistics.mean(dec_ms) / 1e3),
-            "encode_ms": statistics.mean(enc_ms), "decode_ms": statistics.mean(dec_ms),
-            "bits_per_token": 8 * (payload_per_step + 12 * chunks_per_step) / tokens_per_step,
-            "bits_per_component": 8 * payload_per_step / (vecs * d),
-            "paper_bound_bits_per_token": "3.3-4.3 at perplexity 10-20 (Cor. 1: theory for the token stream, not this synthetic KV)",
-            "escapes_per_step": stats.n_escapes / args.steps,
-            "skipped_vector_fraction": stats.skipped_vectors / max(stats.coded_vectors, 1),
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-        }
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     return 0
 
 
-def append_arm(args, torch, plc, workloads, dev):
-    """Decode-time append: B sessions grow by one token per plc_append_step; per-step latency.
-    `--steps` counts groups of 32 append steps (one chunk seal per group)."""
-    from paper_2604_15356_b200 import synth
-    over = {}
-    for kvs in args.set:
-        k, v = kvs.split("=")
-        over[k] = float(v) if "." in v else int(v)
-    cfg = dict(workloads.CONFIGS["append"]); cfg.update(over)
+def every_config(args, torch, plc, workloads, dev, headline):
+    """One compact record per benchmark configuration, measured in this same process after the
+    headline (inputs regenerated per configuration; device memory is released in between)."""
+    import gc
+    out = {"llama2-7b": compact(headline)}
+
+    def free():
+        gc.collect()
+        torch.cuda.empty_cache()
+
+    t0 = time.perf_counter()
+    line, w = run_codec(args, torch, plc, workloads, dev, "tiny", {}, 20, 5)
+    out["tiny"] = compact(line)
+    out["tiny"]["note"] = "1024 vectors: two kernel launches of a few microseconds of work each; launch-latency bound"
+    del w; free()
+    # 70B long context: top-K over all 80 layers, then the full-vocabulary contraction on 4 of the 80 layers
+    line, w = run_codec(args, torch, plc, workloads, dev, "70b-longctx", {}, 3, 3)
+    out["70b-longctx topk"] = compact(line)
+    Lfull, sub = w["cfg"]["L"], 4
+    line, _ = run_codec(args, torch, plc, workloads, dev, "70b-longctx", {}, 2, 3, variant="dense", w=w, layers=(0, sub))
+    r = compact(line)
+    r["extrapolated_full"] = {"layers": Lfull, "ms_per_step": line["ms_per_step"] * Lfull / sub,
+                              "value": line["value"] * sub / Lfull,
+                              "note": "the layers are independent launches of the same shapes: time scales by %d / %d" % (Lfull, sub)}
+    out["70b-longctx dense (4 of 80 layers)"] = r
+    del w; free()
+    a = argparse.Namespace(**vars(args)); a.steps, a.warmup, a.set = 2, 1, []
+    out["dedup"] = compact(dedup_arm(a, torch, plc, workloads, dev))
+    free()
+    a = argparse.Namespace(**vars(args)); a.steps, a.set = 17, []
+    out["append"] = compact(append_arm(a, torch, plc, workloads, dev, sweep=True))
+    free()
+    out["seconds_for_the_other_configs"] = time.perf_counter() - t0
+    return out
+
+
+def append_run(torch, plc, synth, dev, cfg, T, nsteps, seed, pp=None, delta=None, zero_clock=True):
+    """One run of the append path: B sessions grow by one token per plc_append_step for nsteps steps
+    (the first chunk's steps are warm-up).  Returns latencies (ms, sorted), seal-step latencies, stats."""
     B, L, H, d, V, K, CP = cfg["S"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"], cfg["chunk_pos"]
-    nsteps = CP * max(args.steps, 1)
+    pp = cfg["pp"] if pp is None else pp
+    delta = cfg["delta"] if delta is None else delta
     W = 2 * L * H
-    seed = 20260419
-    table = synth.markov_table(V, cfg["pp"], seed, device=dev)
+    table = synth.markov_table(V, pp, seed, device=dev)
     tokens = synth.sample_tokens(table, B, nsteps, seed + 1)
     logits = synth.position_logits(table, tokens)                       # [B][nsteps][V]
-    T = synth.make_tables(L, H, V, d, seed + 2, device=dev)
-    ctx = plc.Context(T, K, cfg["delta"], chunk_pos=CP)
-    sb = ctx.new_session_batch(B, nsteps // CP + 1, int(nsteps * B * W * d * 1.4) + (1 << 20))
+    del table
+    ctx = plc.Context(T, K, delta, chunk_pos=CP)
+    sb = ctx.new_session_batch(B, nsteps // CP + 1, int(nsteps * B * W * d * 1.45) + (1 << 20))
     g = torch.Generator(device=dev); g.manual_seed(seed + 3)
-    lat = []
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nsteps)]
     launches0 = plc.launch_count()
     for i in range(nsteps):
@@ -396,24 +556,57 @@ def append_arm(args, torch, plc, workloads, dev):
     lat = sorted(a.elapsed_time(b) for a, b in ev[CP:])                 # first chunk = warm-up
     seal = sorted(ev[i][0].elapsed_time(ev[i][1]) for i in range(CP, nsteps) if (i + 1) % CP == 0)
     st = ctx.stats()
+    return dict(lat=lat, seal=seal, stats=st, launches=plc.launch_count() - launches0, W=W,
+                bits_per_token=8 * (st.payload_bytes + 12 * st.n_chunks) / max(st.coded_vectors / W, 1),
+                bits_per_component=8 * st.payload_bytes / max(st.coded_vectors * d, 1))
+
+
+def append_arm(args, torch, plc, workloads, dev, sweep=False):
+    """Decode-time append: B sessions grow by one token per plc_append_step; per-step latency.
+    `--steps` counts groups of chunk_pos append steps (one chunk seal per group); the first group is
+    warm-up.  With sweep=True the perplexity x step grid of the streaming configuration is added
+    (p50 / p99 latency and bits per component of every cell)."""
+    from paper_2604_15356_b200 import synth
+    cfg = dict(workloads.CONFIGS["append"]); cfg.update(parse_over(args.set))
+    B, L, H, d, V, K, CP = cfg["S"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"], cfg["chunk_pos"]
+    nsteps = CP * max(args.steps, 2)
+    seed = 20260419
+    T = synth.make_tables(L, H, V, d, seed + 2, device=dev)
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+    r = append_run(torch, plc, synth, dev, cfg, T, nsteps, seed)
+    clocks = sampler.stop()
+    lat, seal, W = r["lat"], r["seal"], r["W"]
     mean_ms = sum(lat) / len(lat)
     peak, kind = measured_peaks()
     gathered = B * W * K * d * 2
+    p50 = lat[len(lat) // 2]
     line = {"metric": METRIC, "value": B / (mean_ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": nsteps - CP, "warmup": CP,
             "ms_per_step": mean_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": "append", "B": B, "L": L, "H": H, "d": d, "V": V, "K": K, "delta": cfg["delta"],
-                       "chunk_pos": CP, "perplexity": cfg["pp"], "encode_only": True},
-            "latency_ms": {"p50": lat[len(lat) // 2], "p99": lat[int(len(lat) * 0.99)], "max": lat[-1],
+                       "chunk_pos": CP, "perplexity": cfg["pp"], "encode_only": True,
+                       "l2": "random rows of a %.1f GB table set, larger than L2" % (T.numel() * 2 / 1e9)},
+            "latency_ms": {"p50": p50, "p99": lat[int(len(lat) * 0.99)], "max": lat[-1],
                            "seal_steps_mean": sum(seal) / max(len(seal), 1)},
-            "bits_per_token": 8 * (st.payload_bytes + 12 * st.n_chunks) / max(st.coded_vectors / W, 1),
-            "roofline": {"kernel": "append_quantise_kernel", "bound": "hbm", "achieved": gathered / (lat[len(lat) // 2] / 1e3) / 1e9,
-                         "peak": peak, "unit": "GB/s", "frac": gathered / (lat[len(lat) // 2] / 1e3) / 1e9 / peak,
-                         "traffic": None, "peak_kind": kind,
-                         "accounting": "random 256-byte T rows per step (B*W*K*d*2 bytes) over the median whole-step time"},
-            "gpu_launches": plc.launch_count() - launches0}
-    print(json.dumps(line))
-    return 0
+            "bits_per_token": r["bits_per_token"], "bits_per_component": r["bits_per_component"],
+            "roofline": {"kernel": "append_quantise_kernel", "bound": "hbm", "achieved": gathered / (p50 / 1e3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": gathered / (p50 / 1e3) / 1e9 / peak,
+                         "traffic": None, "peak_kind": kind, "ms_per_launch": p50,
+                         "accounting": "random 256-byte T rows per step (B*W*K*d*2 bytes, tables far larger than L2: every "
+                                       "row is an HBM read) over the median whole-step time"},
+            "gpu_launches": r["launches"], "clocks": clocks}
+    if sweep:
+        grid = {}
+        for pp in (4.0, 12.0, 20.0, 50.0):
+            for delta in (0.005, 0.02, 0.08):
+                rr = append_run(torch, plc, synth, dev, cfg, T, CP * 9, seed + int(pp), pp=pp, delta=delta)
+                l2 = rr["lat"]
+                grid["pp=%g delta=%g" % (pp, delta)] = {"p50_ms": l2[len(l2) // 2], "p99_ms": l2[int(len(l2) * 0.99)],
+                                                         "bits_per_component": rr["bits_per_component"],
+                                                         "bits_per_token": rr["bits_per_token"]}
+        line["sweep"] = grid
+    return line
 
 
 def dedup_arm(args, torch, plc, workloads, dev):
@@ -425,11 +618,7 @@ def dedup_arm(args, torch, plc, workloads, dev):
     timed (CUDA events around them); the synthetic inputs of a batch are generated between them.
     `--steps` repeats the whole pipeline; the first `--warmup` repetitions are not counted."""
     from paper_2604_15356_b200 import synth
-    over = {}
-    for kvs in args.set:
-        k, v = kvs.split("=")
-        over[k] = float(v) if "." in v else int(v)
-    cfg = dict(workloads.CONFIGS["llama3-8b-dedup"]); cfg.update(over)
+    cfg = dict(workloads.CONFIGS["llama3-8b-dedup"]); cfg.update(parse_over(args.set))
     S, n, L, H, d, V, K, CP = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"], cfg["chunk_pos"]
     Sb = int(cfg.get("Sb", 8))
     assert S % Sb == 0
@@ -450,6 +639,7 @@ def dedup_arm(args, torch, plc, workloads, dev):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     reps, stats_keep = [], None
     launches0 = plc.launch_count()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
     for rep in range(args.warmup + args.steps):
         t = {"logp2": 0.0, "dedup": 0.0, "encode": 0.0, "decode": 0.0}
         spans = []
@@ -492,6 +682,7 @@ def dedup_arm(args, torch, plc, workloads, dev):
             reps.append(t)
             stats_keep = ctx.stats()
     launches = plc.launch_count() - launches0
+    clocks = sampler.stop()
     mean = {k: sum(r[k] for r in reps) / len(reps) for k in reps[0]}
     total_ms = sum(mean.values())
     sh = shared.cpu().numpy().astype("int64")
@@ -500,7 +691,7 @@ def dedup_arm(args, torch, plc, workloads, dev):
     logits_bytes = 2.0 * S * n * V
     line = {"metric": METRIC, "value": coded / (total_ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
+            "dtype": "f32", "data": "synthetic", "encode_ms": mean["encode"], "decode_ms": mean["decode"],
             "config": {"workload": "dedup (llama3-8b-dedup shapes)", "S": S, "n": n, "L": L, "H": H, "d": d, "V": V, "K": K,
                        "delta": cfg["delta"], "chunk_pos": CP, "perplexity": cfg["pp"], "session_batch": Sb,
                        "prefix_trie": "15 segments of U[%d,%d] tokens, 8 leaves" % (seg_lo, seg_hi),
@@ -515,22 +706,21 @@ def dedup_arm(args, torch, plc, workloads, dev):
             "relative_storage_vs_no_dedup": coded / float(S * n),
             "roofline": {"kernel": "topk_softmax_kernel", "bound": "hbm", "achieved": logits_bytes / (mean["logp2"] / 1e3) / 1e9,
                          "peak": peak, "unit": "GB/s", "frac": logits_bytes / (mean["logp2"] / 1e3) / 1e9 / peak,
-                         "traffic": None, "peak_kind": kind,
+                         "traffic": None, "peak_kind": kind, "ms_per_launch": mean["logp2"] / (S // Sb),
                          "accounting": "logits read once (2*S*n*V bytes) over the summed log2 P launches; the encode and "
                                        "decode calls scan the logits of the coded positions once more each"},
-            "gpu_launches": launches}
-    print(json.dumps(line))
-    return 0
+            "gather_rate": {"achieved": stats_keep.coded_vectors * K * d * 2 / (max(mean["encode"], mean["decode"]) / 1e3) / 1e9,
+                            "peak": peak, "unit": "GB/s",
+                            "note": "K*d*2 B of random T rows per coded vector over the slower of encode / decode; the "
+                                    "tables in flight are far beyond L2 here, so these rows are HBM reads"},
+            "gpu_launches": launches, "clocks": clocks}
+    return line
 
 
 def rotq_arm(args, torch, plc, workloads, dev):
     """Predict, rotate and quantise the residual to `--rotq` bits per component (fixed-size records),
     then decode; same workloads, same prediction kernels, no entropy coder."""
-    over = {}
-    for kvs in args.set:
-        k, v = kvs.split("=")
-        over[k] = float(v) if "." in v else int(v)
-    w = workloads.build(args.workload, dev, seed=20260415, **over)
+    w = workloads.build(args.workload, dev, seed=20260415, **parse_over(args.set))
     cfg = w["cfg"]
     S, n, L, H, d, V, K = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"], cfg["V"], cfg["K"]
     W = 2 * L * H
@@ -581,14 +771,15 @@ def rotq_arm(args, torch, plc, workloads, dev):
     return 0
 
 
-def run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None, groups=4):
+def run_e2e(torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None, groups=4, e2e_steps=2, adaptive_b0=0,
+            sharded=False):
     """Same step with HOST buffers: pinned inputs are copied in, the coded bytes and index are
     copied out and back in, the decoded KV is copied out -- all inside the timed region.  The
     layers are cut into groups, each with its own context and CUDA stream, so that the copies of
     one group overlap the kernels and the opposite-direction copies of the others."""
     cfg = w["cfg"]
     S, n, L, H, d = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"]
-    G = groups if (L % groups == 0 and args.variant == "topk") else 1
+    G = groups if L % groups == 0 else 1
     Lg = L // G
     kv_h = w["kv"].cpu().pin_memory()
     lg_h = w["logits"].cpu().pin_memory()
@@ -642,21 +833,22 @@ def run_e2e(args, torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, to
     for c in ctxs:
         assert c.sync_status() == plc.OK
     err = float((kvo_h[:, :, :, :, :64].float() - kv_h[:, :, :, :, :64].float()).abs().max())
-    assert err <= cfg["delta"] * (2.0 ** (args.adaptive - 1) if args.adaptive > 0 else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
+    assert err <= cfg["delta"] * (2.0 ** (adaptive_b0 - 1) if adaptive_b0 > 0 else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(args.e2e_steps):
+    for _ in range(e2e_steps):
         used = step()
     t1.record()
     torch.cuda.synchronize()
-    ms = max_over_ranks(t0.elapsed_time(t1) / args.e2e_steps, dist, dev)
+    ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps, dist, dev)
     idx_bytes = sum(o.numel() * 8 + b.numel() * 4 for o, b in zip(off_h, nby_h))
-    return {"value": job_value(world, tokens_per_step, ms), "unit": UNIT, "ms_per_step": ms,
+    return {"value": tokens_per_step / (ms / 1e3) if sharded else job_value(world, tokens_per_step, ms), "unit": UNIT,
+            "ms_per_step": ms,
             "h2d_bytes_per_step": kv_h.numel() * 2 + lg_h.numel() * 2 + used + idx_bytes,
-            "d2h_bytes_per_step": used + idx_bytes + 8 * G + kvo_h.numel() * 2, "steps": args.e2e_steps,
+            "d2h_bytes_per_step": used + idx_bytes + 8 * G + kvo_h.numel() * 2, "steps": e2e_steps,
             "layer_groups": G}
 
 
@@ -667,12 +859,14 @@ def reference_arm(args, workloads):
     # the sample is built on the CPU at the sample's own size (same recipe)
     w = workloads.build(args.workload, "cpu", seed=20260415, S=1, n=pos, L=layers, max_states=64)
     w["cfg"]["L"] = cfg["L"]                                  # the rate is scaled to the full number of streams
+    import oracle
+    cores = oracle.host_cores()
     for _ in range(min(args.warmup, 1)):
         oracle_sample_rate(w, pos, layers)
     rates = []
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        rates.append(oracle_sample_rate(w, pos, layers))
+        rates.append(oracle_sample_rate(w, pos, layers, workers=cores if cfg["H"] > 1 else 1))
     dt = (time.perf_counter() - t0) / max(args.steps, 1)
     value = statistics.mean(r["value"] for r in rates)
     W = 2 * cfg["L"] * cfg["H"]
@@ -682,7 +876,8 @@ def reference_arm(args, workloads):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": args.workload, "sample": sample},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": rates[0]["workers"], "host_cores": cores,
+                             "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))

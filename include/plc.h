@@ -357,6 +357,11 @@ plc_status plc_set_profiling(plc_ctx* ctx, int32_t on);
  * tests and benchmarks that must state which path they ran.  PLC_E_STATE before the first such call. */
 plc_status plc_last_schedule(const plc_ctx* ctx, int32_t* n_queues, int32_t* sms_per_queue);
 plc_status plc_last_kernel_ms(plc_ctx* ctx, int32_t which, float* ms);
+/* Every profiled launch since the last reset keeps its event pair (up to 4096 per kind; further
+ * launches overwrite the newest).  Waits for them and returns their mean duration and their number
+ * (each optional); reset != 0 then empties the log of that kind.  Meant to be called outside a
+ * timed region: it synchronises with the recorded events. */
+plc_status plc_kernel_ms(plc_ctx* ctx, int32_t which, float* mean_ms, int32_t* launches, int32_t reset);
 /* Number of kernels this library has launched in this process (for benchmarks). */
 uint64_t plc_launch_count(void);
 

@@ -396,3 +396,112 @@ def decode(cfg, T, logits, enc, kv_shape, pos_begin=None, pos_end=None, export=F
     rc = lib().plo_decode(C.byref(cfg), _p(Tb), _p(lg), _p(tk), S, n, _p(pb), _p(pe), enc["max_chunks"], _p(enc["payload"]),
                           _p(off), _p(nby), _p(out), C.byref(st), _p(sym))
     return rc, out, sym
+
+
+# ---------------------------------------------------------------------------------------------
+# The same oracle on several host cores.  Streams are independent across heads (nothing couples
+# them in the codec), so the whole-path encode is cut along the head axis, every slice is coded by
+# the unchanged single-threaded `encode` in a process of its own, and the exports are put back
+# together.  Processes are started with "spawn": a fork after the parent has touched CUDA hangs.
+
+def host_cores():
+    """Cores this process may run on."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def _config_fields(cfg):
+    return [getattr(cfg, name) for name, _ in Config._fields_]
+
+
+def _encode_slice(job):
+    fields, T, kv, logits, tokens, pos_begin, pos_end, export, linear = job
+    if linear is not None:
+        E, A, c = linear
+        L, _, H, d, dm = A.shape
+        cfg = linear_config(L, H, d, fields[3], fields[4], fields[5], fields[7], E, A, c)
+        cfg.zero_D = fields[16]
+    else:
+        cfg = Config(*fields[:12], 0, None, None, None, fields[16])
+        cfg.H = T.shape[2]
+    enc = encode(cfg, T, kv, logits, tokens, pos_begin, pos_end, export=export)
+    st = enc["stats"]
+    stats = {name: getattr(st, name) for name, _ in Stats._fields_}
+    return dict(sym=enc["sym"], q=enc["q"], mu=enc["mu"], bits=enc["bits"], stats=stats,
+                chunk_bytes=enc["chunk_bytes"])
+
+
+def encode_parallel(cfg, T, kv, logits, tokens=None, pos_begin=None, pos_end=None, export=False, workers=None, linear=None):
+    """`encode` cut along the head axis over `workers` processes (default: the host's cores).
+    linear = (E, A, c) for the linear-embedding predictor (then T is None).  Returns the merged
+    exports (sym / q / mu as [S,n,L,2,H(,d)]), chunk_bytes [S,L,2,H,max_chunks], a dict of summed
+    statistics, and the number of processes used; payload bytes are not kept."""
+    import multiprocessing as mp
+    H = cfg.H
+    workers = max(1, min(H, workers or host_cores()))
+    bounds = [(H * k // workers, H * (k + 1) // workers) for k in range(workers)]
+    fields = _config_fields(cfg)
+    jobs = []
+    for lo, hi in bounds:
+        Ts = None if T is None else np.ascontiguousarray(T[:, :, lo:hi])
+        kvs = np.ascontiguousarray(kv[:, :, :, lo:hi])
+        lin = None if linear is None else (linear[0], np.ascontiguousarray(linear[1][:, :, lo:hi]),
+                                           np.ascontiguousarray(linear[2][:, :, lo:hi]))
+        jobs.append((fields, Ts, kvs, logits, tokens, pos_begin, pos_end, export, lin))
+    if workers == 1:
+        parts = [_encode_slice(jobs[0])]
+    else:
+        with mp.get_context("spawn").Pool(workers) as pool:
+            parts = pool.map(_encode_slice, jobs)
+    out = dict(workers=workers, bits=parts[0]["bits"])
+    out["chunk_bytes"] = np.concatenate([p["chunk_bytes"] for p in parts], axis=3)
+    if export:
+        out["sym"] = np.concatenate([p["sym"] for p in parts], axis=4)
+        out["q"] = np.concatenate([p["q"] for p in parts], axis=4)
+        out["mu"] = np.concatenate([p["mu"] for p in parts], axis=4)
+    stats = {k: sum(p["stats"][k] for p in parts) for k in parts[0]["stats"]}
+    stats["token_bits"] = parts[0]["stats"]["token_bits"]          # a property of the positions, not of the heads
+    stats["coded_positions"] = parts[0]["stats"]["coded_positions"]
+    out["stats"] = stats
+    return out
+
+
+def _roundtrip_slice(job):
+    import time
+    fields, T, kv, logits, tokens = job
+    cfg = Config(*fields[:12], 0, None, None, None, fields[16])
+    cfg.H = T.shape[2]
+    t0 = time.perf_counter()
+    enc = encode(cfg, T, kv, logits, tokens)
+    t1 = time.perf_counter()
+    rc, out, _ = decode(cfg, T, logits, enc, kv.shape, tokens=tokens if cfg.adaptive_b0 > 0 else None)
+    t2 = time.perf_counter()
+    st = enc["stats"]
+    return dict(rc=rc, encode_s=t1 - t0, decode_s=t2 - t1, payload_bytes=int(st.payload_bytes), ideal_bits=float(st.ideal_bits),
+                token_bits=float(st.token_bits), max_err=float(np.abs(out - kv.astype(np.float32)).max()))
+
+
+def roundtrip_parallel(cfg, T, kv, logits, tokens=None, workers=None):
+    """Encode then decode, cut along the head axis over `workers` processes; every process times
+    its own two calls.  Returns the slowest process's times (the job's time with one process per
+    slice), the summed statistics and the number of processes."""
+    import multiprocessing as mp
+    H = cfg.H
+    workers = max(1, min(H, workers or host_cores()))
+    fields = _config_fields(cfg)
+    jobs = []
+    for k in range(workers):
+        lo, hi = H * k // workers, H * (k + 1) // workers
+        jobs.append((fields, np.ascontiguousarray(T[:, :, lo:hi]), np.ascontiguousarray(kv[:, :, :, lo:hi]), logits, tokens))
+    if workers == 1:
+        parts = [_roundtrip_slice(jobs[0])]
+    else:
+        with mp.get_context("spawn").Pool(workers) as pool:
+            parts = pool.map(_roundtrip_slice, jobs)
+    return dict(workers=workers, rc=max(p["rc"] for p in parts),
+                encode_s=max(p["encode_s"] for p in parts), decode_s=max(p["decode_s"] for p in parts),
+                seconds=max(p["encode_s"] + p["decode_s"] for p in parts),
+                payload_bytes=sum(p["payload_bytes"] for p in parts), ideal_bits=sum(p["ideal_bits"] for p in parts),
+                token_bits=parts[0]["token_bits"], max_err=max(p["max_err"] for p in parts))

@@ -24,7 +24,7 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
            "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters", "plc_rotq_record_bytes", "plc_encode_rotq",
-           "plc_decode_rotq", "plc_poll_status", "plc_last_schedule"]
+           "plc_decode_rotq", "plc_poll_status", "plc_last_schedule", "plc_kernel_ms"]
 
 
 def sources():
@@ -324,6 +324,12 @@ class Context:
         ms = C.c_float()
         _check(lib().plc_last_kernel_ms(self._h, int(which), C.byref(ms)), "plc_last_kernel_ms")
         return ms.value
+
+    def kernel_ms(self, which, reset=False):
+        """(mean duration in ms, launches) of the profiled launches of one kind since the last reset."""
+        ms, cnt = C.c_float(), C.c_int32()
+        _check(lib().plc_kernel_ms(self._h, int(which), C.byref(ms), C.byref(cnt), int(reset)), "plc_kernel_ms")
+        return ms.value, cnt.value
 
     def stats(self, reset=False):
         s = Stats()

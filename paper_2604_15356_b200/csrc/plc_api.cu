@@ -1,6 +1,7 @@
 // C ABI of libplc (see include/plc.h): argument checks, context scratch, kernel launches.
 #include <atomic>
 #include <new>
+#include <vector>
 
 #include "plc_common.cuh"
 #include <cmath>
@@ -36,9 +37,30 @@ struct plc_ctx {
     size_t lin_off[2];
     int last_nq, last_g;            // work-queue layout of the most recent top-K encode / decode launch
     int profiling;                  // record events around the codec kernels
-    cudaEvent_t ev[6];              // encode start/stop, decode start/stop, dense contraction start/stop
-    int ev_valid[3];
+    // Event pairs (start, stop) of the profiled launches since the last reset, per kind: 0 encode
+    // kernel, 1 decode kernel, 2 tensor-core contraction.  Events are created on demand and reused.
+    std::vector<cudaEvent_t> prof_ev[3];
+    int prof_used[3];               // pairs in use
 };
+
+namespace {
+constexpr int kMaxProfPairs = 4096;
+
+// Next event pair of a kind (the newest pair is reused once the log is full); null when profiling is off.
+cudaEvent_t* prof_pair(plc_ctx* c, int which) {
+    if (!c->profiling) return nullptr;
+    std::vector<cudaEvent_t>& v = c->prof_ev[which];
+    if (c->prof_used[which] == kMaxProfPairs) c->prof_used[which] -= 1;
+    const int i = c->prof_used[which];
+    while ((int)v.size() < 2 * (i + 1)) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        v.push_back(e);
+    }
+    c->prof_used[which] = i + 1;
+    return &v[2 * i];
+}
+}  // namespace
 
 namespace {
 
@@ -214,7 +236,6 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
         ok = cudaMalloc(&c->lin_model, bytes) == cudaSuccess &&
              linear_prepare(c->lin_E, c->lin_A, c->lin_c, sh, c->lin_model, c->lin_off, c->status, 0) == cudaSuccess;
     }
-    for (int i = 0; i < 6 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
     if (!ok) { plc_destroy(c); return PLC_E_CUDA; }
     *out = c;
     return PLC_OK;
@@ -224,7 +245,8 @@ plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
     cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->step_exp); cudaFree(c->staging);
     cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch); cudaFree(c->lin_model);
-    for (int i = 0; i < 6; ++i) if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (int k = 0; k < 3; ++k)
+        for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->poll_stream) cudaStreamDestroy(c->poll_stream);
     delete c;
@@ -293,15 +315,14 @@ static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, boo
     a.mu_ld = sh.ncols; a.s1_ld = sh.tables;
     const size_t layer_elems = (size_t)sh.tables * sh.V * sh.d;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-        const bool prof = c->profiling != 0;
-        if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st, prof ? c->ev[4] : nullptr,
-                        prof ? c->ev[5] : nullptr) != cudaSuccess) return PLC_E_CUDA;
-        if (prof) c->ev_valid[2] = 1;
+        cudaEvent_t* pg = prof_pair(c, 2);
+        if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st, pg ? pg[0] : nullptr,
+                        pg ? pg[1] : nullptr) != cudaSuccess) return PLC_E_CUDA;
         a.dense_layer = l;
-        const int w = encode ? 0 : 1;
-        if (prof) cudaEventRecord(c->ev[2 * w], st);
+        cudaEvent_t* pk = prof_pair(c, encode ? 0 : 1);
+        if (pk) cudaEventRecord(pk[0], st);
         if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;
-        if (prof) { cudaEventRecord(c->ev[2 * w + 1], st); c->ev_valid[w] = 1; }
+        if (pk) cudaEventRecord(pk[1], st);
     }
     return PLC_OK;
 }
@@ -317,17 +338,16 @@ static plc_status run_linear(plc_ctx* c, CodecArgs a, const void* logits_dev, bo
     a.mu_dense = reinterpret_cast<const float*>(c->dense_scratch + off[5]);
     a.mu_ld = sh.ncols; a.s1_ld = sh.nt_all;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-        const bool prof = c->profiling != 0;
+        cudaEvent_t* pg = prof_pair(c, 2);
         if (linear_layer(c->lin_A + (size_t)l * sh.ncols * sh.dm, sh, c->dense_scratch, off, c->status, st,
-                         prof ? c->ev[4] : nullptr, prof ? c->ev[5] : nullptr) != cudaSuccess) return PLC_E_CUDA;
-        if (prof) c->ev_valid[2] = 1;
+                         pg ? pg[0] : nullptr, pg ? pg[1] : nullptr) != cudaSuccess) return PLC_E_CUDA;
         a.dense_layer = l;
         a.s1_dense = reinterpret_cast<const float*>(c->dense_scratch + off[3]) + (size_t)l * sh.tables;
         a.mu_bias = c->lin_c + (size_t)l * sh.ncols;
-        const int w = encode ? 0 : 1;
-        if (prof) cudaEventRecord(c->ev[2 * w], st);
+        cudaEvent_t* pk = prof_pair(c, encode ? 0 : 1);
+        if (pk) cudaEventRecord(pk[0], st);
         if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;
-        if (prof) { cudaEventRecord(c->ev[2 * w + 1], st); c->ev_valid[w] = 1; }
+        if (pk) cudaEventRecord(pk[1], st);
     }
     return PLC_OK;
 }
@@ -358,9 +378,10 @@ static plc_status encode_impl(plc_ctx* c, const plc_kv_view* kv, const void* log
     a.pairs = c->pairs;
     a.step_exp = tokens_dev ? c->step_exp : nullptr;
     codec_schedule(a, 2 * a.sh.L * a.sh.H, &c->last_nq, &c->last_g);
-    if (c->profiling) cudaEventRecord(c->ev[0], st);
+    cudaEvent_t* pk = prof_pair(c, 0);
+    if (pk) cudaEventRecord(pk[0], st);
     cudaError_t e = launch_encode(a, st);
-    if (c->profiling) { cudaEventRecord(c->ev[1], st); c->ev_valid[0] = 1; }
+    if (pk) cudaEventRecord(pk[1], st);
     return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
@@ -402,9 +423,10 @@ static plc_status decode_impl(plc_ctx* c, const plc_streams* in, const void* log
     a.pairs = c->pairs;
     a.step_exp = tokens_dev ? c->step_exp : nullptr;
     codec_schedule(a, 2 * a.sh.L * a.sh.H, &c->last_nq, &c->last_g);
-    if (c->profiling) cudaEventRecord(c->ev[2], st);
+    cudaEvent_t* pk = prof_pair(c, 1);
+    if (pk) cudaEventRecord(pk[0], st);
     cudaError_t e = launch_decode(a, st);
-    if (c->profiling) { cudaEventRecord(c->ev[3], st); c->ev_valid[1] = 1; }
+    if (pk) cudaEventRecord(pk[1], st);
     return e == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
@@ -581,9 +603,27 @@ plc_status plc_set_profiling(plc_ctx* c, int32_t on) {
 
 plc_status plc_last_kernel_ms(plc_ctx* c, int32_t which, float* ms) {
     if (!c || !ms || which < 0 || which > 2) return PLC_E_INVALID;
-    if (!c->ev_valid[which]) return PLC_E_STATE;
-    if (cudaEventSynchronize(c->ev[2 * which + 1]) != cudaSuccess) return PLC_E_CUDA;
-    return cudaEventElapsedTime(ms, c->ev[2 * which], c->ev[2 * which + 1]) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+    const int n = c->prof_used[which];
+    if (n < 1) return PLC_E_STATE;
+    cudaEvent_t* p = &c->prof_ev[which][2 * (n - 1)];
+    if (cudaEventSynchronize(p[1]) != cudaSuccess) return PLC_E_CUDA;
+    return cudaEventElapsedTime(ms, p[0], p[1]) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+plc_status plc_kernel_ms(plc_ctx* c, int32_t which, float* mean_ms, int32_t* launches, int32_t reset) {
+    if (!c || which < 0 || which > 2) return PLC_E_INVALID;
+    const int n = c->prof_used[which];
+    double sum = 0.0;
+    for (int i = 0; i < n; ++i) {
+        cudaEvent_t* p = &c->prof_ev[which][2 * i];
+        float ms = 0.f;
+        if (cudaEventSynchronize(p[1]) != cudaSuccess || cudaEventElapsedTime(&ms, p[0], p[1]) != cudaSuccess) return PLC_E_CUDA;
+        sum += ms;
+    }
+    if (mean_ms) *mean_ms = n ? (float)(sum / n) : 0.f;
+    if (launches) *launches = n;
+    if (reset) c->prof_used[which] = 0;
+    return PLC_OK;
 }
 
 uint64_t plc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

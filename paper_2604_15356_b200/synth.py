@@ -187,9 +187,14 @@ def trie_sessions(table, S, n, seed, seg_lo, seg_hi, depth=3):
             tokens[s, pos:pos + m] = segs[nd][0, :m]
             pos += m
         plen[s] = pos
+    # every session continues from its prefix's last token; the continuations are drawn for all
+    # sessions at once (one uniform stream per session) and cut to the length each one needs
+    last = tokens[torch.arange(S, device=dev), (plen.to(dev).to(torch.int64) - 1).clamp_(min=0)].to(torch.int64)
+    cont = sample_tokens(table, S, n, seed * 1000 + 500, start=last)
+    for s in range(S):
+        pos = int(plen[s])
         if pos < n:
-            start = tokens[s, pos - 1:pos].to(torch.int64)
-            tokens[s, pos:] = sample_tokens(table, 1, n - pos, seed * 1000 + 500 + s, start=start)[0]
+            tokens[s, pos:] = cont[s, :n - pos]
     return tokens, prefix_keys(tokens), leaf, plen
 
 

@@ -225,6 +225,29 @@ def test_tables_beyond_l2_take_the_per_sm_queues(dev, orc):
     gpu_decode_check(g, kv, 0.02, n)
 
 
+def test_layer_shards_give_the_whole_context_chunk_for_chunk(dev):
+    """The streams are independent across layers: two contexts, each holding one half of T and coding
+    its half of the KV tensor (what two ranks do under a layer shard), produce chunk for chunk the
+    bytes of the single context that holds all of T.  Table t of shard r is table t + r * W/2 of the whole."""
+    S, n, L, H, d, V, K, CP = 2, 100, 4, 2, 128, 600, 24, 32
+    tokens, logits, T, kv = make_workload(77, S, n, L, H, d, V, K)
+    whole = gpu_encode(dev, T, kv, logits, K, 0.02, CP)
+    assert whole["rc"] == plc.OK
+    W, mc = whole["W"], whole["mc"]
+    seen = set()
+    for r, (lo, hi) in enumerate(((0, 2), (2, 4))):
+        part = gpu_encode(dev, T[lo:hi].contiguous(), kv[lo:hi].contiguous(), logits, K, 0.02, CP)
+        assert part["rc"] == plc.OK and part["W"] == W // 2
+        for s_ in range(S):
+            for t_ in range(W // 2):
+                for c in range(mc):
+                    tw = t_ + lo * 2 * H
+                    assert np.array_equal(part["st"].chunk((s_ * (W // 2) + t_) * mc + c), whole["st"].chunk((s_ * W + tw) * mc + c))
+                    seen.add((s_, tw, c))
+        assert part["ctx"].stats().payload_bytes < whole["ctx"].stats().payload_bytes
+    assert len(seen) == S * W * mc
+
+
 def test_position_ranges_and_empty_sessions(dev, orc):
     tokens, logits, T, kv = make_workload(7, 3, 100, 1, 2, 128, 512, 32)
     pb, pe = [0, 37, 100], [100, 91, 100]
@@ -546,13 +569,35 @@ def test_f16_output(dev):
     assert float((out.float() - kvd.float()).abs().max()) <= 0.01 + 1e-3 + 8 * 2 ** -11
 
 
-@pytest.mark.parametrize("S,n,L,H,d,V", [(1, 200, 1, 1, 128, 1000), (2, 70, 2, 2, 64, 520), (1, 130, 1, 1, 64, 4096)])
+def _oracle_export(orc, cfg, T, kv, logits, linear=None):
+    """(sym, q, mu, payload_bytes) of the oracle's whole-path encode; the full-vocabulary cases with
+    several column tiles are cut along the head axis over the host's cores (same oracle, one process
+    per slice)."""
+    rows, cols = logits.shape[0] * logits.shape[1], 2 * cfg.H * cfg.d
+    if rows * cols * cfg.V * cfg.L > 2e9:
+        e = orc.encode_parallel(cfg, None if T is None else T.numpy(), kv.numpy(), logits.numpy(), None, export=True,
+                                linear=None if linear is None else tuple(t.numpy() for t in linear))
+        return e["sym"], e["q"], e["mu"], e["stats"]["payload_bytes"]
+    e = orc.encode(cfg, None if T is None else T.numpy(), kv.numpy(), logits.numpy(), None, export=True)
+    return e["sym"], e["q"], e["mu"], e["stats"].payload_bytes
+
+
+def _note(**kw):
+    """Measured agreement rates of the tensor-core variants, printed (pytest -s / -rP shows them)."""
+    print("measured: " + ", ".join(f"{k}={v:.3g}" if isinstance(v, float) else f"{k}={v}" for k, v in kw.items()))
+
+
+# the last three cases have 2H*d = 1024 output columns (four column tiles of the contraction) and two
+# ragged row tiles; the last one runs the real vocabulary of the 70B configuration
+@pytest.mark.parametrize("S,n,L,H,d,V", [(1, 200, 1, 1, 128, 1000), (2, 70, 2, 2, 64, 520), (1, 130, 1, 1, 64, 4096),
+                                         (1, 200, 1, 4, 128, 1000), (2, 150, 2, 4, 128, 2000), (1, 130, 1, 4, 128, 32000)])
 def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
     """Def. 5 over the whole vocabulary as a bf16 tensor-core contraction (fp32 accumulation).
     Tolerances: mu as for the top-K path; symbols may differ from the oracle (exact sum of the same
-    bf16 products) where (kv - mu)/delta is within 5e-3 of a rounding boundary -- the accumulation
-    error of a V-term fp32 tensor-core sum plus the binary32 exp of the softmax -- fewer than 2e-3
-    of them; the coder stays bit-exact on the GPU's own symbols and decode inverts encode."""
+    bf16 products) where (kv - mu)/delta is within the prediction's own deviation (< 5e-3 step) of a
+    rounding boundary -- the accumulation error of a V-term fp32 tensor-core sum plus the binary32
+    exp of the softmax -- fewer than 2e-3 of them (measured: 4e-5 at V <= 4096, 4.4e-4 at V = 32000);
+    the coder stays bit-exact on the GPU's own symbols and decode inverts encode."""
     K, CP, delta = 8, 32, 0.02
     tokens, logits, T, kv = make_workload(300 + V, S, n, L, H, d, V, K, pp=12.0)
     ctx = plc.Context(T.to(dev), K, delta, chunk_pos=CP, variant=plc.PRED_DENSE)
@@ -565,19 +610,24 @@ def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
     ctx.encode(kvd, lgd, st, debug=plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr()))
     assert ctx.sync_status() == plc.OK
     cfg = orc.Config(L, H, d, V, K, delta, 0.0, CP, 1)
-    enc = orc.encode(cfg, T.numpy(), kv.numpy(), logits.numpy(), None, export=True)
-    mu_o = enc["mu"].reshape(S, n, W, d); sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W)
+    sym_o, q_o, mu_o, bytes_o = _oracle_export(orc, cfg, T, kv, logits)
+    mu_o = mu_o.reshape(S, n, W, d); sym_o = sym_o.reshape(S, n, W, d); q_o = q_o.reshape(S, n, W)
     mu_g, sym_g, q_g = mu.cpu().numpy(), sym.cpu().numpy(), q.cpu().numpy()
     scale = np.maximum(np.abs(mu_o).max(-1), 1e-3)
     assert (np.abs(mu_g - mu_o).max(-1) <= 1e-3 * scale).all(), float((np.abs(mu_g - mu_o).max(-1) / scale).max())
     diff = sym_g != sym_o
     assert diff.mean() < 2e-3, diff.mean()
     if diff.any():
+        # a symbol moves (by one) only where the prediction's own deviation carries r/delta across a boundary
         assert np.abs(sym_g - sym_o)[diff].max() == 1
         kvv = np.transpose(kv.numpy().astype(np.float64), (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)
         t = (kvv - mu_o.astype(np.float64)) / delta
-        assert np.abs(t - np.floor(t) - 0.5)[diff].max() < 5e-3
+        moved = np.abs(mu_g.astype(np.float64) - mu_o) / delta
+        assert (np.abs(t - np.floor(t) - 0.5)[diff] <= moved[diff] + 1e-3).all() and moved[diff].max() < 5e-3
     assert (q_g != q_o).mean() < 2e-2 and np.abs(q_g - q_o).max() <= 1
+    # every column tile carries its own table's prediction: per table, the mean error is as small as overall
+    per_table = (np.abs(mu_g - mu_o).max(-1) / scale).reshape(-1, W).max(0)
+    assert per_table.max() <= 1e-3
     total = 0
     for s_ in range(S):
         for t_ in range(W):
@@ -586,7 +636,9 @@ def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
                 ref, _, _ = orc.rans_encode_chunk(sym_g[s_, c * CP:c * CP + P, t_], q_g[s_, c * CP:c * CP + P, t_])
                 assert np.array_equal(st.chunk((s_ * W + t_) * mc + c), ref), (s_, t_, c)
                 total += len(ref)
-    assert abs(total / enc["stats"].payload_bytes - 1) < 2e-3
+    assert abs(total / bytes_o - 1) < 2e-3
+    _note(case=f"dense V={V} cols={W * d // L}", mu_rel=float((np.abs(mu_g - mu_o).max(-1) / scale).max()),
+          sym_mismatch=float(diff.mean()), q_mismatch=float((q_g != q_o).mean()), size_ratio=total / bytes_o)
     out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
     sym2 = torch.zeros_like(sym)
     ctx.decode(st, lgd, out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None))
@@ -595,7 +647,8 @@ def test_dense_variant_parity(dev, orc, S, n, L, H, d, V):
     assert float((out.cpu() - kv.float()).abs().max()) <= delta / 2 + 1e-3
 
 
-@pytest.mark.parametrize("S,n,L,H,d,V,dm", [(1, 200, 2, 1, 128, 1000, 64), (2, 70, 3, 2, 64, 520, 192), (1, 130, 1, 3, 32, 2048, 256)])
+@pytest.mark.parametrize("S,n,L,H,d,V,dm", [(1, 200, 2, 1, 128, 1000, 64), (2, 70, 3, 2, 64, 520, 192), (1, 130, 1, 3, 32, 2048, 256),
+                                            (1, 150, 2, 4, 128, 2048, 192), (1, 130, 1, 4, 128, 32000, 128)])
 def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
     """Sec. 7.1, linear-embedding predictor: KV^ = c + A Ebar as two chained bf16 tensor-core
     contractions (Ebar = P E, then A Ebar), variance by Thm. 2 with F := c + A E.
@@ -603,8 +656,8 @@ def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
     lands within an accumulation error of a bf16 rounding boundary the GPU may take the other
     neighbour: mu then moves by 2^-8 |Ebar_k A_jk|, i.e. a few 1e-4 of the vector's scale; the bound
     used is 3e-3 of max|mu|.  Symbols may differ by one where (kv - mu)/delta is within 0.1 of a
-    rounding boundary (fewer than 1 % of them); classes by one step in fewer than 2 %; the coder is
-    bit-exact on the GPU's own symbols and decode inverts encode."""
+    rounding boundary by no more than mu itself moved (fewer than 1 % of them); classes by one step in
+    fewer than 2 %; the coder is bit-exact on the GPU's own symbols and decode inverts encode."""
     CP, delta = 32, 0.02
     table = synth.markov_table(V, 12.0, 700 + V)
     tokens = synth.sample_tokens(table, S, n, 701 + V)
@@ -621,8 +674,8 @@ def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
     ctx.encode(kvd, lgd, st, debug=plc.DebugBuffers(sym.data_ptr(), q.data_ptr(), mu.data_ptr()))
     assert ctx.sync_status() == plc.OK
     cfg = orc.linear_config(L, H, d, V, 1, delta, CP, E.numpy(), A.numpy(), c.numpy())
-    enc = orc.encode(cfg, None, kv.numpy(), logits.numpy(), None, export=True)
-    mu_o = enc["mu"].reshape(S, n, W, d); sym_o = enc["sym"].reshape(S, n, W, d); q_o = enc["q"].reshape(S, n, W)
+    sym_o, q_o, mu_o, bytes_o = _oracle_export(orc, cfg, None, kv, logits, linear=(E, A, c))
+    mu_o = mu_o.reshape(S, n, W, d); sym_o = sym_o.reshape(S, n, W, d); q_o = q_o.reshape(S, n, W)
     mu_g, sym_g, q_g = mu.cpu().numpy(), sym.cpu().numpy(), q.cpu().numpy()
     scale = np.maximum(np.abs(mu_o).max(-1), 1e-3)
     rel = np.abs(mu_g - mu_o).max(-1) / scale
@@ -630,10 +683,12 @@ def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
     diff = sym_g != sym_o
     assert diff.mean() < 1e-2, diff.mean()
     if diff.any():
+        # a symbol moves (by one) only where the prediction's own deviation carries r/delta across a boundary
         assert np.abs(sym_g - sym_o)[diff].max() == 1
         kvv = np.transpose(kv.numpy().astype(np.float64), (2, 4, 0, 1, 3, 5)).reshape(S, n, W, d)
         t = (kvv - mu_o.astype(np.float64)) / delta
-        assert np.abs(t - np.floor(t) - 0.5)[diff].max() < 0.1
+        moved = np.abs(mu_g.astype(np.float64) - mu_o) / delta
+        assert (np.abs(t - np.floor(t) - 0.5)[diff] <= moved[diff] + 1e-3).all()
     assert (q_g != q_o).mean() < 2e-2 and np.abs(q_g - q_o).max() <= 1
     total = 0
     for s_ in range(S):
@@ -643,7 +698,9 @@ def test_linear_embedding_variant_parity(dev, orc, S, n, L, H, d, V, dm):
                 ref, _, _ = orc.rans_encode_chunk(sym_g[s_, ch * CP:ch * CP + P, t_], q_g[s_, ch * CP:ch * CP + P, t_])
                 assert np.array_equal(st.chunk((s_ * W + t_) * mc + ch), ref), (s_, t_, ch)
                 total += len(ref)
-    assert abs(total / enc["stats"].payload_bytes - 1) < 5e-3
+    assert abs(total / bytes_o - 1) < 5e-3
+    _note(case=f"linear V={V} cols={W * d // L} dm={dm}", mu_rel=float(rel.max()), sym_mismatch=float(diff.mean()),
+          q_mismatch=float((q_g != q_o).mean()), size_ratio=total / bytes_o)
     out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
     sym2 = torch.zeros_like(sym)
     ctx.decode(st, lgd, out, debug=plc.DebugBuffers(sym2.data_ptr(), None, None))
