@@ -128,9 +128,11 @@ typedef struct {
 } plc_stats;
 
 /* State of a batch of B sessions that grow by one position per plc_append_step (lock step).
- * open_sym_dev [B][W][chunk_pos][d] int32 and open_q_dev [B][W][chunk_pos] int32 hold the positions
- * of the chunk that is still open; steps counts the positions appended so far (host side).
- * The index in `streams` is [B][W][max_chunks]; chunk c holds positions [c*chunk_pos, ...). */
+ * open_sym_dev [2][B][W][chunk_pos][d] int32 and open_q_dev [2][B][W][chunk_pos] int32 hold the
+ * symbols and classes of positions that are not coded yet, in two buffers: chunk c uses buffer
+ * c mod 2, so that the chunk completed last can be coded while the next one fills.  steps counts the
+ * positions appended so far (host side).  The index in `streams` is [B][W][max_chunks] (the caller
+ * zeroes it); chunk c holds positions [c*chunk_pos, ...). */
 typedef struct {
     int32_t B;
     int32_t steps;
@@ -295,14 +297,19 @@ plc_status plc_decode_rotq(plc_ctx* ctx, const void* records_dev, uint64_t recor
 
 /* Decode-time append (integration point 1 for one new token per session).  kv_step_dev
  * [L][2][B][H][d] f16, logits_step_dev [B][V] f16.  The new position's symbols and class go to the
- * open chunk; when it holds chunk_pos positions it is coded into sb->streams (a LIFO coder cannot
- * be extended in place, so a stream grows chunk by chunk).  sb->steps is advanced. */
+ * open chunk (a LIFO coder cannot be extended in place, so a stream grows chunk by chunk).  A chunk
+ * that has reached chunk_pos positions is coded into sb->streams over the following chunk_pos steps,
+ * 1/chunk_pos of the B*W streams per step (stream i = table*B + session in slice
+ * floor(i*chunk_pos / (B*W)) is coded by the step at which steps mod chunk_pos equals the slice
+ * number), so that every step costs the same: chunk c of every stream is in sb->streams once
+ * steps >= (c+2)*chunk_pos - 1, or after plc_append_flush.  sb->steps is advanced. */
 plc_status plc_append_step(plc_ctx* ctx, plc_session_batch* sb, const void* kv_step_dev, const void* logits_step_dev,
                            void* stream);
-/* Codes the partly filled open chunk (if any) so that all sb->steps positions are decodable with
+/* Codes what is not coded yet (the remaining slices of the chunk completed last and the partly
+ * filled open chunk, if any) so that all sb->steps positions are decodable with
  * plc_decode(S = B, n = steps).  No further plc_append_step is allowed afterwards. */
 plc_status plc_append_flush(plc_ctx* ctx, plc_session_batch* sb, void* stream);
-/* Bytes of open_sym_dev / open_q_dev for B sessions. */
+/* Bytes of open_sym_dev / open_q_dev for B sessions (both buffers). */
 plc_status plc_append_sizes(const plc_ctx* ctx, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes);
 
 /* Entropy-codes one chunk per stream from symbols and classes that are already on the device,
@@ -313,8 +320,9 @@ plc_status plc_append_sizes(const plc_ctx* ctx, int32_t B, uint64_t* open_sym_by
  * whose creation allocates.)  The bitstream is exactly the one plc_append_step / plc_append_flush
  * write for the same symbols and classes.
  *   sym_dev [n_streams][chunk_capacity][head_dim] int32, q_dev [n_streams][chunk_capacity] int32:
- *   the first n_pos positions of every stream are coded (the layout of plc_session_batch's open
- *   chunk, with n_streams = B*W); classes outside [-24, 135] are clamped and reported.
+ *   the first n_pos positions of every stream are coded (the layout of one buffer of
+ *   plc_session_batch's open chunks, with n_streams = B*W); classes outside [-24, 135] are clamped
+ *   and reported.
  *   Chunk `chunk_index` of stream i goes to index slot i*out->max_chunks + chunk_index.
  *   status_dev: one device word, an OUTPUT: 0, or a bit-or of 1 (payload capacity exceeded; nothing
  *   is written past it and *total_bytes_dev holds the size needed), 4 (a class was out of range) and

@@ -26,6 +26,9 @@ struct plc_ctx {
     unsigned int* status;
     unsigned int* status_host;      // pinned word plc_poll_status copies into
     cudaStream_t poll_stream;       // non-blocking stream of plc_poll_status
+    cudaStream_t side_stream;       // append path: the slice of a completed chunk is coded beside the step's own kernels
+    cudaEvent_t side_ev[2];         // fork / join of the side stream
+    unsigned int* side_ticket;      // work counter of the side stream's launches
     Counters* counters;
     uint8_t* dense_scratch;         // dense variant: P, Tb, n2b, mu, s1; linear variant: P, Ebar, s1, A_layer, mu
     size_t dense_bytes;
@@ -223,6 +226,10 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
               cudaMalloc(&c->status, sizeof(unsigned int)) == cudaSuccess &&
               cudaMallocHost(&c->status_host, sizeof(unsigned int)) == cudaSuccess &&
               cudaStreamCreateWithFlags(&c->poll_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->side_ev[0], cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->side_ev[1], cudaEventDisableTiming) == cudaSuccess &&
+              cudaMalloc(&c->side_ticket, sizeof(unsigned int)) == cudaSuccess &&
               cudaMalloc(&c->counters, sizeof(Counters)) == cudaSuccess;
     if (ok) ok = cudaMemset(c->status, 0, sizeof(unsigned int)) == cudaSuccess &&
                  cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
@@ -249,6 +256,9 @@ plc_status plc_destroy(plc_ctx* c) {
         for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->poll_stream) cudaStreamDestroy(c->poll_stream);
+    if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    for (int i = 0; i < 2; ++i) if (c->side_ev[i]) cudaEventDestroy(c->side_ev[i]);
+    cudaFree(c->side_ticket);
     delete c;
     return PLC_OK;
 }
@@ -495,17 +505,31 @@ plc_status plc_decode_rotq(plc_ctx* c, const void* records_dev, uint64_t records
 plc_status plc_append_sizes(const plc_ctx* c, int32_t B, uint64_t* open_sym_bytes, uint64_t* open_q_bytes) {
     if (!c || B < 0 || !open_sym_bytes || !open_q_bytes) return PLC_E_INVALID;
     const uint64_t W = 2ull * c->cfg.n_layers * c->cfg.n_kv_heads;
-    *open_q_bytes = 4ull * B * W * c->cfg.chunk_pos;
+    *open_q_bytes = 2ull * 4ull * B * W * c->cfg.chunk_pos;            // two buffers: chunk c fills buffer c mod 2
     *open_sym_bytes = *open_q_bytes * c->cfg.head_dim;
     return PLC_OK;
 }
 
-static plc_status seal(plc_ctx* c, plc_session_batch* sb, int chunk_index, int count, cudaStream_t st) {
+// Codes items [first, first + items) (item = table * B + session) of chunk `chunk_index`, whose `count`
+// positions sit in open buffer chunk_index mod 2.
+static plc_status seal(plc_ctx* c, plc_session_batch* sb, int chunk_index, int count, unsigned first, unsigned items,
+                       cudaStream_t st, bool side = false) {
+    if (items == 0 || count == 0) return PLC_OK;
     CodecArgs a = base_args(c);
+    if (side) a.ticket = c->side_ticket;
     a.S = sb->B; a.n = 0;
     a.st = to_dev(&sb->streams);
-    a.open_sym = sb->open_sym_dev; a.open_q = sb->open_q_dev; a.open_count = count; a.chunk_index = chunk_index;
+    const size_t per_buf = (size_t)sb->B * 2 * c->cfg.n_layers * c->cfg.n_kv_heads * c->cfg.chunk_pos;
+    a.open_sym = sb->open_sym_dev + (size_t)(chunk_index & 1) * per_buf * c->cfg.head_dim;
+    a.open_q = sb->open_q_dev + (size_t)(chunk_index & 1) * per_buf;
+    a.open_count = count; a.chunk_index = chunk_index; a.open_first = first; a.open_items = items;
     return launch_append_seal(a, st) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+}
+
+// Slice j of CP equal slices of the B*W streams.
+static void seal_slice(long long n_streams, int CP, int j, unsigned* first, unsigned* items) {
+    const long long lo = n_streams * j / CP, hi = n_streams * (j + 1) / CP;
+    *first = (unsigned)lo; *items = (unsigned)(hi - lo);
 }
 
 plc_status plc_append_step(plc_ctx* c, plc_session_batch* sb, const void* kv_step_dev, const void* logits_step_dev,
@@ -518,26 +542,56 @@ plc_status plc_append_step(plc_ctx* c, plc_session_batch* sb, const void* kv_ste
     plc_status rc = check_streams(&sb->streams, sb->steps / CP + 1);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t d = c->cfg.head_dim, H = c->cfg.n_kv_heads, B = sb->B;
+    const long long n_streams = (long long)B * 2 * c->cfg.n_layers * H;
+    // The chunk completed last is coded a slice of the streams at a time, one slice per step, so that no
+    // step carries the coding of all streams.  Slices 1 .. CP-1 read a buffer that this step does not
+    // touch: they run on a stream of the context's own beside this step's kernels (forked from and
+    // joined to the caller's stream, so the call stays stream-ordered for the caller).  Slice 0 reads
+    // the position this very step writes and follows it on the caller's stream.
+    const int after = sb->steps + 1, done = after / CP, phase = after % CP;
+    unsigned first = 0, items = 0;
+    if (done >= 1) seal_slice(n_streams, CP, phase, &first, &items);
+    const bool beside = done >= 1 && phase != 0 && items > 0;
+    if (beside) {
+        if (cudaEventRecord(c->side_ev[0], st) != cudaSuccess || cudaStreamWaitEvent(c->side_stream, c->side_ev[0], 0) != cudaSuccess)
+            return PLC_E_CUDA;
+        rc = seal(c, sb, done - 1, CP, first, items, c->side_stream, true);
+        if (rc) return rc;
+        if (cudaEventRecord(c->side_ev[1], c->side_stream) != cudaSuccess) return PLC_E_CUDA;
+    }
     rc = run_topk_for(c, logits_step_dev, sb->B, 1, nullptr, nullptr, st);
     if (rc) return rc;
     CodecArgs a = base_args(c);
-    const int64_t d = c->cfg.head_dim, H = c->cfg.n_kv_heads, B = sb->B;
+    const size_t per_buf = (size_t)n_streams * CP;
+    const int chunk = sb->steps / CP;
     a.kv = KvView{const_cast<void*>(kv_step_dev), 2 * B * H * d, B * H * d, H * d, d, 0};
     a.S = sb->B; a.n = 1;
-    a.open_sym = sb->open_sym_dev; a.open_q = sb->open_q_dev; a.open_slot = sb->steps % CP;
+    a.open_sym = sb->open_sym_dev + (size_t)(chunk & 1) * per_buf * d;
+    a.open_q = sb->open_q_dev + (size_t)(chunk & 1) * per_buf;
+    a.open_slot = sb->steps % CP;
     if (launch_append_quantise(a, st) != cudaSuccess) return PLC_E_CUDA;
-    sb->steps += 1;
-    if (sb->steps % CP == 0) return seal(c, sb, sb->steps / CP - 1, CP, st);
+    sb->steps = after;
+    if (beside) return cudaStreamWaitEvent(st, c->side_ev[1], 0) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
+    if (done >= 1) return seal(c, sb, done - 1, CP, first, items, st);
     return PLC_OK;
 }
 
 plc_status plc_append_flush(plc_ctx* c, plc_session_batch* sb, void* stream) {
     if (!c || !sb || !sb->open_sym_dev || !sb->open_q_dev || sb->B < 1 || sb->steps < 0) return PLC_E_INVALID;
-    const int CP = c->cfg.chunk_pos, rem = sb->steps % CP;
-    if (rem == 0) return PLC_OK;
-    plc_status rc = check_streams(&sb->streams, sb->steps / CP + 1);
+    const int CP = c->cfg.chunk_pos, rem = sb->steps % CP, done = sb->steps / CP;
+    plc_status rc = check_streams(&sb->streams, done + (rem ? 1 : 0));
     if (rc) return rc;
-    return seal(c, sb, sb->steps / CP, rem, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long n_streams = (long long)sb->B * 2 * c->cfg.n_layers * c->cfg.n_kv_heads;
+    if (done >= 1 && rem != CP - 1) {          // slices rem + 1 .. CP - 1 of the last complete chunk are still uncoded
+        unsigned first, items, f2, i2;
+        seal_slice(n_streams, CP, rem + 1, &first, &items);
+        seal_slice(n_streams, CP, CP - 1, &f2, &i2);
+        rc = seal(c, sb, done - 1, CP, first, f2 + i2 - first, st);
+        if (rc) return rc;
+    }
+    return seal(c, sb, done, rem, 0u, (unsigned)n_streams, st);
 }
 
 plc_status plc_sync_status(plc_ctx* c, void* stream) {

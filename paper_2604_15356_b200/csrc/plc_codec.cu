@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
     int2* sp0 = g_pair_smem + (threadIdx.x >> 5) * 2 * Kp;
     const int Wl = DENSE ? 2 * H : Wt;                       // tables this launch covers
-    const unsigned total = FROM_OPEN ? (unsigned)a.S * Wt : (unsigned)Wl * a.S * a.st.max_chunks;
+    const unsigned total = FROM_OPEN ? a.open_items : (unsigned)Wl * a.S * a.st.max_chunks;
     const float inv_d = 1.0f / D, inv_delta = a.sh.inv_delta, inv_delta2 = a.sh.inv_delta2,
                 floor2 = a.sh.sigma_floor * a.sh.sigma_floor;
     const int c0 = first_comp<D>(lane);
@@ -587,7 +587,8 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     for (unsigned item = next(); item < total; item = next()) {
         Item it;
         if (FROM_OPEN) {
-            it.t = (int)(item / a.S); it.s = (int)(item % a.S); it.c = a.chunk_index;
+            const unsigned oi = a.open_first + item;
+            it.t = (int)(oi / a.S); it.s = (int)(oi % a.S); it.c = a.chunk_index;
             it.p0 = 0; it.P = a.open_count;
             it.slot = ((long long)it.s * Wt + it.t) * a.st.max_chunks + it.c;
         } else {
@@ -1053,7 +1054,7 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     return dispatch_d(a.sh.d, [&](auto D) {
-        long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
+        long long warps = (long long)a.open_items;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (long long)sm_count() * kBlocksPerSM) blocks = (long long)sm_count() * kBlocksPerSM;
         auto ko = a.sh.zero_q != kZeroOff ? encode_kernel<decltype(D)::value, kSrcOpen, true> : encode_kernel<decltype(D)::value, kSrcOpen, false>;

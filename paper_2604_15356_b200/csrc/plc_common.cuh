@@ -205,6 +205,7 @@ struct CodecArgs {
     const __half* mu_bias;                         // optional [2*H][d] f16 added to mu (linear predictor's c), or null
     // append path: symbols come from / go to the open chunk
     int32_t* open_sym; int32_t* open_q; int open_slot; int open_count; int chunk_index;
+    unsigned open_first, open_items;               // seal launch: the (table, session) items [open_first, open_first + open_items)
 };
 int codec_grid_warps(int device);
 // Work-queue layout a gather launch over n_tables tables would use: nq queues, g SMs per queue.

@@ -287,19 +287,38 @@ def test_append_full_batch_sampled_chunks(orc):
     pb = torch.tensor([p[0] for p in picks], device=dev); pt = torch.tensor([p[1] for p in picks], device=dev)
     kv_keep = np.zeros((len(picks), steps, d), np.float16)
     g = torch.Generator(device=dev); g.manual_seed(seed + 3)
-    open_sym = sb.open_sym.view(B, W, CP, d); open_q = sb.open_q.view(B, W, CP)
+    open_sym = sb.open_sym.view(2, B, W, CP, d); open_q = sb.open_q.view(2, B, W, CP)   # chunk c fills buffer c mod 2
     sealed = {}
+    lat = []
     for i in range(steps):
         tok = tokens[:, i].to(torch.int64)
         kv_step = (T[:, :, :, tok, :].permute(0, 1, 3, 2, 4).float() +
                    cfg["sigma"] * torch.randn(L, 2, B, H, d, device=dev, generator=g)).to(torch.float16).contiguous()
         flat = kv_step.permute(2, 0, 1, 3, 4).reshape(B, W, d)                # [B][table][d], table = (l*2 + kv)*H + h
         kv_keep[:, i] = flat[pb, pt].cpu().numpy()
-        ctx.append_step(sb, kv_step, logits[:, i, :].contiguous())
+        lg = logits[:, i, :].contiguous()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.append_step(sb, kv_step, lg)
+        e1.record()
+        lat.append((e0, e1))
         if (i + 1) % CP == 0:
-            sealed[(i + 1) // CP - 1] = (open_sym[pb, pt].cpu().numpy(), open_q[pb, pt].cpu().numpy(), CP)
+            c = (i + 1) // CP - 1
+            sealed[c] = (open_sym[c & 1][pb, pt].cpu().numpy(), open_q[c & 1][pb, pt].cpu().numpy(), CP)
+    # a completed chunk is coded a slice of the streams per step: after 70 steps chunk 0 is in the container
+    # in full (coded by steps 32 .. 63), chunk 1 only for the slices of steps 64 .. 69
+    torch.cuda.synchronize()
+    nby = sb.streams.chunk_bytes.view(B * W, 3).cpu().numpy()
+    item = np.arange(B * W)                                               # item = table * B + session
+    slot_of_item = (item % B) * W + item // B
+    assert np.all(nby[:, 0] > 128)
+    assert np.all((nby[slot_of_item, 1] > 0) == (item * CP // (B * W) <= steps % CP)) and not nby[:, 2].any()
     ctx.append_flush(sb)
-    sealed[steps // CP] = (open_sym[pb, pt].cpu().numpy(), open_q[pb, pt].cpu().numpy(), steps % CP)
+    c = steps // CP
+    sealed[c] = (open_sym[c & 1][pb, pt].cpu().numpy(), open_q[c & 1][pb, pt].cpu().numpy(), steps % CP)
+    # every step costs about the same: no step carries the coding of all streams at once
+    ms = sorted(a.elapsed_time(b) for a, b in lat[CP:])
+    assert ms[-1] <= 2.0 * ms[len(ms) // 2], (ms[len(ms) // 2], ms[-1])
     assert ctx.sync_status() == plc.OK
     stats = ctx.stats()
     assert stats.n_chunks == B * W * 3 and stats.coded_vectors == B * W * steps

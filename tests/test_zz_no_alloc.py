@@ -34,13 +34,12 @@ def test_static_coder_matches_append_sealing_twice():
         sb = ctx.new_session_batch(B, 1, cap)
         for i in range(steps):
             ctx.append_step(sb, kv[:, :, :, :, i, :].contiguous(), logits[:, i, :].contiguous())
-        if steps % CP:
-            ctx.append_flush(sb)
+        ctx.append_flush(sb)                            # codes whatever the steps have not coded yet
         assert ctx.sync_status() == plc.OK
         ref = [sb.streams.chunk(s) for s in range(B * W)]
         assert all(len(r) > 128 for r in ref)
-        sym = sb.open_sym.view(B * W, CP, d)
-        q = sb.open_q.view(B * W, CP)
+        sym = sb.open_sym.view(2, B * W, CP, d)[0]      # chunk 0 sits in the first of the two open buffers
+        q = sb.open_q.view(2, B * W, CP)[0]
         status = torch.full((1,), 77, dtype=torch.int32, device=dev)
         for call in range(2):                           # two calls in a row share the static array
             out = plc.StreamSet(B * W, 1, cap, dev)
