@@ -36,7 +36,8 @@ struct plc_ctx {
     const __half* lin_A;
     const __half* lin_c;
     int lin_dm;
-    uint8_t* lin_model;             // E transposed (bf16) and the candidate-norm table of every (layer, table)
+    uint8_t* lin_model;             // linear: E transposed (bf16) and the candidate-norm table of every (layer, table);
+                                    // dense: the candidate-norm table alone
     size_t lin_off[2];
     int last_nq, last_g;            // work-queue layout of the most recent top-K encode / decode launch
     int profiling;                  // record events around the codec kernels
@@ -134,6 +135,7 @@ DenseShape dense_shape(const plc_ctx* c, long long rows) {
     sh.rows = rows; sh.V = c->cfg.vocab; sh.d = c->cfg.head_dim; sh.tables = 2 * c->cfg.n_kv_heads;
     sh.ldv = (sh.V + 63) / 64 * 64;
     sh.ncols = sh.tables * sh.d; sh.ncols_pad = (sh.ncols + 255) / 256 * 256;
+    sh.nt_all = c->cfg.n_layers * sh.tables; sh.nt_all_pad = (sh.nt_all + 255) / 256 * 256;
     return sh;
 }
 
@@ -235,6 +237,12 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
                  cudaMemset(c->counters, 0, sizeof(Counters)) == cudaSuccess;
     if (ok && T_dev) ok = launch_rownorm(c->T, c->rownorm2, rows, cfg->head_dim, 0) == cudaSuccess &&
                           cudaDeviceSynchronize() == cudaSuccess;
+    if (ok && T_dev && cfg->variant == PLC_PRED_DENSE) {     // candidate norms of every layer, once
+        const DenseShape sh = dense_shape(c, 0);
+        ok = (long long)cfg->n_layers * 2 * cfg->n_kv_heads <= 65536 &&
+             cudaMalloc(&c->lin_model, dense_model_bytes(sh)) == cudaSuccess &&
+             dense_prepare(c->T, cfg->n_layers, sh, c->lin_model, 0) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
+    }
     if (ok && lin) {
         c->lin_E = static_cast<const __half*>(lin->E_dev); c->lin_A = static_cast<const __half*>(lin->A_dev);
         c->lin_c = static_cast<const __half*>(lin->c_dev); c->lin_dm = lin->d_model;
@@ -319,16 +327,17 @@ static plc_status run_dense(plc_ctx* c, CodecArgs a, const void* logits_dev, boo
     size_t off[5];
     plc_status rc = ensure_dense(c, sh, off);
     if (rc) return rc;
-    if (dense_softmax(static_cast<const __half*>(logits_dev), sh, c->dense_scratch, off, st) != cudaSuccess) return PLC_E_CUDA;
+    if (dense_begin(static_cast<const __half*>(logits_dev), sh, c->lin_model, c->dense_scratch, off, c->status, st) != cudaSuccess)
+        return PLC_E_CUDA;
     a.mu_dense = reinterpret_cast<const float*>(c->dense_scratch + off[3]);
-    a.s1_dense = reinterpret_cast<const float*>(c->dense_scratch + off[4]);
-    a.mu_ld = sh.ncols; a.s1_ld = sh.tables;
+    a.mu_ld = sh.ncols; a.s1_ld = sh.nt_all;
     const size_t layer_elems = (size_t)sh.tables * sh.V * sh.d;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         cudaEvent_t* pg = prof_pair(c, 2);
         if (dense_layer(c->T + l * layer_elems, sh, c->dense_scratch, off, c->status, st, pg ? pg[0] : nullptr,
                         pg ? pg[1] : nullptr) != cudaSuccess) return PLC_E_CUDA;
         a.dense_layer = l;
+        a.s1_dense = reinterpret_cast<const float*>(c->dense_scratch + off[4]) + (size_t)l * sh.tables;
         cudaEvent_t* pk = prof_pair(c, encode ? 0 : 1);
         if (pk) cudaEventRecord(pk[0], st);
         if ((encode ? launch_encode(a, st) : launch_decode(a, st)) != cudaSuccess) return PLC_E_CUDA;

@@ -228,8 +228,13 @@ struct DenseShape {
     int V, d, tables;      // tables = 2 * H of one layer
     int ldv;               // V rounded up to 64 (row pitch of P and Tb, in elements)
     int ncols, ncols_pad;  // tables * d, rounded up to 256
+    int nt_all, nt_all_pad;   // L * tables (one variance column per layer and table), rounded up to 256
 };
-size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]: P, Tb, n2b, mu, s1*/);
+size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]: P, Tb, -, mu, s1*/);
+size_t dense_model_bytes(const DenseShape& sh);
+cudaError_t dense_prepare(const __half* T, int L, const DenseShape& sh, uint8_t* model, cudaStream_t st);
+cudaError_t dense_begin(const __half* logits, const DenseShape& sh, const uint8_t* model, uint8_t* scratch, const size_t* off,
+                        unsigned int* status, cudaStream_t st);
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st);
 // Linear-embedding predictor (Sec. 7.1).
 struct LinearShape {

@@ -91,7 +91,12 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
     volatile uint32_t* failed = tmem_slot + 1;        // set by any role whose wait ran out
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * bn;
+    // Column tile fastest in launch order: the CTAs resident together then share their row blocks of A
+    // (each block of A is fetched from HBM once and found in L2 by the other column tiles), and B, the
+    // smaller operand, is what gets re-read from L2.
+    const int ntn = (int)gridDim.y;
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+    const int m0 = (lin / ntn) * kBM, n0 = (lin % ntn) * bn;
     const uint32_t stage_tx = (uint32_t)(kABytes + bn * kBK * 2), idesc = make_idesc(bn);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), tfull = smem_u32(bars + 2 * kStages);
 
@@ -400,10 +405,35 @@ size_t dense_scratch_bytes(const DenseShape& sh, size_t* off /*[5]*/) {
     size_t o = 0;
     off[0] = o; o += up((size_t)sh.rows * sh.ldv * 2);                 // P
     off[1] = o; o += up((size_t)sh.ncols_pad * sh.ldv * 2);            // Tb
-    off[2] = o; o += up((size_t)((sh.tables + 15) / 16 * 16) * sh.ldv * 2);   // Nb (row norms, bf16)
+    off[2] = o;                                                        // (unused)
     off[3] = o; o += up((size_t)sh.rows * sh.ncols * 4);               // mu
-    off[4] = o; o += up((size_t)sh.rows * sh.tables * 4);              // s1
+    off[4] = o; o += up((size_t)sh.rows * sh.nt_all * 4);              // s1 of every (layer, table)
     return o;
+}
+
+size_t dense_model_bytes(const DenseShape& sh) { return (size_t)sh.nt_all_pad * sh.ldv * 2; }
+
+// Creation: Nb_all[l * tables + t][v] = bf16(sum_j bf16(T[l][t][v][j])^2 / d) for every layer; rows beyond
+// L * tables and columns beyond V are zero.
+cudaError_t dense_prepare(const __half* T, int L, const DenseShape& sh, uint8_t* model, cudaStream_t st) {
+    __nv_bfloat16* Nb = reinterpret_cast<__nv_bfloat16*>(model);
+    cudaError_t e = cudaMemsetAsync(Nb, 0, dense_model_bytes(sh), st);
+    if (e != cudaSuccess) return e;
+    const long long nrows = (long long)L * sh.tables * sh.V;
+    rownorm_bf16_kernel<<<blocks_for(nrows * 32), 256, 0, st>>>(T, nrows, sh.V, sh.d, sh.ldv, Nb);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// Per call: P = bf16(softmax(logits)) and the variance term of every layer in one contraction,
+// s1[row][l * tables + t] = sum_v P[row][v] Nb_all[l * tables + t][v].
+cudaError_t dense_begin(const __half* logits, const DenseShape& sh, const uint8_t* model, uint8_t* scratch, const size_t* off,
+                        unsigned int* status, cudaStream_t st) {
+    cudaError_t e = dense_softmax(logits, sh, scratch, off, st);
+    if (e != cudaSuccess) return e;
+    return launch_gemm(reinterpret_cast<const __nv_bfloat16*>(scratch + off[0]), sh.rows,
+                       reinterpret_cast<const __nv_bfloat16*>(model), sh.nt_all_pad, sh.ldv, 256,
+                       reinterpret_cast<float*>(scratch + off[4]), sh.nt_all, sh.nt_all, status, st);
 }
 
 cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* scratch, const size_t* off, cudaStream_t st) {
@@ -418,14 +448,13 @@ cudaError_t dense_softmax(const __half* logits, const DenseShape& sh, uint8_t* s
     return cudaGetLastError();
 }
 
-// Prediction of one layer: fills mu [rows][ncols] and s1 [rows][tables] in the scratch.
+// Prediction of one layer: fills mu [rows][ncols] in the scratch (the variance term of every layer was
+// formed by dense_begin).
 cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
                         unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1) {
     __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(scratch + off[0]);
     __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(scratch + off[1]);
-    __nv_bfloat16* Nb = reinterpret_cast<__nv_bfloat16*>(scratch + off[2]);
     float* mu = reinterpret_cast<float*>(scratch + off[3]);
-    float* s1 = reinterpret_cast<float*>(scratch + off[4]);
     cudaError_t e;
     if (sh.ncols_pad > sh.ncols) {       // rows of Tb beyond the real columns must read as zero
         e = cudaMemsetAsync(Tb + (size_t)sh.ncols * sh.ldv, 0, (size_t)(sh.ncols_pad - sh.ncols) * sh.ldv * 2, st);
@@ -433,29 +462,11 @@ cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* sc
     }
     dim3 tg((sh.ldv + 31) / 32, sh.d / 32, sh.tables);
     transpose_bf16_kernel<<<tg, 256, 0, st>>>(T_layer, sh.tables, sh.V, sh.d, sh.ldv, Tb);
-    const long long nrows = (long long)sh.tables * sh.V;
-    e = cudaMemsetAsync(Nb, 0, (size_t)((sh.tables + 15) / 16 * 16) * sh.ldv * 2, st);     // padding rows / columns read as zero
-    if (e != cudaSuccess) return e;
-    rownorm_bf16_kernel<<<blocks_for(nrows * 32), 256, 0, st>>>(T_layer, nrows, sh.V, sh.d, sh.ldv, Nb);
-    CUtensorMap ma, mb;
-    const int nb_rows = (sh.tables + 15) / 16 * 16;                     // norm matrix rows, <= 256
-    CUtensorMap mn;
-    if (!make_map(&ma, P, (uint64_t)sh.ldv, (uint64_t)sh.rows, (uint64_t)sh.ldv, kBM)) return cudaErrorUnknown;
-    if (!make_map(&mb, Tb, (uint64_t)sh.ldv, (uint64_t)sh.ncols_pad, (uint64_t)sh.ldv, kBN)) return cudaErrorUnknown;
-    if (!make_map(&mn, Nb, (uint64_t)sh.ldv, (uint64_t)nb_rows, (uint64_t)sh.ldv, (uint32_t)nb_rows)) return cudaErrorUnknown;
-    e = cudaFuncSetAttribute(dense_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
-    if (e != cudaSuccess) return e;
-    dim3 gg((unsigned)((sh.rows + kBM - 1) / kBM), (unsigned)(sh.ncols_pad / kBN));
+    count_launch();
     if (ev0) cudaEventRecord(ev0, st);
-    dense_gemm_kernel<<<gg, kGemmThreads, kGemmSmem, st>>>(ma, mb, mu, (long long)sh.ncols, (int)sh.rows, sh.ncols,
-                                                           sh.ldv / kBK, kBN, status);
+    e = launch_gemm(P, sh.rows, Tb, sh.ncols_pad, sh.ldv, kBN, mu, (long long)sh.ncols, sh.ncols, status, st);
     if (ev1) cudaEventRecord(ev1, st);
-    // variance term: s1 = P * Nb^T, the same kernel with an N tile of nb_rows columns
-    dim3 gn(gg.x, 1);
-    dense_gemm_kernel<<<gn, kGemmThreads, kGemmSmem, st>>>(ma, mn, s1, (long long)sh.tables, (int)sh.rows, sh.tables,
-                                                           sh.ldv / kBK, nb_rows, status);
-    count_launch(4);
-    return cudaGetLastError();
+    return e;
 }
 
 // ---------------------------------------------------------------------------------------------
