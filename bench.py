@@ -55,12 +55,13 @@ def parse_over(pairs):
     return over
 
 
-# Issue-slot use of the fused kernels (sm__throughput) from the ncu capture summarised in
+# Issue-slot use of the fused kernels (smsp__issue_active) from the ncu capture summarised in
 # profiles/fused_kernels_mid_L4.md; quoted beside the roofline fraction, not part of it.
-NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.636, "decode_kernel": 0.658}
+NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.649, "decode_kernel": 0.640}
 
 
-def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None):
+def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None,
+                   l1_gbs=None):
     """Roofline record of the fused predict + quantise + code kernels (the slower of the two).
     Two ceilings apply to a launch: HBM on the COMPULSORY bytes (KV once, bitstream once, every
     table once) and the plain fp32 ALUs on the mixture's K*d fused multiply-adds per vector; the
@@ -88,6 +89,12 @@ def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, 
          "northstar_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
                            "L1 / L2 hits, so this is an on-chip gather rate, not an HBM utilisation",
          "traffic": None if traffic_per_vector is None else traffic_per_vector[name] * vecs}
+    if l1_gbs:
+        gath = vecs * K * d * 2 / sec / 1e9
+        r["l1_gather"] = {"achieved": gath, "peak": l1_gbs, "unit": "GB/s", "frac": gath / l1_gbs,
+                          "peak_kind": "measured in this run: 128-bit loads that all hit L1, same launch shape",
+                          "note": "every gathered row (K*d*2 B per vector) reaches the registers through L1 whatever the hit "
+                                  "rate; an on-chip ceiling quoted beside the two above, not part of `frac`"}
     if alu_frac >= hbm_frac:
         r.update(bound="alu", achieved=flop_ach, peak=flop_peak, unit="TFLOP/s", frac=alu_frac)
     else:
@@ -138,7 +145,7 @@ class ClockSampler:
 # DRAM bytes per vector of the fused kernels, from the ncu capture summarised in
 # profiles/fused_kernels_mid_L4.md (dram__bytes_read.sum + dram__bytes_write.sum over 4.19 M vectors;
 # traffic grows in proportion to the vectors).  Valid for the default workload and chunk size only.
-NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.3, "decode_kernel": 431.9}
+NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.6, "decode_kernel": 433.2}
 NCU_TRAFFIC_NOTE = ("dram__bytes_read + dram__bytes_write of a 4-layer ncu capture (profiles/fused_kernels_mid_L4.md) "
                     "scaled by the vectors of a launch")
 
@@ -329,7 +336,8 @@ def run_codec(args, torch, plc, workloads, dev, name, over, steps, warmup, dist=
     default_kernels = name == "llama2-7b" and not over and variant == "topk" and not adaptive and not zero_rate and \
         not sigma_floor and layers is None
     roofline = fused_roofline(vecs, K, d, 0 if linear else T.numel() * 2, kv_bytes, payload_per_step, ek, dk, sm_mhz, sms, peak,
-                              peak_kind, NCU_DRAM_BYTES_PER_VECTOR if default_kernels else None)
+                              peak_kind, NCU_DRAM_BYTES_PER_VECTOR if default_kernels else None,
+                              plc.probe_l1_gbs() if variant == "topk" else None)
     if roofline["traffic"] is not None:
         roofline["traffic_note"] = NCU_TRAFFIC_NOTE
     if dense or linear:
