@@ -60,8 +60,7 @@ def parse_over(pairs):
 NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.649, "decode_kernel": 0.640}
 
 
-def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None,
-                   l1_gbs=None):
+def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None):
     """Roofline record of the fused predict + quantise + code kernels (the slower of the two).
     Two ceilings apply to a launch: HBM on the COMPULSORY bytes (KV once, bitstream once, every
     table once) and the plain fp32 ALUs on the mixture's K*d fused multiply-adds per vector; the
@@ -85,16 +84,12 @@ def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, 
          "fp32_fma": {"achieved": flop_ach, "peak": flop_peak, "unit": "TFLOP/s", "frac": alu_frac,
                       "peak_kind": "SMs x 128 lanes x 2 flop x sampled SM clock (%d x %.0f MHz)" % (sms, sm_mhz)},
          "issue_slot_use_ncu": NCU_ISSUE_SLOT_USE.get(name),
+         "busiest_units_ncu": "heavy half of the FMA pipe 66 %, L1 data pipe 60 %, issue slots 64 % "
+                              "(profiles/fused_kernels_mid_L4.md: no single unit saturated)",
          "northstar_bytes_frac": bytes_ns / sec / 1e9 / peak,
          "northstar_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
                            "L1 / L2 hits, so this is an on-chip gather rate, not an HBM utilisation",
          "traffic": None if traffic_per_vector is None else traffic_per_vector[name] * vecs}
-    if l1_gbs:
-        gath = vecs * K * d * 2 / sec / 1e9
-        r["l1_gather"] = {"achieved": gath, "peak": l1_gbs, "unit": "GB/s", "frac": gath / l1_gbs,
-                          "peak_kind": "measured in this run: 128-bit loads that all hit L1, same launch shape",
-                          "note": "every gathered row (K*d*2 B per vector) reaches the registers through L1 whatever the hit "
-                                  "rate; an on-chip ceiling quoted beside the two above, not part of `frac`"}
     if alu_frac >= hbm_frac:
         r.update(bound="alu", achieved=flop_ach, peak=flop_peak, unit="TFLOP/s", frac=alu_frac)
     else:
@@ -336,8 +331,7 @@ def run_codec(args, torch, plc, workloads, dev, name, over, steps, warmup, dist=
     default_kernels = name == "llama2-7b" and not over and variant == "topk" and not adaptive and not zero_rate and \
         not sigma_floor and layers is None
     roofline = fused_roofline(vecs, K, d, 0 if linear else T.numel() * 2, kv_bytes, payload_per_step, ek, dk, sm_mhz, sms, peak,
-                              peak_kind, NCU_DRAM_BYTES_PER_VECTOR if default_kernels else None,
-                              plc.probe_l1_gbs() if variant == "topk" else None)
+                              peak_kind, NCU_DRAM_BYTES_PER_VECTOR if default_kernels else None)
     if roofline["traffic"] is not None:
         roofline["traffic_note"] = NCU_TRAFFIC_NOTE
     if dense or linear:

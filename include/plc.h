@@ -370,11 +370,6 @@ plc_status plc_last_kernel_ms(plc_ctx* ctx, int32_t which, float* ms);
  * (each optional); reset != 0 then empties the log of that kind.  Meant to be called outside a
  * timed region: it synchronises with the recorded events. */
 plc_status plc_kernel_ms(plc_ctx* ctx, int32_t which, float* mean_ms, int32_t* launches, int32_t reset);
-/* Measurement aid for benchmarks: the rate (GB/s, whole GPU) at which L1 hits reach registers with
- * 128-bit loads in the fused kernels' launch shape -- the on-chip ceiling of the candidate-row gather
- * (K*d*2 bytes per vector come through L1 whatever the hit rate).  Allocates and frees a small buffer,
- * runs on the default stream and synchronises. */
-plc_status plc_probe_l1_gbs(float* gbs);
 /* Number of kernels this library has launched in this process (for benchmarks). */
 uint64_t plc_launch_count(void);
 

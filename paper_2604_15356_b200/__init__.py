@@ -24,7 +24,7 @@ EXPORTS = ["plc_create", "plc_destroy", "plc_reserve", "plc_topk_softmax", "plc_
            "plc_launch_count", "plc_rans_encode_static", "plc_encode_adaptive", "plc_decode_adaptive",
            "plc_trie_create", "plc_trie_destroy", "plc_trie_insert", "plc_trie_best_match", "plc_trie_evict",
            "plc_trie_stats", "plc_create_linear", "plc_prefix_clusters", "plc_rotq_record_bytes", "plc_encode_rotq",
-           "plc_decode_rotq", "plc_poll_status", "plc_last_schedule", "plc_kernel_ms", "plc_probe_l1_gbs"]
+           "plc_decode_rotq", "plc_poll_status", "plc_last_schedule", "plc_kernel_ms"]
 
 
 def sources():
@@ -424,13 +424,6 @@ def build_table(qp):
     _check(lib().plc_build_table(int(qp), f.ctypes.data_as(C.c_void_p), c.ctypes.data_as(C.c_void_p)),
            "plc_build_table")
     return f, c
-
-
-def probe_l1_gbs():
-    """Measured L1 -> register rate of the whole GPU in GB/s (128-bit loads, all hits)."""
-    g = C.c_float()
-    _check(lib().plc_probe_l1_gbs(C.byref(g)), "plc_probe_l1_gbs")
-    return g.value
 
 
 def launch_count():

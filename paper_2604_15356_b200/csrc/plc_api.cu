@@ -658,29 +658,6 @@ plc_status plc_last_schedule(const plc_ctx* c, int32_t* n_queues, int32_t* sms_p
     return PLC_OK;
 }
 
-plc_status plc_probe_l1_gbs(float* gbs) {
-    if (!gbs) return PLC_E_INVALID;
-    const size_t bytes = l1_probe_bytes();
-    void* buf = nullptr;
-    cudaEvent_t e0 = nullptr, e1 = nullptr;
-    plc_status rc = PLC_E_CUDA;
-    const int iters = 2000;
-    float ms = 0.f;
-    if (cudaMalloc(&buf, bytes) == cudaSuccess && cudaMemset(buf, 0, bytes) == cudaSuccess &&
-        cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess &&
-        launch_l1_probe(buf, 50, buf, 0) == cudaSuccess &&                       // warm-up
-        cudaEventRecord(e0, 0) == cudaSuccess && launch_l1_probe(buf, iters, buf, 0) == cudaSuccess &&
-        cudaEventRecord(e1, 0) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
-        cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && ms > 0.f) {
-        *gbs = (float)((double)bytes * iters / (ms * 1e-3) / 1e9);
-        rc = PLC_OK;
-    }
-    if (e0) cudaEventDestroy(e0);
-    if (e1) cudaEventDestroy(e1);
-    cudaFree(buf);
-    return rc;
-}
-
 plc_status plc_set_profiling(plc_ctx* c, int32_t on) {
     if (!c) return PLC_E_INVALID;
     c->profiling = on != 0;

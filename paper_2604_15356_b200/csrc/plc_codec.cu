@@ -957,23 +957,6 @@ __global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecAr
     }
 }
 
-// Measurement aid: every warp re-reads its own 4 KB of a buffer with 128-bit loads, so that after the
-// first touch all loads are L1 hits; bytes / time is the rate at which an SM's L1 feeds registers when
-// all SMs run the fused kernels' launch shape (the ceiling of the row gather).
-__global__ void __launch_bounds__(kThreads, kBlocksPerSM) l1_probe_kernel(const uint4* __restrict__ buf, int iters, uint4* __restrict__ sink) {
-    const uint4* mine = buf + ((size_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * 256 + (threadIdx.x & 31);
-    uint4 acc = make_uint4(0u, 0u, 0u, 0u);
-    for (int it = 0; it < iters; ++it) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint4 r;
-            asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(mine + 32 * j));
-            acc.x ^= r.x; acc.y ^= r.y; acc.z ^= r.z; acc.w ^= r.w;
-        }
-    }
-    if (acc.x == 0x9e3779b9u && acc.y == 0x7f4a7c15u) sink[blockIdx.x * kThreads + threadIdx.x] = acc;   // keeps the loads alive
-}
-
 template <class F>
 cudaError_t dispatch_d(int d, F&& f) {
     switch (d) {
@@ -1032,14 +1015,6 @@ static void set_queues(CodecArgs& a, int n_tables) {
     int nq = (sms + (int)g - 1) / (int)g;
     nq = std::max(1, std::min(nq, std::min(n_tables, kTicketWords)));
     a.sched_g = (int)g; a.sched_nq = nq;
-}
-
-size_t l1_probe_bytes() { return (size_t)sm_count() * kBlocksPerSM * kThreads * sizeof(uint4) * 8; }
-
-cudaError_t launch_l1_probe(const void* buf, int iters, void* sink, cudaStream_t st) {
-    l1_probe_kernel<<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(static_cast<const uint4*>(buf), iters, static_cast<uint4*>(sink));
-    count_launch();
-    return cudaGetLastError();
 }
 
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st) {

@@ -255,8 +255,6 @@ cudaError_t linear_layer(const __half* A_layer, const LinearShape& sh, uint8_t* 
 cudaError_t dense_layer(const __half* T_layer, const DenseShape& sh, uint8_t* scratch, const size_t* off,
                         unsigned int* status, cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1);   // events bracket the contraction
 cudaError_t launch_rownorm(const __half* T, float* out, long long rows, int d, cudaStream_t st);
-size_t l1_probe_bytes();                          // bytes the L1 probe reads per sweep (= size of its buffer)
-cudaError_t launch_l1_probe(const void* buf, int iters, void* sink, cudaStream_t st);
 cudaError_t launch_encode(const CodecArgs& a, cudaStream_t st);
 cudaError_t launch_decode(const CodecArgs& a, cudaStream_t st);
 cudaError_t launch_append_quantise(const CodecArgs& a, cudaStream_t st);   // predict + quantise into the open chunk
