@@ -218,7 +218,7 @@ def shard_slots(S, L, H, mc, world, rank):
 
 def run_codec(args, torch, plc, workloads, dev, name, over, steps, warmup, dist=None, world=1, rank=0,
               variant="topk", d_model=4096, adaptive_b0=0, zero_rate=0.0, sigma_floor=0.0, shard=None,
-              want_e2e=False, want_cpu=False, e2e_steps=2, e2e_groups=4, w=None, layers=None):
+              want_e2e=False, want_cpu=False, e2e_steps=4, e2e_groups=4, w=None, layers=None):
     """Times `steps` passes (encode then decode) of workload `name` after `warmup` untimed ones and
     returns (line, workload).  `w` reuses a workload already built; `layers` = (lo, hi) restricts the
     run to a slice of its layers (views, nothing is copied)."""
@@ -420,7 +420,7 @@ def main():
                          "GPU, a compact record of every benchmark configuration (see --no-configs)")
     ap.add_argument("--no-configs", action="store_true", help="default run: headline only")
     ap.add_argument("--chunk-pos", type=int, default=None)
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--e2e-groups", type=int, default=4, help="layer groups (streams) of the host-buffer step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -778,7 +778,9 @@ def run_e2e(torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None
     """Same step with HOST buffers: pinned inputs are copied in, the coded bytes and index are
     copied out and back in, the decoded KV is copied out -- all inside the timed region.  The
     layers are cut into groups, each with its own context and CUDA stream, so that the copies of
-    one group overlap the kernels and the opposite-direction copies of the others."""
+    one group overlap the kernels and the opposite-direction copies of the others; consecutive steps
+    are not joined (a step's output copies run beside the next step's input copies), only the end of
+    the timed region is."""
     cfg = w["cfg"]
     S, n, L, H, d = cfg["S"], cfg["n"], cfg["L"], cfg["H"], cfg["d"]
     G = groups if L % groups == 0 else 1
@@ -786,7 +788,8 @@ def run_e2e(torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None
     kv_h = w["kv"].cpu().pin_memory()
     lg_h = w["logits"].cpu().pin_memory()
     kvo_h = torch.empty_like(kv_h).pin_memory()
-    kv_d, lg_d, out_d = torch.empty_like(w["kv"]), torch.empty_like(w["logits"]), torch.empty_like(w["kv"])
+    kv_d, out_d = torch.empty_like(w["kv"]), torch.empty_like(w["kv"])
+    lg_d = [torch.empty_like(w["logits"]), torch.empty_like(w["logits"])]   # steps alternate between two logits buffers
     ctxs, sts, pay_h, off_h, nby_h, tot_h, streams = [], [], [], [], [], [], []
     for g in range(G):
         c = make_ctx(w["T"][g * Lg:(g + 1) * Lg])
@@ -799,19 +802,27 @@ def run_e2e(torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None
         nby_h.append(torch.empty_like(st.chunk_bytes, device="cpu").pin_memory())
         tot_h.append(torch.zeros(1, dtype=torch.int64).pin_memory())
         streams.append(torch.cuda.Stream(device=dev))
-    ev0 = torch.cuda.Event()
+    copy_stream = torch.cuda.Stream(device=dev)
+    ev_lg = [torch.cuda.Event(), torch.cuda.Event()]
+    done = [[torch.cuda.Event() for _ in range(G)] for _ in range(2)]
 
-    def step():
-        main = torch.cuda.current_stream()
-        lg_d.copy_(lg_h, non_blocking=True)
-        ev0.record(main)
+    def step(i):
+        """Step i.  Nothing joins the groups between steps: a group goes on to the next step's input copy
+        as soon as its own output copy is queued, so one group's device-to-host copy of decoded KV runs
+        beside another group's host-to-device copy of the next step's input."""
+        b = i & 1
+        with torch.cuda.stream(copy_stream):
+            for g in range(G):
+                copy_stream.wait_event(done[b][g])            # step i - 2 is through with this logits buffer
+            lg_d[b].copy_(lg_h, non_blocking=True)
+            ev_lg[b].record(copy_stream)
         for g in range(G):
             lo, hi = g * Lg, (g + 1) * Lg
             with torch.cuda.stream(streams[g]):
-                streams[g].wait_event(ev0)
+                streams[g].wait_event(ev_lg[b])
                 kv_d[lo:hi].copy_(kv_h[lo:hi], non_blocking=True)
                 sts[g].total_bytes.zero_()
-                ctxs[g].encode(kv_d[lo:hi], lg_d, sts[g], tokens=tok)
+                ctxs[g].encode(kv_d[lo:hi], lg_d[b], sts[g], tokens=tok)
                 tot_h[g].copy_(sts[g].total_bytes, non_blocking=True)
         used_all = 0
         for g in range(G):
@@ -824,27 +835,38 @@ def run_e2e(torch, plc, make_ctx, w, dev, world, dist, tokens_per_step, tok=None
                 off_h[g].copy_(st.chunk_offset, non_blocking=True); nby_h[g].copy_(st.chunk_bytes, non_blocking=True)
                 st.payload[:used].copy_(pay_h[g][:used], non_blocking=True)
                 st.chunk_offset.copy_(off_h[g], non_blocking=True); st.chunk_bytes.copy_(nby_h[g], non_blocking=True)
-                ctxs[g].decode(st, lg_d, out_d[lo:hi], tokens=tok)
+                ctxs[g].decode(st, lg_d[b], out_d[lo:hi], tokens=tok)
                 kvo_h[lo:hi].copy_(out_d[lo:hi], non_blocking=True)
-        for g in range(G):
-            main.wait_stream(streams[g])
+                done[b][g].record(streams[g])
         return used_all
 
-    used = step()
+    def join():
+        main = torch.cuda.current_stream()
+        for g in range(G):
+            main.wait_stream(streams[g])
+
+    used = step(0)
+    join()
     torch.cuda.synchronize()
     for c in ctxs:
         assert c.sync_status() == plc.OK
     err = float((kvo_h[:, :, :, :, :64].float() - kv_h[:, :, :, :, :64].float()).abs().max())
     assert err <= cfg["delta"] * (2.0 ** (adaptive_b0 - 1) if adaptive_b0 > 0 else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
+    kvo_h.zero_()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(e2e_steps):
-        used = step()
+    for i in range(e2e_steps):
+        used = step(i + 1)
+    join()
     t1.record()
     torch.cuda.synchronize()
+    for c in ctxs:
+        assert c.sync_status() == plc.OK
+    err = float((kvo_h[:, :, :, :, -64:].float() - kv_h[:, :, :, :, -64:].float()).abs().max())     # the last timed step's output
+    assert err <= cfg["delta"] * (2.0 ** (adaptive_b0 - 1) if adaptive_b0 > 0 else 1.0) / 2 + 1e-3 + 8 * 2 ** -11, err
     ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps, dist, dev)
     idx_bytes = sum(o.numel() * 8 + b.numel() * 4 for o, b in zip(off_h, nby_h))
     return {"value": tokens_per_step / (ms / 1e3) if sharded else job_value(world, tokens_per_step, ms), "unit": UNIT,
