@@ -86,8 +86,8 @@ def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, 
          "issue_slot_use_ncu": NCU_ISSUE_SLOT_USE.get(name),
          "busiest_units_ncu": "heavy half of the FMA pipe 66 %, L1 data pipe 60 %, issue slots 64 % "
                               "(profiles/fused_kernels_mid_L4.md: no single unit saturated)",
-         "northstar_bytes_frac": bytes_ns / sec / 1e9 / peak,
-         "northstar_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
+         "gathered_row_bytes_frac": bytes_ns / sec / 1e9 / peak,
+         "gathered_row_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
                            "L1 / L2 hits, so this is an on-chip gather rate, not an HBM utilisation",
          "traffic": None if traffic_per_vector is None else traffic_per_vector[name] * vecs}
     if alu_frac >= hbm_frac:

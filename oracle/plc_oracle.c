@@ -26,8 +26,8 @@
  *   best-match lookup = deepest stored ancestor ....... Sec. 7.3 (trie-based prefix index)
  *   per-vector quantiser on the residual .............. Prop. 3, step 3 (rotated fixed-rate quantiser)
  * The paper names no entropy coder beyond "standard source coding" (Prop. 2, proof); the coder
- * below (uniform step, discretised-Laplace model, 32-lane interleaved rANS) is this build's
- * stated reading and is defined in full in the comments of each function.
+ * below (uniform step, discretised-Laplace model, 32-lane interleaved rANS) is the
+ * stated reading of this codec and is defined in full in the comments of each function.
  */
 #include <math.h>
 #include <stdint.h>
@@ -295,7 +295,7 @@ void plo_reconstruct(const double* mu, const int32_t* sym, int d, float delta, f
 /* ---------------------------------------------------------------- rotated fixed-rate quantiser */
 
 /* Prop. 3, step 3: "any per-vector quantizer" applied to R_i.  Besides the entropy-coded uniform
- * quantiser above, this build offers the generic member of the family the paper points to (a
+ * quantiser above, the codec offers the generic member of the family the paper points to (a
  * random rotation followed by a b-bit scalar quantiser; the paper gives no details of TurboQuant,
  * so nothing of it is reproduced here).  For one residual vector r of d = 2^m components:
  *   x_j = eps_j r_j                          eps_j = -1 where neg[j] != 0, else +1   (input to the method)
