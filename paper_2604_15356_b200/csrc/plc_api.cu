@@ -18,6 +18,7 @@ struct plc_ctx {
     const __half* T;
     float* rownorm2;
     int2* pairs;
+    uint8_t* cand;                  // [positions] candidate lists + headers of the two-kernel selection
     int* step_exp;                  // [positions] adaptive step exponents
     long long pairs_cap;            // positions
     uint16_t* staging;
@@ -102,15 +103,29 @@ int padded_k(const plc_config& cfg) {
     return (cfg.top_k + rows - 1) / rows * rows;
 }
 
+// Scratch of the two-kernel selection: headers first (16 bytes per row), then the lists.
+size_t cand_word_bytes(const plc_config& cfg) { return cfg.vocab <= 65536 ? 4 : 8; }
+size_t cand_bytes(const plc_config& cfg, long long positions) {
+    return (size_t)positions * (16 + (size_t)kTopkListCap * cand_word_bytes(cfg));
+}
+void set_cand(const plc_ctx* c, TopkArgs& a, long long positions);
+
 plc_status ensure_pairs(plc_ctx* c, long long positions) {
     if (positions <= c->pairs_cap) return PLC_OK;
     if (c->pairs) cudaFree(c->pairs);
     if (c->step_exp) cudaFree(c->step_exp);
-    c->pairs = nullptr; c->step_exp = nullptr; c->pairs_cap = 0;
+    if (c->cand) cudaFree(c->cand);
+    c->pairs = nullptr; c->step_exp = nullptr; c->cand = nullptr; c->pairs_cap = 0;
     if (cudaMalloc(&c->pairs, sizeof(int2) * (size_t)positions * padded_k(c->cfg)) != cudaSuccess) return PLC_E_CUDA;
     if (cudaMalloc(&c->step_exp, sizeof(int) * (size_t)positions) != cudaSuccess) return PLC_E_CUDA;
+    if (cudaMalloc(&c->cand, cand_bytes(c->cfg, positions)) != cudaSuccess) return PLC_E_CUDA;
     c->pairs_cap = positions;
     return PLC_OK;
+}
+
+void set_cand(const plc_ctx* c, TopkArgs& a, long long positions) {
+    a.cand_hdr = reinterpret_cast<float4*>(c->cand);
+    a.cand = c->cand + (size_t)positions * 16;
 }
 
 CodecArgs base_args(const plc_ctx* c) {
@@ -258,7 +273,7 @@ static plc_status create_common(plc_ctx** out, const plc_config* cfg, const void
 
 plc_status plc_destroy(plc_ctx* c) {
     if (!c) return PLC_E_INVALID;
-    cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->step_exp); cudaFree(c->staging);
+    cudaFree(c->rownorm2); cudaFree(c->pairs); cudaFree(c->cand); cudaFree(c->step_exp); cudaFree(c->staging);
     cudaFree(c->ticket); cudaFree(c->status); cudaFree(c->counters); cudaFree(c->dense_scratch); cudaFree(c->lin_model);
     for (int k = 0; k < 3; ++k)
         for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
@@ -285,6 +300,11 @@ plc_status plc_topk_softmax(plc_ctx* c, const void* logits_dev, const int32_t* t
     a.V = c->cfg.vocab; a.K = c->cfg.top_k;
     a.idx = idx_dev; a.w = w_dev; a.lse = lse_dev; a.zk = zk_dev; a.logp2 = logp2_dev;
     a.n_per_session = 1;
+    if (idx_dev || w_dev || zk_dev) {                    // the selection uses the context's scratch
+        plc_status rc = ensure_pairs(c, N);
+        if (rc) return rc;
+        set_cand(c, a, c->pairs_cap);
+    }
     return launch_topk(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PLC_OK : PLC_E_CUDA;
 }
 
@@ -313,6 +333,7 @@ static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n,
     TopkArgs a{};
     a.logits = static_cast<const __half*>(logits_dev); a.N = (long long)S * n; a.V = c->cfg.vocab; a.K = c->cfg.top_k;
     a.pairs = c->pairs; a.Kp = padded_k(c->cfg); a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
+    set_cand(c, a, c->pairs_cap);
     if (tokens) {
         a.tokens = tokens; a.step_exp = c->step_exp; a.bits_out = bits_out;
         a.b0 = c->cfg.adaptive_b0; a.extra = c->cfg.adaptive_extra; a.hbar = c->cfg.adaptive_hbar;

@@ -156,7 +156,12 @@ struct TopkArgs {
     int* step_exp; int* bits_out; int b0, extra; float hbar;
     // Rows are skipped (nothing written) when pos ranges are given and the row is outside them.
     int n_per_session; const int32_t* pos_begin; const int32_t* pos_end;
+    // Optional scratch of the two-kernel selection: per row kTopkListCap order words (8 bytes each, 4 while
+    // V <= 65536) and a header {l_max, sum of exp(l - l_max), number of candidates or -1}.  With it
+    // the streaming kernel only collects the candidates of a row and a second kernel ranks them.
+    void* cand; float4* cand_hdr;
 };
+constexpr int kTopkListCap = 256;
 cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st);
 
 cudaError_t launch_prefix_dedup(const int32_t* tokens, const int32_t* lens, const float* logp2, int S, int64_t stride,

@@ -5,12 +5,17 @@
 // maximum per thread; the ceil(K / warps)-th largest thread maximum of every warp, minimised over the
 // warps, is a value with at least K row elements at or above it, i.e. a lower bound of the K-th
 // largest logit that needs no histogram.  Pass 1 (served by L2) sums exp(l - l_max) over the row
-// and collects the few elements at or above that bound (typically 1.2-2 K of them); they are ranked
-// by counting (long lists: sorted), which yields the K selected in their final order.  Rows whose
+// and notes the groups of 8 logits that hold an element at or above that bound; after the pass the
+// noted groups are taken apart, one per thread, into a candidate list (typically 1.2-2 K entries).
+// A list of at most 256 goes to global memory and a second kernel (one warp per row, bitonic sort in
+// registers) orders it and writes the K selected, their weights and Z_k; without the scratch for
+// that, or for longer lists, the block ranks by counting (long lists: sorted) itself.  Rows whose
 // candidates overflow the list (large tie groups, adversarial layouts) and larger K take the radix-select path:
 // a 4096-bin histogram of the order-preserving 16-bit key finds the bin that holds the K-th largest,
 // a 16-way refinement finds the key itself, and equal keys are taken in index order.
 // Reductions use warp shuffles in a fixed order, so results are bit-reproducible from run to run.
+#include <type_traits>
+
 #include "plc_common.cuh"
 
 namespace plc {
@@ -45,7 +50,7 @@ struct __align__(16) Smem {
     uint32_t red_t[THREADS / 32];
     float red_s[THREADS / 32];
     int scan[THREADS / 32];
-    int nsel, ncand, bstar, count_above, cstar, thr, need, neq, running, nlist;
+    int nsel, ncand, bstar, count_above, cstar, thr, need, neq, running, nlist, nhit;
     float row_max, row_sum, sum_k;
     uint32_t theta;
 };
@@ -312,7 +317,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
             if (i < b || i >= e) continue;
         }
         const __half* row = a.logits + rowi * (long long)V;
-        if (tid == 0) sm.nlist = 0;
+        if (tid == 0) { sm.nlist = 0; sm.nhit = 0; }
 
         // Pass 0 (HBM): one maximum per thread.
         uint32_t tkey = 0;
@@ -372,10 +377,12 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
                         s += exp_rel(f.x, nb);
                         s += exp_rel(f.y, nb);
                     }
-                    // collect unless both halves of the pairwise maximum are below the bound
+                    // A group of 8 with a logit at or above the bound is only noted here (few lanes get
+                    // here, so anything longer would run once per group with the rest of the warp idle);
+                    // the noted groups are taken apart after the pass, one per thread.
                     if (fast && !__hblt2(*reinterpret_cast<const __half2*>(&top), *reinterpret_cast<const __half2*>(&th2))) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) collect2(wds[j], th2, i0 + 2 * j, narrow, &sm.nlist, sm.hist);
+                        const int slot = atomicAdd(&sm.nhit, 1);
+                        if (slot < kCandCap) sm.sel_idx[slot] = i0;          // sel_idx is idle on this path
                     }
                 }
             }
@@ -396,8 +403,38 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         float sum_all = 0.f;
 #pragma unroll
         for (int w = 0; w < NW; ++w) sum_all += sm.red_s[w];
+        if (VEC && fast) {
+            const int nhit = sm.nhit;
+            if (nhit > kCandCap) {
+                if (tid == 0) sm.nlist = kCandCap + 1;                    // too many: the radix select takes the row
+            } else {
+                const uint32_t tb = bits_of_key(theta);
+                const uint32_t th2 = tb | (tb << 16);
+                for (int t = tid; t < nhit; t += THREADS) {
+                    const int i0 = sm.sel_idx[t];
+                    const uint4 r = *reinterpret_cast<const uint4*>(row + i0);
+                    const uint32_t wds[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) collect2(wds[j], th2, i0 + 2 * j, narrow, &sm.nlist, sm.hist);
+                }
+            }
+            __syncthreads();
+        }
         const int nlist = sm.nlist;
-        if (fast && nlist >= K && nlist <= kCandCap) {
+        // Two-kernel selection: a list that one warp can sort goes to global memory as it is and
+        // topk_rank_kernel finishes the row (order, weights, Z_k); everything else stays here.
+        const bool handed = fast && a.cand && K <= 128 && nlist >= K && nlist <= kTopkListCap;
+        if (a.cand_hdr && tid == 0)
+            a.cand_hdr[rowi] = make_float4(lmax, sum_all, __int_as_float(handed ? nlist : -1), 0.f);
+        if (handed) {
+            if (narrow) {
+                uint32_t* dst = static_cast<uint32_t*>(a.cand) + rowi * kTopkListCap;
+                for (int c = tid; c < nlist; c += THREADS) dst[c] = list32[c];
+            } else {
+                unsigned long long* dst = static_cast<unsigned long long*>(a.cand) + rowi * kTopkListCap;
+                for (int c = tid; c < nlist; c += THREADS) dst[c] = list64[c];
+            }
+        } else if (fast && nlist >= K && nlist <= kCandCap) {
             // Order the candidates (at least K of them); the first K are the result.  Short lists are
             // ranked by counting (n^2 / THREADS compares per thread, no barriers), long ones sorted.
             constexpr int kRankMax = 192;
@@ -449,7 +486,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         }
 
         float sum_k = 0.f;
-        if (select) {
+        if (select && !handed) {
             for (int k = tid; k < K; k += THREADS) sm.ek[k] = expf(val_of_key(sm.cand_key[k]) - lmax);
             __syncthreads();
             if (wid == 0) {
@@ -473,7 +510,7 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
         if (tid == 0) {
             float lse = lmax + logf(sum_all);
             if (a.lse) a.lse[rowi] = lse;
-            if (a.zk) a.zk[rowi] = sum_k / sum_all;
+            if (a.zk && !handed) a.zk[rowi] = sum_k / sum_all;
             if (a.tokens && (a.logp2 || a.step_exp || a.bits_out)) {
                 const int tk = a.tokens[rowi];
                 const float v = (tk >= 0 && tk < V) ? (__half2float(row[tk]) - lse) * 1.44269504088896341f : __int_as_float(0x7fc00000);
@@ -489,6 +526,98 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
             }
         }
         __syncthreads();
+    }
+}
+
+// One compare-exchange step of a bitonic network on 256 order words held 8 per lane: word e = r * 32 +
+// lane sits in v[r].  K2 = the size of the bitonic blocks being merged, J = the distance.  The
+// network sorts descending overall.
+template <class W, int K2, int J>
+__device__ __forceinline__ void bitonic_step(W (&v)[8], int lane) {
+    if constexpr (J >= 32) {
+        constexpr int RJ = J >> 5;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if ((r & RJ) == 0) {
+                const bool desc = (((r * 32) & K2) == 0) || K2 == 256;       // K2 >= 64 here: the bit of e lies in r
+                const W x = v[r], y = v[r | RJ];
+                const bool sw = desc ? (x < y) : (x > y);
+                v[r] = sw ? y : x; v[r | RJ] = sw ? x : y;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const W p = __shfl_xor_sync(kFull, v[r], J);
+            const int e = r * 32 + lane;
+            const bool lower = (lane & J) == 0;
+            const bool desc = K2 == 256 || (e & K2) == 0;
+            const bool keep_max = lower == desc;
+            const W mx = v[r] > p ? v[r] : p, mn = v[r] > p ? p : v[r];
+            v[r] = keep_max ? mx : mn;
+        }
+    }
+}
+template <class W, int K2, int J>
+__device__ __forceinline__ void bitonic_merge(W (&v)[8], int lane) {
+    bitonic_step<W, K2, J>(v, lane);
+    if constexpr (J > 1) bitonic_merge<W, K2, J / 2>(v, lane);
+}
+template <class W, int K2>
+__device__ __forceinline__ void bitonic_sort256(W (&v)[8], int lane) {
+    if constexpr (K2 > 2) bitonic_sort256<W, K2 / 2>(v, lane);
+    bitonic_merge<W, K2, K2 / 2>(v, lane);
+}
+
+// Second kernel of the two-kernel selection: one warp per row sorts the row's candidate list (at
+// most 256 order words, larger = earlier in (logit descending, index ascending)) in registers and
+// writes what the streaming kernel would have written for the first K: order, renormalised weights
+// (the same sums in the same order), Z_k.  Rows the streaming kernel finished itself carry -1.
+template <bool NARROW>
+__global__ void __launch_bounds__(256) topk_rank_kernel(TopkArgs a) {
+    using W = std::conditional_t<NARROW, uint32_t, unsigned long long>;
+    const int lane = threadIdx.x & 31, K = a.K;
+    const long long warp = (long long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long long)gridDim.x * 8;
+    for (long long rowi = warp; rowi < a.N; rowi += nw) {
+        if (a.pos_begin || a.pos_end) {
+            int s = (int)(rowi / a.n_per_session), i = (int)(rowi % a.n_per_session);
+            int b = a.pos_begin ? a.pos_begin[s] : 0, e = a.pos_end ? a.pos_end[s] : a.n_per_session;
+            if (i < b || i >= e) continue;
+        }
+        const float4 hdr = a.cand_hdr[rowi];
+        const int nlist = __float_as_int(hdr.z);
+        if (nlist < 0) continue;
+        const W* src = static_cast<const W*>(a.cand) + rowi * kTopkListCap;
+        W v[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v[r] = r * 32 + lane < nlist ? src[r * 32 + lane] : (W)0;   // 0 orders after everything
+        bitonic_sort256<W, 256>(v, lane);
+        const float lmax = hdr.x;
+        float ek[4];
+        int idx[4];
+        float p = 0.f;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {                   // K <= 128: the first K words sit in v[0..3]
+            const uint32_t key = NARROW ? (uint32_t)(v[r] >> 16) : (uint32_t)((unsigned long long)v[r] >> 32);
+            idx[r] = NARROW ? (int)(0xffffu - ((uint32_t)v[r] & 0xffffu)) : (int)(0xffffffffu - (uint32_t)v[r]);
+            ek[r] = r * 32 + lane < K ? expf(val_of_key(key) - lmax) : 0.f;
+            if (r * 32 + lane < K) p += ek[r];
+        }
+        const float sum_k = warp_sum(p);
+        const int idx0 = __shfl_sync(kFull, idx[0], 0);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int k = r * 32 + lane;
+            if (k < K) {
+                const float w = ek[r] / sum_k;
+                if (a.pairs) a.pairs[rowi * a.Kp + k] = make_int2(idx[r], __float_as_int(w));
+                if (a.idx) a.idx[rowi * K + k] = idx[r];
+                if (a.w) a.w[rowi * K + k] = w;
+            }
+        }
+        if (a.pairs)
+            for (int k = K + lane; k < a.Kp; k += 32) a.pairs[rowi * a.Kp + k] = make_int2(idx0, 0);
+        if (a.zk && lane == 0) a.zk[rowi] = sum_k / hdr.y;
     }
 }
 
@@ -519,7 +648,18 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
         else launch(topk_softmax_kernel<false, 256>, 256, 5);
     }
     count_launch();
-    return cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const bool select = a.pairs || a.idx || a.w || a.zk;
+    if (a.cand && a.cand_hdr && select && a.K <= 128) {
+        const long long want = (a.N + 7) / 8, cap = (long long)sms * 8;
+        const unsigned blocks = (unsigned)(want < cap ? want : cap);
+        if (a.V <= 65536) topk_rank_kernel<true><<<blocks, 256, 0, st>>>(a);
+        else topk_rank_kernel<false><<<blocks, 256, 0, st>>>(a);
+        count_launch();
+        e = cudaGetLastError();
+    }
+    return e;
 }
 
 }  // namespace plc
