@@ -167,9 +167,11 @@ def gpu_decode_check(g, kv, delta, n, pos_begin=None, pos_end=None, out_dtype=pl
 def test_topk_softmax_parity(dev, orc):
     rng = np.random.default_rng(0)
     # the last three shapes have rows longer than 128 KB (the kernel's wide blocks), vectorised and not;
-    # K = 300 and K = 1024 are beyond the per-thread-maximum bound and take the radix-select path
+    # K = 300 and K = 1024 are beyond the per-thread-maximum bound and take the radix-select path; K up to 128 on
+    # ordinary rows hands the candidate list to the ranking kernel (32-bit order words up to V = 65536, 64-bit beyond)
     for V, K, N in [(256, 16, 40), (32000, 64, 24), (1000, 64, 16), (37, 5, 9), (4096, 1, 8), (2048, 1024, 4),
-                    (32000, 256, 6), (8192, 300, 5), (70008, 64, 7), (65541, 40, 6), (128256, 256, 5)]:
+                    (32000, 256, 6), (8192, 300, 5), (70008, 64, 7), (65541, 40, 6), (128256, 256, 5),
+                    (32000, 128, 9), (32000, 100, 9), (128256, 64, 6), (4096, 128, 8)]:
         lg = (rng.standard_normal((N, V)) * 2.5).astype(np.float16)
         lg[1, :] = np.float16(0.25)                              # every logit equal
         lg[2, ::2] = lg[2, 0]                                    # half the row tied at one value
@@ -192,6 +194,37 @@ def test_topk_softmax_parity(dev, orc):
         only = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev), want=("lse", "logp2"))
         assert set(only) == {"lse", "logp2"}                      # no selected set asked for: the selection is skipped
         assert torch.equal(only["lse"], out["lse"]) and torch.equal(only["logp2"], out["logp2"])
+
+
+def test_status_and_profiling_read_outs(dev):
+    """The small read-out calls: status polling does not clear, the kernel-time log counts launches and
+    resets, the work-queue layout is reported after a top-K encode."""
+    tokens, logits, T, kv = make_workload(21, 1, 64, 1, 2, 128, 512, 32)
+    ctx = plc.Context(T.to(dev), 32, 0.02, chunk_pos=32)
+    with pytest.raises(plc.PlcError) as e:
+        ctx.last_schedule()                                        # nothing launched yet
+    assert e.value.code == plc.E_STATE
+    assert ctx.poll_status() == (plc.OK, 0)
+    ctx.set_profiling(True)
+    st = plc.StreamSet(ctx.W, 2, 3 * 64 * ctx.W * 128 + 4096, dev)
+    kvd, lgd = kv.to(dev), logits.to(dev)
+    for _ in range(3):
+        st.total_bytes.zero_()
+        ctx.encode(kvd, lgd, st)
+    ms, n = ctx.kernel_ms(0)
+    assert n == 3 and ms > 0 and ctx.kernel_ms(1) == (0.0, 0)
+    assert abs(ctx.last_kernel_ms(0) - ms) < 10 * ms
+    assert ctx.kernel_ms(0, reset=True)[1] == 3 and ctx.kernel_ms(0)[1] == 0
+    nq, g = ctx.last_schedule()
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    assert nq >= 1 and 1 <= g <= sms
+    # a damaged chunk: the poll sees the bit and leaves it, the synchronous read clears it
+    out = torch.zeros(kv.shape, dtype=torch.float32, device=dev)
+    st.chunk_bytes[0] = int(st.chunk_bytes[0]) - 40
+    ctx.decode(st, lgd, out)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == (plc.E_CORRUPT, 2) and ctx.poll_status() == (plc.E_CORRUPT, 2)
+    assert ctx.sync_status() == plc.E_CORRUPT and ctx.poll_status() == (plc.OK, 0)
 
 
 def test_tiny_config_full_parity(dev, orc):
