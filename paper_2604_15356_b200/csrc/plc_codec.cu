@@ -41,6 +41,8 @@ struct Geo {
     static constexpr int ROWS = 32 / R;    // rows fetched by one warp-wide load
 };
 
+// Encoder tables are indexed by hi + 31 (hi in [-31, 31]; entry 63 = escape): the symbol's place in
+// the alphabet (0, +1, -1, +2, ...) only matters for the cumulative counts, which are kept.
 struct EncTables { EncEntry enc[kNumTables][kNumSym]; };
 // Decoder tables: cum[] for the search, fc[] = f | (c << 16) for the state update.
 struct DecTables { uint16_t cum[kNumTables][kNumSym + 2]; uint32_t fc[kNumTables][kNumSym]; };
@@ -52,8 +54,10 @@ __device__ inline void build_enc_tables(EncTables* t) {
         uint32_t c = 0;
         for (int i = 0; i < kNumSym; ++i) {
             uint32_t fi = f[i];
-            t->enc[id][i].rcp = fi == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / fi);
-            t->enc[id][i].fc = fi | (c << 16);
+            const int hi = (i & 1) ? (i + 1) / 2 : -(i / 2);            // alphabet order 0, +1, -1, +2, ...
+            const int at = i == kEsc ? kEsc : hi + kHiMax;
+            t->enc[id][at].rcp = fi == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / fi);
+            t->enc[id][at].fc = fi | (c << 16);
             c += fi;
         }
     }
@@ -223,10 +227,9 @@ __device__ __forceinline__ int encode_step(int sym, int s_dyn, const EncEntry* t
     const int S2 = 2 * S;
     const int u = sym + (S ? (1 << (S - 1)) : 0);                  // |sym| <= 2^30, S <= 15: no overflow
     const int hi = u >> S;                                         // bits below S of u are the raw part
-    const int nh = -hi;
-    const uint32_t zz0 = (uint32_t)((nh << 1) ^ (nh >> 31));       // 0, +1 -> 1, -1 -> 2, +2 -> 3, ...
-    const bool esc = zz0 > 2u * kHiMax;                            // |hi| > 31
-    const EncEntry e = tbl[min(zz0, (uint32_t)kEsc)];
+    const uint32_t at = (uint32_t)(hi + kHiMax);
+    const bool esc = at > 2u * kHiMax;                             // |hi| > 31
+    const EncEntry e = tbl[min(at, (uint32_t)kEsc)];
     const uint32_t f = e.fc & 0xffffu;
     const bool emit = x >= (f << 17);
     const uint32_t emask = __ballot_sync(kFull, emit);
@@ -559,7 +562,9 @@ __device__ __forceinline__ void dense_finish(const CodecArgs& a, int t_local, in
 enum { kSrcGather = 0, kSrcOpen = 1, kSrcDense = 2 };
 
 // ZR: the zero-rate rule (Thm. 3) is on; a separate instantiation keeps the plain coder's loop free of it.
-template <int D, int SRC, bool ZR>
+// FLEX: the call exports intermediate values or statistics, or uses a per-position step; the plain
+// instantiation carries none of those branches in its position loop.
+template <int D, int SRC, bool ZR, bool FLEX>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     constexpr bool FROM_OPEN = SRC == kSrcOpen;
@@ -656,7 +661,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
                 }
                 float inv_delta_p = inv_delta, inv_delta2_p = inv_delta2;
                 int zero_q = ZR ? a.sh.zero_q : 0;
-                if (a.step_exp) {                                                  // adaptive step delta * 2^e
+                if (FLEX && a.step_exp) {                                          // adaptive step delta * 2^e
                     const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
                     inv_delta_p = ldexpf(inv_delta, -e);
                     inv_delta2_p = ldexpf(inv_delta2, -2 * e);
@@ -669,7 +674,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
 #pragma unroll
                 for (int g = 0; g < G; ++g) sym[g] = quantise(kvv[g], mu[g], inv_delta_p);
                 __syncwarp();                                                     // readers of this slot are done
-                if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
+                if (FLEX && (a.dbg.sym || a.dbg.q || a.dbg.mu)) {
                     const long long o = ((long long)it.s * a.n + it.p0 + p) * Wt + it.t;
                     if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
 #pragma unroll
@@ -682,18 +687,17 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
             if (ZR && skip) { ++n_skipped; continue; }                             // nothing is coded
             int s, qp;
             class_params(q, s, qp);
-            if (a.dbg.ideal) {                      // statistics only: log2(2^15 / f) + s raw bits (+ 32 per escape)
+            if (FLEX && a.dbg.ideal) {              // statistics only: log2(2^15 / f) + s raw bits (+ 32 per escape)
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    const int nh = -((sym[g] + (s ? (1 << (s - 1)) : 0)) >> s);
-                    const uint32_t zz0 = (uint32_t)((nh << 1) ^ (nh >> 31));
-                    const uint32_t f = tb.enc[qp - kQMin][min(zz0, (uint32_t)kEsc)].fc & 0xffffu;
-                    ideal += (float)(kProbBits + s) - log2f((float)f) + (zz0 > 2u * kHiMax ? 32.f : 0.f);
+                    const uint32_t at = (uint32_t)(((sym[g] + (s ? (1 << (s - 1)) : 0)) >> s) + kHiMax);
+                    const uint32_t f = tb.enc[qp - kQMin][min(at, (uint32_t)kEsc)].fc & 0xffffu;
+                    ideal += (float)(kProbBits + s) - log2f((float)f) + (at > 2u * kHiMax ? 32.f : 0.f);
                 }
             }
-            wp = encode_position<G>(sym, s, a.step_exp != nullptr, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
+            wp = encode_position<G>(sym, s, FLEX && a.step_exp != nullptr, tb.enc[qp - kQMin], x, stage, wp, lc, n_escapes);
         }
-        if (a.dbg.ideal) {
+        if (FLEX && a.dbg.ideal) {
             ideal = warp_sum(ideal);
             if (lane == 0) atomicAdd(&a.counters->ideal_bits, (double)ideal);
         }
@@ -702,7 +706,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) encode_kernel(const Co
     }
 }
 
-template <int D, bool DENSE, bool ZR>
+template <int D, bool DENSE, bool ZR, bool FLEX>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     __shared__ DecTables tb;
@@ -770,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
             }
             float delta_p = delta, inv_delta2_p = inv_delta2;
             int zero_q = ZR ? a.sh.zero_q : 0;
-            if (a.step_exp) {
+            if (FLEX && a.step_exp) {
                 const int e = __ldg(a.step_exp + (long long)it.s * a.n + it.p0 + p);
                 delta_p = ldexpf(delta, e);
                 inv_delta2_p = ldexpf(inv_delta2, -2 * e);
@@ -786,13 +790,13 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) decode_kernel(const Co
             } else {
                 int s, qp;
                 class_params(q, s, qp);
-                decode_position<G>(sym, s, a.step_exp != nullptr, tb.cum[qp - kQMin], tb.fc[qp - kQMin], x, words, rp, last, lc);
+                decode_position<G>(sym, s, FLEX && a.step_exp != nullptr, tb.cum[qp - kQMin], tb.fc[qp - kQMin], x, words, rp, last, lc);
 #pragma unroll
                 for (int g = 0; g < G; ++g) out[g] = __fmaf_rn((float)sym[g], delta_p, mu[g]);
             }
             store_vec<G>(a.kv.base, kvo, out, a.sh.out_dtype);
             kvo += a.kv.sp;
-            if (a.dbg.sym || a.dbg.q || a.dbg.mu) {
+            if (FLEX && (a.dbg.sym || a.dbg.q || a.dbg.mu)) {
                 const long long o = ((long long)it.s * a.n + it.p0 + p) * Wt + it.t;
                 if (a.dbg.q && lane == 0) a.dbg.q[o] = q;
 #pragma unroll
@@ -1033,14 +1037,18 @@ cudaError_t launch_encode(const CodecArgs& a0, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int) * kTicketWords, st);
     if (e != cudaSuccess) return e;
     const bool zr = a.sh.zero_q != kZeroOff;
+    const bool flex = a.dbg.sym || a.dbg.q || a.dbg.mu || a.dbg.ideal || a.step_exp;
     return dispatch_d(a.sh.d, [&](auto D) {
+        constexpr int d = decltype(D)::value;
         if (a.mu_dense) {
-            auto kd = zr ? encode_kernel<decltype(D)::value, kSrcDense, true> : encode_kernel<decltype(D)::value, kSrcDense, false>;
+            auto kd = zr ? (flex ? encode_kernel<d, kSrcDense, true, true> : encode_kernel<d, kSrcDense, true, false>)
+                         : (flex ? encode_kernel<d, kSrcDense, false, true> : encode_kernel<d, kSrcDense, false, false>);
             kd<<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
             count_launch();
             return cudaGetLastError();
         }
-        auto kern = zr ? encode_kernel<decltype(D)::value, kSrcGather, true> : encode_kernel<decltype(D)::value, kSrcGather, false>;
+        auto kern = zr ? (flex ? encode_kernel<d, kSrcGather, true, true> : encode_kernel<d, kSrcGather, true, false>)
+                       : (flex ? encode_kernel<d, kSrcGather, false, true> : encode_kernel<d, kSrcGather, false, false>);
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
@@ -1057,7 +1065,7 @@ cudaError_t launch_append_seal(const CodecArgs& a, cudaStream_t st) {
         long long warps = (long long)a.open_items;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
         if (blocks > (long long)sm_count() * kBlocksPerSM) blocks = (long long)sm_count() * kBlocksPerSM;
-        auto ko = a.sh.zero_q != kZeroOff ? encode_kernel<decltype(D)::value, kSrcOpen, true> : encode_kernel<decltype(D)::value, kSrcOpen, false>;
+        auto ko = a.sh.zero_q != kZeroOff ? encode_kernel<decltype(D)::value, kSrcOpen, true, false> : encode_kernel<decltype(D)::value, kSrcOpen, false, false>;
         ko<<<(unsigned)blocks, kThreads, 0, st>>>(a);
         count_launch();
         return cudaGetLastError();
@@ -1070,14 +1078,18 @@ cudaError_t launch_decode(const CodecArgs& a0, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int) * kTicketWords, st);
     if (e != cudaSuccess) return e;
     const bool zr = a.sh.zero_q != kZeroOff;
+    const bool flex = a.dbg.sym || a.dbg.q || a.dbg.mu || a.step_exp;
     return dispatch_d(a.sh.d, [&](auto D) {
+        constexpr int d = decltype(D)::value;
         if (a.mu_dense) {
-            auto kd = zr ? decode_kernel<decltype(D)::value, true, true> : decode_kernel<decltype(D)::value, true, false>;
+            auto kd = zr ? (flex ? decode_kernel<d, true, true, true> : decode_kernel<d, true, true, false>)
+                         : (flex ? decode_kernel<d, true, false, true> : decode_kernel<d, true, false, false>);
             kd<<<sm_count() * kBlocksPerSM, kThreads, 0, st>>>(a);
             count_launch();
             return cudaGetLastError();
         }
-        auto kern = zr ? decode_kernel<decltype(D)::value, false, true> : decode_kernel<decltype(D)::value, false, false>;
+        auto kern = zr ? (flex ? decode_kernel<d, false, true, true> : decode_kernel<d, false, true, false>)
+                       : (flex ? decode_kernel<d, false, false, true> : decode_kernel<d, false, false, false>);
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
