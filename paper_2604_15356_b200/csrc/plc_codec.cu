@@ -184,9 +184,16 @@ __device__ __forceinline__ void predict(const char* __restrict__ col, const floa
 // The pairs of a position are brought into the warp's shared-memory slot with cp.async, one
 // position ahead of their use and without passing through registers (two slots per warp).
 __device__ __forceinline__ void prefetch_pairs(int2* sp, const int2* __restrict__ gp, int Kp, int lane) {
-    for (int k = lane; k < Kp; k += 32) {
-        const unsigned dst = (unsigned)__cvta_generic_to_shared(sp + k);
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(gp + k) : "memory");
+    if ((Kp & 1) == 0) {                            // two entries (16 bytes) per copy: the slots and the rows of `pairs` are 16-byte aligned
+        for (int k = 2 * lane; k < Kp; k += 64) {
+            const unsigned dst = (unsigned)__cvta_generic_to_shared(sp + k);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gp + k) : "memory");
+        }
+    } else {
+        for (int k = lane; k < Kp; k += 32) {
+            const unsigned dst = (unsigned)__cvta_generic_to_shared(sp + k);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(gp + k) : "memory");
+        }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -532,7 +539,7 @@ __device__ __forceinline__ int quantise(float kv, float mu, float inv_delta) {
     return (int)n;
 }
 
-extern __shared__ int2 g_pair_smem[];   // per warp: two slots of Kp entries
+extern __shared__ __align__(16) int2 g_pair_smem[];   // per warp: two slots of Kp entries
 
 // Prediction read from the dense variant's buffers: mu [row][tables_in_layer*D] and the variance
 // term s1 [row][tables_in_layer] (sum_v p_v ||T_v||^2 / d); sigma2 = max(0, s1 - ||mu||^2 / d).
