@@ -57,7 +57,7 @@ def parse_over(pairs):
 
 # Issue-slot use of the fused kernels (smsp__issue_active) from the ncu capture summarised in
 # profiles/fused_kernels_mid_L4.md; quoted beside the roofline fraction, not part of it.
-NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.649, "decode_kernel": 0.640}
+NCU_ISSUE_SLOT_USE = {"encode_kernel": 0.637, "decode_kernel": 0.638}
 
 
 def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, peak, peak_kind, traffic_per_vector=None):
@@ -84,7 +84,7 @@ def fused_roofline(vecs, K, d, t_bytes, kv_bytes, payload, ek, dk, sm_mhz, sms, 
          "fp32_fma": {"achieved": flop_ach, "peak": flop_peak, "unit": "TFLOP/s", "frac": alu_frac,
                       "peak_kind": "SMs x 128 lanes x 2 flop x sampled SM clock (%d x %.0f MHz)" % (sms, sm_mhz)},
          "issue_slot_use_ncu": NCU_ISSUE_SLOT_USE.get(name),
-         "busiest_units_ncu": "heavy half of the FMA pipe 66 %, L1 data pipe 60 %, issue slots 64 % "
+         "busiest_units_ncu": "heavy half of the FMA pipe 67 %, L1 data pipe 60 %, issue slots 64 % "
                               "(profiles/fused_kernels_mid_L4.md: no single unit saturated)",
          "gathered_row_bytes_frac": bytes_ns / sec / 1e9 / peak,
          "gathered_row_note": "KV + K*d*2 B of gathered rows per vector + bitstream over the HBM copy peak; the rows are "
@@ -140,7 +140,7 @@ class ClockSampler:
 # DRAM bytes per vector of the fused kernels, from the ncu capture summarised in
 # profiles/fused_kernels_mid_L4.md (dram__bytes_read.sum + dram__bytes_write.sum over 4.19 M vectors;
 # traffic grows in proportion to the vectors).  Valid for the default workload and chunk size only.
-NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.6, "decode_kernel": 433.2}
+NCU_DRAM_BYTES_PER_VECTOR = {"encode_kernel": 671.0, "decode_kernel": 433.1}
 NCU_TRAFFIC_NOTE = ("dram__bytes_read + dram__bytes_write of a 4-layer ncu capture (profiles/fused_kernels_mid_L4.md) "
                     "scaled by the vectors of a launch")
 
