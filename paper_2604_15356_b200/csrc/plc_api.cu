@@ -106,7 +106,7 @@ int padded_k(const plc_config& cfg) {
 // Scratch of the two-kernel selection: headers first (16 bytes per row), then the lists.
 size_t cand_word_bytes(const plc_config& cfg) { return cfg.vocab <= 65536 ? 4 : 8; }
 size_t cand_bytes(const plc_config& cfg, long long positions) {
-    return (size_t)positions * (16 + (size_t)kTopkListCap * cand_word_bytes(cfg));
+    return (size_t)positions * (16 + (size_t)kTopkListCap * cand_word_bytes(cfg)) + 16;   // + the redo counter
 }
 void set_cand(const plc_ctx* c, TopkArgs& a, long long positions);
 
@@ -126,6 +126,7 @@ plc_status ensure_pairs(plc_ctx* c, long long positions) {
 void set_cand(const plc_ctx* c, TopkArgs& a, long long positions) {
     a.cand_hdr = reinterpret_cast<float4*>(c->cand);
     a.cand = c->cand + (size_t)positions * 16;
+    a.redo = reinterpret_cast<unsigned int*>(c->cand + (size_t)positions * (16 + (size_t)kTopkListCap * cand_word_bytes(c->cfg)));
 }
 
 CodecArgs base_args(const plc_ctx* c) {
@@ -299,7 +300,7 @@ plc_status plc_topk_softmax(plc_ctx* c, const void* logits_dev, const int32_t* t
     a.logits = static_cast<const __half*>(logits_dev); a.tokens = tokens_dev; a.N = N;
     a.V = c->cfg.vocab; a.K = c->cfg.top_k;
     a.idx = idx_dev; a.w = w_dev; a.lse = lse_dev; a.zk = zk_dev; a.logp2 = logp2_dev;
-    a.n_per_session = 1;
+    a.n_per_session = 1; a.status = c->status;
     if (idx_dev || w_dev || zk_dev) {                    // the selection uses the context's scratch
         plc_status rc = ensure_pairs(c, N);
         if (rc) return rc;
@@ -333,7 +334,7 @@ static plc_status run_topk_for(plc_ctx* c, const void* logits_dev, int S, int n,
     TopkArgs a{};
     a.logits = static_cast<const __half*>(logits_dev); a.N = (long long)S * n; a.V = c->cfg.vocab; a.K = c->cfg.top_k;
     a.pairs = c->pairs; a.Kp = padded_k(c->cfg); a.n_per_session = n; a.pos_begin = pb; a.pos_end = pe;
-    set_cand(c, a, c->pairs_cap);
+    set_cand(c, a, c->pairs_cap); a.status = c->status;
     if (tokens) {
         a.tokens = tokens; a.step_exp = c->step_exp; a.bits_out = bits_out;
         a.b0 = c->cfg.adaptive_b0; a.extra = c->cfg.adaptive_extra; a.hbar = c->cfg.adaptive_hbar;

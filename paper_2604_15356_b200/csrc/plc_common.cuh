@@ -160,6 +160,10 @@ struct TopkArgs {
     // V <= 65536) and a header {l_max, sum of exp(l - l_max), number of candidates or -1}.  With it
     // the streaming kernel only collects the candidates of a row and a second kernel ranks them.
     void* cand; float4* cand_hdr;
+    // Rows the shared-memory-staged kernel leaves to the general one carry -2 in their header and are
+    // counted in *redo; a launch with redo_only set visits only those (and returns at once if none).
+    unsigned int* redo; int redo_only;
+    unsigned int* status;   // device status word (bounded waits report kStTimeout there), or null
 };
 constexpr int kTopkListCap = 256;
 cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st);

@@ -23,6 +23,7 @@ namespace {
 
 constexpr int kBins = 4096;
 constexpr int kCandCap = 1024;
+constexpr int kHdrRedo = -2;                        // header mark: the row is left to the general kernel
 
 __device__ __forceinline__ uint32_t key_of(uint32_t u) {
     u &= 0xffffu;
@@ -310,12 +311,14 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     uint32_t* list32 = sm.hist;
     unsigned long long* list64 = reinterpret_cast<unsigned long long*>(sm.hist);
 
+    if (a.redo_only && *a.redo == 0) return;                             // nothing was left over
     for (long long rowi = blockIdx.x; rowi < a.N; rowi += gridDim.x) {
         if (a.pos_begin || a.pos_end) {
             int s = (int)(rowi / a.n_per_session), i = (int)(rowi % a.n_per_session);
             int b = a.pos_begin ? a.pos_begin[s] : 0, e = a.pos_end ? a.pos_end[s] : a.n_per_session;
             if (i < b || i >= e) continue;
         }
+        if (a.redo_only && __float_as_int(a.cand_hdr[rowi].z) != kHdrRedo) continue;
         const __half* row = a.logits + rowi * (long long)V;
         if (tid == 0) { sm.nlist = 0; sm.nhit = 0; }
 
@@ -529,6 +532,205 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
     }
 }
 
+// ---- rows that fit in shared memory -------------------------------------------------------------
+// The same row work as the fast path above, but the row is brought into shared memory ONCE by a
+// bulk asynchronous copy (one instruction of one thread, completion on an mbarrier) and both passes
+// and the taking apart of the noted groups read it there: the second pass costs no L2 round trips,
+// no registers hold loads in flight, and the copy of a block's next row runs under the tail of the
+// current one.  Three blocks per SM keep about 190 KB of copies or rows per SM in flight.  Rows
+// whose candidates do not fit the hand-over (ties, more than 256 at or above the bound) are marked
+// for the general kernel.  Every wait on the barrier is bounded.
+constexpr int kStageBytes = 64 * 1024;             // largest row buffer: V <= 32768 binary16 logits
+__host__ __device__ constexpr int stage_row_bytes(int V) { return (V * 2 + 127) & ~127; }
+constexpr int kStageThreads = 256;
+constexpr uint32_t kStageSpin = 1u << 24;
+
+struct __align__(16) StageSm {
+    unsigned long long bar;
+    uint32_t list[kCandCap];
+    int32_t hit[kCandCap];
+    uint32_t red_k[kStageThreads / 32];
+    uint32_t red_t[kStageThreads / 32];
+    float red_s[kStageThreads / 32];
+    int nlist, nhit;
+};
+
+__device__ __forceinline__ bool stage_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kStageSpin; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+// The row after `rowi` (stride: the grid) that lies inside its session's position range, or N.
+__device__ __forceinline__ long long stage_next_row(const TopkArgs& a, long long rowi) {
+    for (; rowi < a.N; rowi += gridDim.x) {
+        if (!(a.pos_begin || a.pos_end)) return rowi;
+        const int s = (int)(rowi / a.n_per_session), i = (int)(rowi % a.n_per_session);
+        const int b = a.pos_begin ? a.pos_begin[s] : 0, e = a.pos_end ? a.pos_end[s] : a.n_per_session;
+        if (i >= b && i < e) return rowi;
+    }
+    return a.N;
+}
+
+__global__ void __launch_bounds__(kStageThreads) topk_staged_kernel(TopkArgs a) {
+    constexpr int THREADS = kStageThreads, NW = THREADS / 32;
+    extern __shared__ __align__(128) unsigned char stage_raw[];
+    const __half* buf = reinterpret_cast<const __half*>(stage_raw);
+    StageSm& sm = *reinterpret_cast<StageSm*>(stage_raw + stage_row_bytes(a.V));
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int V = a.V, K = a.K;
+    const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
+    const int per_warp = (K + NW - 1) / NW;
+    const bool select = a.pairs || a.idx || a.w || a.zk;            // the launcher sends only rows of the fast path here
+    const uint32_t row_bytes = (uint32_t)V * 2u;
+    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&sm.bar);
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage_raw);
+
+    auto fetch = [&](long long rowi) {                               // one thread: the whole row in one copy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the buffer's last readers used ordinary loads
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(row_bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "l"(a.logits + rowi * (long long)V), "r"(row_bytes), "r"(bar) : "memory");
+    };
+
+    long long rowi = stage_next_row(a, blockIdx.x);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(1u) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0 && rowi < a.N) fetch(rowi);
+    uint32_t parity = 0;
+    while (rowi < a.N) {
+        const long long next = stage_next_row(a, rowi + gridDim.x);
+        if (tid == 0) { sm.nlist = 0; sm.nhit = 0; }
+        bool ok = stage_wait(bar, parity);
+        if (!ok) ok = stage_wait(bar, parity);                        // a copy in flight is waited for once more before giving up
+        if (__syncthreads_or(!ok)) {
+            if (tid == 0 && a.status) atomicOr(a.status, kStTimeout);
+            return;
+        }
+        parity ^= 1u;
+
+        // Pass 0: one maximum per thread.
+        uint32_t m2 = 0xfc00fc00u;                                   // (-inf, -inf)
+#pragma unroll 4
+        for (int t = 0; t < ntiles; ++t) {
+            const int i0 = t * (THREADS * 8) + tid * 8;
+            if (i0 < V) {
+                const uint4 r = *reinterpret_cast<const uint4*>(buf + i0);
+                m2 = hmax2_bits(m2, hmax2_bits(hmax2_bits(r.x, r.y), hmax2_bits(r.z, r.w)));
+            }
+        }
+        uint32_t tkey = max(key_of(m2 & 0xffffu), key_of(m2 >> 16));
+        if (tid * 8 >= V) tkey = 0;                                   // this thread owns nothing
+        const uint32_t wmax = __reduce_max_sync(kFull, tkey);
+        uint32_t wth = 0;
+        if (select) {
+            uint32_t v = tkey;
+            for (int r = 0; r < per_warp; ++r) {
+                wth = __reduce_max_sync(kFull, v);
+                const uint32_t eq = __ballot_sync(kFull, v == wth);
+                if (lane == __ffs(eq) - 1) v = 0;
+            }
+        }
+        if (lane == 0) { sm.red_k[wid] = wmax; sm.red_t[wid] = wth; }
+        __syncthreads();
+        uint32_t km = sm.red_k[0], theta = sm.red_t[0];
+#pragma unroll
+        for (int w = 1; w < NW; ++w) { km = max(km, sm.red_k[w]); theta = min(theta, sm.red_t[w]); }
+        theta = max(theta, kKeyNegInf);
+        const float lmax = val_of_key(km);
+
+        // Pass 1: sum of exp(l - l_max); groups of 8 with an element at or above the bound are noted.
+        const float nb = -lmax * 1.44269504088896341f;
+        const uint32_t tb = bits_of_key(theta);
+        const uint32_t th2 = tb | (tb << 16);
+        float s = 0.f;
+#pragma unroll 2
+        for (int t = 0; t < ntiles; ++t) {
+            const int i0 = t * (THREADS * 8) + tid * 8;
+            if (i0 < V) {
+                const uint4 r = *reinterpret_cast<const uint4*>(buf + i0);
+                const uint32_t wds[4] = {r.x, r.y, r.z, r.w};
+                const uint32_t top = hmax2_bits(hmax2_bits(r.x, r.y), hmax2_bits(r.z, r.w));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&wds[j]));
+                    s += exp_rel(f.x, nb);
+                    s += exp_rel(f.y, nb);
+                }
+                if (select && !__hblt2(*reinterpret_cast<const __half2*>(&top), *reinterpret_cast<const __half2*>(&th2))) {
+                    const int slot = atomicAdd(&sm.nhit, 1);
+                    if (slot < kCandCap) sm.hit[slot] = i0;
+                }
+            }
+        }
+        s = warp_sum(s);
+        if (lane == 0) sm.red_s[wid] = s;
+        __syncthreads();
+        float sum_all = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) sum_all += sm.red_s[w];
+        int nlist = 0;
+        if (select) {
+            const int nhit = sm.nhit;
+            if (nhit <= kCandCap) {
+                for (int t = tid; t < nhit; t += THREADS) {
+                    const int i0 = sm.hit[t];
+                    const uint4 r = *reinterpret_cast<const uint4*>(buf + i0);
+                    const uint32_t wds[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) collect2(wds[j], th2, i0 + 2 * j, true, &sm.nlist, sm.list);
+                }
+            }
+            __syncthreads();
+            nlist = nhit <= kCandCap ? sm.nlist : kCandCap + 1;
+        }
+        // the row buffer is free: the next row's copy runs under the rest of this one
+        if (tid == 0 && next < a.N) fetch(next);
+
+        const bool handed = select && nlist >= K && nlist <= kTopkListCap;
+        if (select) {
+            if (tid == 0) {
+                a.cand_hdr[rowi] = make_float4(lmax, sum_all, __int_as_float(handed ? nlist : kHdrRedo), 0.f);
+                if (!handed) atomicAdd(a.redo, 1u);
+            }
+            if (handed) {
+                uint32_t* out = static_cast<uint32_t*>(a.cand) + rowi * kTopkListCap;
+                for (int c = tid; c < nlist; c += THREADS) out[c] = sm.list[c];
+            }
+        }
+        if (tid == 0 && (!select || handed)) {                          // a row that is left over gets these from the general kernel
+            const float lse = lmax + logf(sum_all);
+            if (a.lse) a.lse[rowi] = lse;
+            if (a.tokens && (a.logp2 || a.step_exp || a.bits_out)) {
+                const int tk = a.tokens[rowi];
+                const float v = (tk >= 0 && tk < V) ? (__half2float(a.logits[rowi * (long long)V + tk]) - lse) * 1.44269504088896341f
+                                                    : __int_as_float(0x7fc00000);
+                if (a.logp2) a.logp2[rowi] = v;
+                if (a.step_exp || a.bits_out) {
+                    // Def. 7: b = max(1, floor(b0 h / hbar)), capped at b0 + extra; decided in binary32
+                    const float r = __fmul_rn((float)a.b0, __fdiv_rn(-v, a.hbar));
+                    int b = (r >= 1.0f) ? (int)floorf(r) : 1;
+                    b = min(b, a.b0 + a.extra);
+                    if (a.step_exp) a.step_exp[rowi] = a.b0 - b;
+                    if (a.bits_out) a.bits_out[rowi] = b;
+                }
+            }
+        }
+        __syncthreads();                                                 // sm.list, sm.nlist are free again
+        rowi = next;
+    }
+}
+
 // One compare-exchange step of a bitonic network on 256 order words held 8 per lane: word e = r * 32 +
 // lane sits in v[r].  K2 = the size of the bitonic blocks being merged, J = the distance.  The
 // network sorts descending overall.
@@ -633,13 +835,37 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
     // with five blocks per SM, longer rows by 512 threads with two blocks per SM (two, so that one
     // block streams while the other sits at the barrier between its passes).
     const bool wide = (long long)a.V * 2 > 128 * 1024;
+    TopkArgs g = a;                                           // what the general kernel is launched with
     auto launch = [&](auto kern, int threads, int cap) {
         int occ = 1;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, 0) != cudaSuccess || occ < 1) occ = 1;
         const long long per_sm = occ < cap ? occ : cap;       // the rows in flight stay within L2
         const long long blocks = a.N < sms * per_sm ? a.N : sms * per_sm;
-        kern<<<(unsigned)blocks, threads, 0, st>>>(a);
+        kern<<<(unsigned)blocks, threads, 0, st>>>(g);
     };
+    const bool select = a.pairs || a.idx || a.w || a.zk;
+    // Rows that fit in shared memory go through the staged kernel when it can finish them: no
+    // selection at all, or the hand-over to the ranking kernel (K <= 128 and the scratch for it).
+    const bool staged = vec && (long long)a.V * 2 <= kStageBytes &&
+                        (!select || (a.K <= 128 && a.cand && a.cand_hdr && a.redo));
+    cudaError_t e = cudaSuccess;
+    if (staged) {
+        const size_t smem = stage_row_bytes(a.V) + sizeof(StageSm);
+        e = cudaFuncSetAttribute(topk_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (select) {
+            e = cudaMemsetAsync(a.redo, 0, sizeof(unsigned int), st);
+            if (e != cudaSuccess) return e;
+        }
+        int occ = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, topk_staged_kernel, kStageThreads, smem) != cudaSuccess || occ < 1) occ = 1;
+        const long long blocks = a.N < (long long)sms * occ ? a.N : (long long)sms * occ;
+        topk_staged_kernel<<<(unsigned)blocks, kStageThreads, smem, st>>>(a);
+        count_launch();
+        e = cudaGetLastError();
+        if (e != cudaSuccess || !select) return e;
+        g.redo_only = 1;                                      // then only what the staged kernel left over
+    }
     if (wide) {
         if (vec) launch(topk_softmax_kernel<true, 512>, 512, 2);
         else launch(topk_softmax_kernel<false, 512>, 512, 2);
@@ -648,9 +874,8 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
         else launch(topk_softmax_kernel<false, 256>, 256, 5);
     }
     count_launch();
-    cudaError_t e = cudaGetLastError();
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const bool select = a.pairs || a.idx || a.w || a.zk;
     if (a.cand && a.cand_hdr && select && a.K <= 128) {
         const long long want = (a.N + 7) / 8, cap = (long long)sms * 8;
         const unsigned blocks = (unsigned)(want < cap ? want : cap);
