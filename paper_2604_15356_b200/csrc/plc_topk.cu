@@ -539,9 +539,17 @@ __global__ void __launch_bounds__(THREADS) topk_softmax_kernel(TopkArgs a) {
 // no registers hold loads in flight, and the copy of a block's next row runs under the tail of the
 // current one.  Three blocks per SM keep about 190 KB of copies or rows per SM in flight.  Rows
 // whose candidates do not fit the hand-over (ties, more than 256 at or above the bound) are marked
-// for the general kernel.  Every wait on the barrier is bounded.
+// for the general kernel.  A call that wants no selection (lse / log2 P only) may have rows longer
+// than the buffer: they pass through it in chunks, one HBM read and no L2 pass at all.  Every wait
+// on the barrier is bounded.
 constexpr int kStageBytes = 64 * 1024;             // largest row buffer: V <= 32768 binary16 logits
-__host__ __device__ constexpr int stage_row_bytes(int V) { return (V * 2 + 127) & ~127; }
+// A row longer than the buffer is staged in equal chunks (a multiple of 8 logits each); only calls
+// without a selection take such rows here: maximum and sum are carried from chunk to chunk.
+__host__ __device__ constexpr int stage_chunks(int V) { return (V * 2 + kStageBytes - 1) / kStageBytes; }
+__host__ __device__ constexpr int stage_chunk_elems(int V) {
+    return stage_chunks(V) <= 1 ? V : (((V + stage_chunks(V) - 1) / stage_chunks(V) + 7) & ~7);
+}
+__host__ __device__ constexpr int stage_buf_bytes(int V) { return (stage_chunk_elems(V) * 2 + 127) & ~127; }
 constexpr int kStageThreads = 256;
 constexpr uint32_t kStageSpin = 1u << 24;
 
@@ -583,33 +591,39 @@ __global__ void __launch_bounds__(kStageThreads) topk_staged_kernel(TopkArgs a) 
     constexpr int THREADS = kStageThreads, NW = THREADS / 32;
     extern __shared__ __align__(128) unsigned char stage_raw[];
     const __half* buf = reinterpret_cast<const __half*>(stage_raw);
-    StageSm& sm = *reinterpret_cast<StageSm*>(stage_raw + stage_row_bytes(a.V));
+    StageSm& sm = *reinterpret_cast<StageSm*>(stage_raw + stage_buf_bytes(a.V));
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const int V = a.V, K = a.K;
-    const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
+    const int Vrow = a.V, K = a.K;
+    const int nchunks = stage_chunks(Vrow), ce = stage_chunk_elems(Vrow);
     const int per_warp = (K + NW - 1) / NW;
-    const bool select = a.pairs || a.idx || a.w || a.zk;            // the launcher sends only rows of the fast path here
-    const uint32_t row_bytes = (uint32_t)V * 2u;
+    const bool select = a.pairs || a.idx || a.w || a.zk;            // the launcher sends only one-chunk rows of the fast path here with a selection
     const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&sm.bar);
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage_raw);
 
-    auto fetch = [&](long long rowi) {                               // one thread: the whole row in one copy
+    auto fetch = [&](long long rowi, int c) {                        // one thread: the whole chunk in one copy
+        const uint32_t bytes = (uint32_t)min(ce, Vrow - c * ce) * 2u;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the buffer's last readers used ordinary loads
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(row_bytes) : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst), "l"(a.logits + rowi * (long long)V), "r"(row_bytes), "r"(bar) : "memory");
+                     ::"r"(dst), "l"(a.logits + rowi * (long long)Vrow + (long long)c * ce), "r"(bytes), "r"(bar) : "memory");
     };
 
     long long rowi = stage_next_row(a, blockIdx.x);
+    int c = 0;
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(1u) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (tid == 0 && rowi < a.N) fetch(rowi);
+    if (tid == 0 && rowi < a.N) fetch(rowi, 0);
     uint32_t parity = 0;
+    float run_max = 0.f, run_sum = 0.f;                              // over the chunks of the row so far
     while (rowi < a.N) {
-        const long long next = stage_next_row(a, rowi + gridDim.x);
+        int next_c = c + 1;
+        long long next = rowi;
+        if (next_c == nchunks) { next_c = 0; next = stage_next_row(a, rowi + gridDim.x); }
+        const int V = min(ce, Vrow - c * ce);                        // logits in the buffer
+        const int ntiles = (V + THREADS * 8 - 1) / (THREADS * 8);
         if (tid == 0) { sm.nlist = 0; sm.nhit = 0; }
         bool ok = stage_wait(bar, parity);
         if (!ok) ok = stage_wait(bar, parity);                        // a copy in flight is waited for once more before giving up
@@ -694,40 +708,51 @@ __global__ void __launch_bounds__(kStageThreads) topk_staged_kernel(TopkArgs a) 
             __syncthreads();
             nlist = nhit <= kCandCap ? sm.nlist : kCandCap + 1;
         }
-        // the row buffer is free: the next row's copy runs under the rest of this one
-        if (tid == 0 && next < a.N) fetch(next);
+        // the buffer is free: the next copy runs under the rest of this row
+        if (tid == 0 && next < a.N) fetch(next, next_c);
 
-        const bool handed = select && nlist >= K && nlist <= kTopkListCap;
-        if (select) {
-            if (tid == 0) {
-                a.cand_hdr[rowi] = make_float4(lmax, sum_all, __int_as_float(handed ? nlist : kHdrRedo), 0.f);
-                if (!handed) atomicAdd(a.redo, 1u);
-            }
-            if (handed) {
-                uint32_t* out = static_cast<uint32_t*>(a.cand) + rowi * kTopkListCap;
-                for (int c = tid; c < nlist; c += THREADS) out[c] = sm.list[c];
-            }
+        // maximum and sum over the chunks so far (the same values in every thread)
+        float lmax_row = lmax, sum_row = sum_all;
+        if (c > 0) {
+            lmax_row = fmaxf(run_max, lmax);
+            sum_row = (run_max > -INFINITY ? run_sum * expf(run_max - lmax_row) : 0.f) +
+                      (lmax > -INFINITY ? sum_all * expf(lmax - lmax_row) : 0.f);
         }
-        if (tid == 0 && (!select || handed)) {                          // a row that is left over gets these from the general kernel
-            const float lse = lmax + logf(sum_all);
-            if (a.lse) a.lse[rowi] = lse;
-            if (a.tokens && (a.logp2 || a.step_exp || a.bits_out)) {
-                const int tk = a.tokens[rowi];
-                const float v = (tk >= 0 && tk < V) ? (__half2float(a.logits[rowi * (long long)V + tk]) - lse) * 1.44269504088896341f
-                                                    : __int_as_float(0x7fc00000);
-                if (a.logp2) a.logp2[rowi] = v;
-                if (a.step_exp || a.bits_out) {
-                    // Def. 7: b = max(1, floor(b0 h / hbar)), capped at b0 + extra; decided in binary32
-                    const float r = __fmul_rn((float)a.b0, __fdiv_rn(-v, a.hbar));
-                    int b = (r >= 1.0f) ? (int)floorf(r) : 1;
-                    b = min(b, a.b0 + a.extra);
-                    if (a.step_exp) a.step_exp[rowi] = a.b0 - b;
-                    if (a.bits_out) a.bits_out[rowi] = b;
+        run_max = lmax_row; run_sum = sum_row;
+
+        if (next_c == 0) {                                               // last chunk: the row is complete
+            const bool handed = select && nlist >= K && nlist <= kTopkListCap;
+            if (select) {
+                if (tid == 0) {
+                    a.cand_hdr[rowi] = make_float4(lmax_row, sum_row, __int_as_float(handed ? nlist : kHdrRedo), 0.f);
+                    if (!handed) atomicAdd(a.redo, 1u);
+                }
+                if (handed) {
+                    uint32_t* out = static_cast<uint32_t*>(a.cand) + rowi * kTopkListCap;
+                    for (int i = tid; i < nlist; i += THREADS) out[i] = sm.list[i];
+                }
+            }
+            if (tid == 0 && (!select || handed)) {                      // a row that is left over gets these from the general kernel
+                const float lse = lmax_row + logf(sum_row);
+                if (a.lse) a.lse[rowi] = lse;
+                if (a.tokens && (a.logp2 || a.step_exp || a.bits_out)) {
+                    const int tk = a.tokens[rowi];
+                    const float v = (tk >= 0 && tk < Vrow) ? (__half2float(a.logits[rowi * (long long)Vrow + tk]) - lse) * 1.44269504088896341f
+                                                           : __int_as_float(0x7fc00000);
+                    if (a.logp2) a.logp2[rowi] = v;
+                    if (a.step_exp || a.bits_out) {
+                        // Def. 7: b = max(1, floor(b0 h / hbar)), capped at b0 + extra; decided in binary32
+                        const float r = __fmul_rn((float)a.b0, __fdiv_rn(-v, a.hbar));
+                        int b = (r >= 1.0f) ? (int)floorf(r) : 1;
+                        b = min(b, a.b0 + a.extra);
+                        if (a.step_exp) a.step_exp[rowi] = a.b0 - b;
+                        if (a.bits_out) a.bits_out[rowi] = b;
+                    }
                 }
             }
         }
         __syncthreads();                                                 // sm.list, sm.nlist are free again
-        rowi = next;
+        rowi = next; c = next_c;
     }
 }
 
@@ -844,13 +869,14 @@ cudaError_t launch_topk(const TopkArgs& a, cudaStream_t st) {
         kern<<<(unsigned)blocks, threads, 0, st>>>(g);
     };
     const bool select = a.pairs || a.idx || a.w || a.zk;
-    // Rows that fit in shared memory go through the staged kernel when it can finish them: no
-    // selection at all, or the hand-over to the ranking kernel (K <= 128 and the scratch for it).
-    const bool staged = vec && (long long)a.V * 2 <= kStageBytes &&
-                        (!select || (a.K <= 128 && a.cand && a.cand_hdr && a.redo));
+    // The staged kernel takes what it can finish: calls without a selection (rows of any length, in
+    // chunks), and rows that fit in its buffer when the selection can be handed to the ranking
+    // kernel (K <= 128 and the scratch for it).
+    const bool staged = vec && (select ? (long long)a.V * 2 <= kStageBytes && a.K <= 128 && a.cand && a.cand_hdr && a.redo
+                                       : a.V < (1 << 30));
     cudaError_t e = cudaSuccess;
     if (staged) {
-        const size_t smem = stage_row_bytes(a.V) + sizeof(StageSm);
+        const size_t smem = stage_buf_bytes(a.V) + sizeof(StageSm);
         e = cudaFuncSetAttribute(topk_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (select) {

@@ -188,12 +188,18 @@ def test_topk_softmax_parity(dev, orc):
         np.testing.assert_allclose(out["lse"].cpu().numpy(), lse, atol=2e-5)
         np.testing.assert_allclose(out["zk"].cpu().numpy(), zk, rtol=2e-5)
         np.testing.assert_allclose(out["logp2"].cpu().numpy(), lp, atol=1e-4)
+        # a call that asks for no selected set takes its own route (rows staged in shared memory, rows
+        # longer than the buffer in chunks with a running maximum and sum): same lse and log2 P
+        only = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev), want=("lse", "logp2"))
+        np.testing.assert_allclose(only["lse"].cpu().numpy(), lse, atol=2e-5)
+        np.testing.assert_allclose(only["logp2"].cpu().numpy(), lp, atol=1e-4)
+        assert ctx.sync_status() == plc.OK
         again = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev))
         for k in out:
             assert torch.equal(out[k], again[k])                  # run-to-run identical
-        only = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev), want=("lse", "logp2"))
-        assert set(only) == {"lse", "logp2"}                      # no selected set asked for: the selection is skipped
-        assert torch.equal(only["lse"], out["lse"]) and torch.equal(only["logp2"], out["logp2"])
+        only2 = ctx.topk_softmax(torch.from_numpy(lg).to(dev), torch.from_numpy(tok).to(dev), want=("lse", "logp2"))
+        assert set(only2) == {"lse", "logp2"}                     # no selected set asked for: the selection is skipped
+        assert torch.equal(only2["lse"], only["lse"]) and torch.equal(only2["logp2"], only["logp2"])   # run-to-run identical
 
 
 def test_status_and_profiling_read_outs(dev):
