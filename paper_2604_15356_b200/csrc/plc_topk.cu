@@ -550,7 +550,10 @@ __host__ __device__ constexpr int stage_chunk_elems(int V) {
     return stage_chunks(V) <= 1 ? V : (((V + stage_chunks(V) - 1) / stage_chunks(V) + 7) & ~7);
 }
 __host__ __device__ constexpr int stage_buf_bytes(int V) { return (stage_chunk_elems(V) * 2 + 127) & ~127; }
-constexpr int kStageThreads = 256;
+#ifndef PLC_STAGE_THREADS
+#define PLC_STAGE_THREADS 256
+#endif
+constexpr int kStageThreads = PLC_STAGE_THREADS;
 constexpr uint32_t kStageSpin = 1u << 24;
 
 struct __align__(16) StageSm {
