@@ -14,6 +14,9 @@
 // a 4096-bin histogram of the order-preserving 16-bit key finds the bin that holds the K-th largest,
 // a 16-way refinement finds the key itself, and equal keys are taken in index order.
 // Reductions use warp shuffles in a fixed order, so results are bit-reproducible from run to run.
+// Rows that fit a 64 KB shared-memory buffer (and rows of any length when no selection is asked for)
+// first go through topk_staged_kernel further down, which does the same row work on a copy of the
+// row in shared memory; this kernel then takes only what that one marks as left over.
 #include <type_traits>
 
 #include "plc_common.cuh"
