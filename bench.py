@@ -438,6 +438,9 @@ def main():
                     help="standard deviation added in quadrature to the mixture's before the scale class is taken")
     ap.add_argument("--zero-rate", type=float, default=0.0,
                     help="D > 0: zero-rate rule (Thm. 3), positions with mixture variance <= D carry no symbols")
+    ap.add_argument("--topk-only", action="store_true",
+                    help="time the top-K softmax call alone on synthetic logits (V and K of --workload; rows chosen so "
+                         "that the input is about 1 GB, larger than L2), with and without the selection")
     ap.add_argument("--shard", default=None, choices=["layers"],
                     help="with --gpus N: cut ONE batch across the ranks by layer (strong scaling) instead of one batch per rank")
     args = ap.parse_args()
@@ -462,6 +465,9 @@ def main():
     plc.build()
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    if args.topk_only:
+        print(json.dumps(topk_arm(args, torch, plc, workloads, dev)))
+        return 0
     if args.workload == "append":
         print(json.dumps(append_arm(args, torch, plc, workloads, dev)))
         return 0
@@ -723,6 +729,49 @@ def dedup_arm(args, torch, plc, workloads, dev):
                                           "decode calls scan the logits of the coded positions once more each"},
             "gpu_launches": launches, "clocks": clocks}
     return line
+
+
+def topk_arm(args, torch, plc, workloads, dev):
+    """The top-K softmax call by itself: N rows of V seeded logits (N*V*2 bytes of about 1 GB, so every call
+    reads its input from HBM), once with the K largest, their weights, lse, Z_k and log2 P asked for, once
+    with lse / log2 P only.  CUDA events around 100 x `--steps` calls after `--warmup`."""
+    shapes = {"dedup": (128256, 64), "tiny": (256, 16)}
+    V, K = shapes.get(args.workload, (32000, 64))
+    over = parse_over(args.set)
+    V, K = int(over.get("V", V)), int(over.get("K", K))
+    N = max(1, int(over.get("N", (1 << 30) // (2 * V))))
+    g = torch.Generator(device=dev); g.manual_seed(20260415)
+    logits = (torch.randn(N, V, device=dev, generator=g) * 3.0).to(torch.float16)
+    tokens = torch.randint(0, V, (N,), device=dev, dtype=torch.int32, generator=g)
+    ctx = plc.Context(torch.zeros(1, 2, 1, V, 32, dtype=torch.float16, device=dev), K, 0.02)
+    peak, kind = measured_peaks()
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+    launches0 = plc.launch_count()
+    out = {}
+    for name, want in (("with_selection", ("idx", "w", "lse", "zk", "logp2")), ("lse_logp2_only", ("lse", "logp2"))):
+        for _ in range(max(args.warmup, 3)):
+            ctx.topk_softmax(logits, tokens, want=want)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        calls = 100 * args.steps                       # long enough for the clock sampler to see the region
+        e0.record()
+        for _ in range(calls):
+            ctx.topk_softmax(logits, tokens, want=want)
+        e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / calls
+        gbs = N * V * 2 / (ms / 1e3) / 1e9
+        out[name] = {"ms_per_call": ms, "achieved": gbs, "unit": "GB/s", "frac": gbs / peak}
+    assert ctx.sync_status() == plc.OK
+    clocks = sampler.stop()
+    sel = out["with_selection"]
+    return {"metric": "logits rows/s through the top-K softmax call", "value": N / (sel["ms_per_call"] / 1e3), "unit": "rows/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": sel["ms_per_call"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "top-K softmax alone", "rows": N, "V": V, "K": K, "l2": "input of %.2f GB, larger than L2" % (N * V * 2 / 1e9)},
+            "roofline": {"kernel": "topk_staged_kernel" if V * 2 <= 65536 else "topk_softmax_kernel", "bound": "hbm",
+                         "achieved": sel["achieved"], "peak": peak, "unit": "GB/s", "frac": sel["frac"], "traffic": None,
+                         "peak_kind": kind, "accounting": "the logits once (rows * V * 2 bytes) over the whole call (all its kernels)"},
+            "modes": out, "gpu_launches": plc.launch_count() - launches0, "clocks": clocks}
 
 
 def rotq_arm(args, torch, plc, workloads, dev):
