@@ -937,9 +937,14 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) rotq_kernel(const Code
 }
 
 // Decode-time append: one warp per (session, table) predicts the new position and stores its
-// symbols and class in slot a.open_slot of the stream's open chunk.
+// symbols and class in slot a.open_slot of the stream's open chunk.  The rows come from HBM at
+// random, so what counts is row loads in flight: four blocks per SM (64 registers, the whole
+// unrolled batch of row loads issued before the first use) measured best.
+#ifndef PLC_APPEND_BLOCKS
+#define PLC_APPEND_BLOCKS 4
+#endif
 template <int D>
-__global__ void __launch_bounds__(kThreads) append_quantise_kernel(const CodecArgs a) {
+__global__ void __launch_bounds__(kThreads, PLC_APPEND_BLOCKS) append_quantise_kernel(const CodecArgs a) {
     constexpr int G = Geo<D>::G;
     const int lane = threadIdx.x & 31;
     const int Wt = 2 * a.sh.L * a.sh.H, H = a.sh.H, Kp = a.sh.Kp;
@@ -1126,11 +1131,14 @@ cudaError_t launch_append_quantise(const CodecArgs& a, cudaStream_t st) {
     return dispatch_d(a.sh.d, [&](auto D) {
         long long warps = (long long)a.S * 2 * a.sh.L * a.sh.H;
         long long blocks = (warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
-        if (blocks > (long long)sm_count() * 8) blocks = (long long)sm_count() * 8;
         auto kern = append_quantise_kernel<decltype(D)::value>;
         size_t sm = 0;
         cudaError_t e2 = pair_smem_bytes(kern, a.sh.Kp, sm);
         if (e2 != cudaSuccess) return e2;
+        // one wave: as many blocks as are resident together, each walking its share of the items
+        int occ = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, sm) != cudaSuccess || occ < 1) occ = 1;
+        if (blocks > (long long)sm_count() * occ) blocks = (long long)sm_count() * occ;
         kern<<<(unsigned)blocks, kThreads, sm, st>>>(a);
         count_launch();
         return cudaGetLastError();
